@@ -1,0 +1,110 @@
+"""Python face of the CPU oracle (TEST INFRASTRUCTURE ONLY).
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package; the CUDA library never does, and this package never imports the
+CUDA library or its binding.
+
+`build()` compiles `patconv_ref.c` with gcc into `libpatconv_ref.so` next to
+it; `conv()` runs one layer.  Floating-point inputs (fp32 or fp16 arrays) are
+widened to double exactly before the call, so the oracle's result is the
+double-precision value of the layer on the stored inputs.  Parity status:
+pinned (see the header of patconv_ref.c).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "patconv_ref.c")
+_LIB = os.path.join(_HERE, "libpatconv_ref.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle if the shared object is missing or stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        P = ctypes.c_void_p
+        I = ctypes.c_int
+        lib.patconv_ref_f64.argtypes = [P, P, P, P, I, P, I, I, I, I, I, I, I, P, P]
+        lib.patconv_ref_f64.restype = I
+        lib.patconv_ref_i64.argtypes = [P, P, P, P, I, P, I, I, I, I, I, I, I, P]
+        lib.patconv_ref_i64.restype = I
+        lib.patconv_ref_threads.restype = I
+        _lib = lib
+    return _lib
+
+
+def threads() -> int:
+    """Host threads the oracle uses (OpenMP's maximum)."""
+    return int(_load().patconv_ref_threads())
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def out_shape(h: int, w: int, stride: int):
+    return (h + 2 - 3) // stride + 1, (w + 2 - 3) // stride + 1
+
+
+def conv(x, w, pid, masks, bias=None, relu=False, stride=1, with_scale=False):
+    """One pattern-pruned 3x3 layer, padding 1.
+
+    x     [N,H,W,Cin]   float16/32/64, or uint8 for the integer layer
+    w     [Cout,Cin,3,3] same family as x (int8 for the integer layer); dense:
+          values at pruned positions are ignored
+    pid   [Cout,Cin] int16 pattern id per kernel, -1 = kernel removed
+    masks [P] uint16, bit 3*dy+dx = tap kept
+    bias  [Cout] float (int32 for the integer layer) or None
+    Returns y [N,Ho,Wo,Cout] as float64 (int64 for the integer layer); with
+    `with_scale` also S = |bias| + sum |w*x| per output (floating point only).
+    """
+    lib = _load()
+    x = np.asarray(x)
+    w = np.asarray(w)
+    n, h, wd, c_in = x.shape
+    c_out = w.shape[0]
+    if w.shape != (c_out, c_in, 3, 3):
+        raise ValueError("w must be [Cout,Cin,3,3]")
+    pid = np.ascontiguousarray(pid, dtype=np.int16)
+    masks = np.ascontiguousarray(masks, dtype=np.uint16)
+    if pid.shape != (c_out, c_in):
+        raise ValueError("pid must be [Cout,Cin]")
+    ho, wo = out_shape(h, wd, stride)
+    if x.dtype == np.uint8:
+        if w.dtype != np.int8:
+            raise ValueError("integer layer wants int8 weights")
+        xc = np.ascontiguousarray(x)
+        wc = np.ascontiguousarray(w)
+        bc = None if bias is None else np.ascontiguousarray(bias, dtype=np.int32)
+        y = np.empty((n, ho, wo, c_out), dtype=np.int64)
+        rc = lib.patconv_ref_i64(_ptr(xc), _ptr(wc), _ptr(pid), _ptr(masks), len(masks), _ptr(bc),
+                                 int(bool(relu)), n, h, wd, c_in, c_out, stride, _ptr(y))
+        if rc:
+            raise ValueError("oracle error %d" % rc)
+        return y
+    xc = np.ascontiguousarray(x, dtype=np.float64)
+    wc = np.ascontiguousarray(w, dtype=np.float64)
+    bc = None if bias is None else np.ascontiguousarray(bias, dtype=np.float64)
+    y = np.empty((n, ho, wo, c_out), dtype=np.float64)
+    s = np.empty_like(y) if with_scale else None
+    rc = lib.patconv_ref_f64(_ptr(xc), _ptr(wc), _ptr(pid), _ptr(masks), len(masks), _ptr(bc),
+                             int(bool(relu)), n, h, wd, c_in, c_out, stride, _ptr(y), _ptr(s))
+    if rc:
+        raise ValueError("oracle error %d" % rc)
+    return (y, s) if with_scale else y
