@@ -1,0 +1,198 @@
+/*
+ * libpatconv -- inference-time execution of a pattern-pruned 3x3 convolution
+ * layer on NVIDIA B200 (sm_100a).
+ *
+ * The layer (paper Sec. 2.1, "Pattern-Based Pruning"): every surviving 3x3
+ * kernel keeps the 4 weights of one shape out of a small library of pre-defined
+ * patterns; connectivity pruning removes whole kernels, i.e. cuts the link
+ * between one input and one output channel.  For every n, oy, ox, oc
+ *
+ *   y = act( bias[oc] + sum_{ic: kernel (oc,ic) survives} sum_{t in pattern(oc,ic)}
+ *                          W[oc][ic][t] * x[n][oy*s + dy(t) - 1][ox*s + dx(t) - 1][ic] )
+ *
+ * with t = 3*dy + dx, zero padding of 1, stride s in {1,2}, cross-correlation
+ * (no kernel flip), act = ReLU or identity.
+ *
+ * Plain C ABI: pointers and sizes only.  Every function returns a status code;
+ * nothing throws, aborts or traps.  Unless stated otherwise a pointer named
+ * *_host is host memory and *_dev is memory of the CUDA device the handle was
+ * packed for.
+ */
+#ifndef XGEN_PATCONV_H
+#define XGEN_PATCONV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct xgen_patconv_packed xgen_patconv_packed; /* opaque; owns host and device memory */
+
+typedef enum {
+    XGEN_OK = 0,
+    XGEN_ERR_INVALID_ARG = 1,  /* null pointer, misaligned pointer, non-positive size          */
+    XGEN_ERR_BAD_PATTERN = 2,  /* mask without exactly 4 of 9 bits, or pattern id out of range  */
+    XGEN_ERR_SHAPE = 3,        /* tensor extents that do not fit the packed layer or 32-bit indexing */
+    XGEN_ERR_UNSUPPORTED = 4,  /* stride, padding or data type outside what is built            */
+    XGEN_ERR_ALLOC = 5,        /* host or device allocation failed                               */
+    XGEN_ERR_CUDA = 6,         /* a CUDA runtime call failed, or the handle has no device copy   */
+    XGEN_ERR_TIMEOUT = 7       /* reserved for device-side bounded waits                         */
+} xgen_status;
+
+/* Numeric variants.  F32: x, W, y fp32.  F16_F32ACC: x, W, y IEEE fp16, bias
+ * fp32, sums and bias+ReLU in fp32, one round-to-nearest-even at the store.
+ * I8_I32: x uint8 (zero point 0), W int8, bias int32, y int32 (the exact
+ * integer sum, before any requantisation; scales are the caller's metadata). */
+typedef enum { XGEN_F32 = 0, XGEN_F16_F32ACC = 1, XGEN_I8_I32 = 2 } xgen_dtype;
+
+typedef struct {
+    int32_t c_in;                   /* input channels,  >= 1                                   */
+    int32_t c_out;                  /* output channels (filters), >= 1                         */
+    int32_t stride;                 /* 1 or 2                                                  */
+    int32_t pad;                    /* must be 1                                               */
+    xgen_dtype dtype;
+    int32_t num_patterns;           /* P, 1..126                                               */
+    const uint16_t *pattern_masks;  /* [P] host; bit (3*dy+dx) set = tap kept; popcount 4      */
+} xgen_patconv_desc;
+
+/* What xgen_patconv_query reports about a packed layer. */
+typedef struct {
+    int64_t kernels_total;        /* c_in * c_out                                             */
+    int64_t kernels_surviving;    /* kernels with a pattern (not removed)                     */
+    int64_t macs_per_pixel;       /* 4 * kernels_surviving: useful multiply-adds per output pixel */
+    int64_t weight_bytes;         /* bytes of kept weights at the layer's storage precision   */
+    int64_t index_bytes;          /* bytes a compact encoding of this layout spends on
+                                     everything that is not a weight: one opcode byte and one
+                                     operand byte per command, plus the offset and slot tables */
+    int64_t csr_index_bytes;      /* index bytes CSR would need for the same non-zeros
+                                     (one 4-byte column per weight + one row pointer per filter) */
+    int64_t stream_bytes;         /* bytes of the command stream as stored on the device      */
+    int32_t filters_per_group;    /* J: filters one warp accumulates together                 */
+    int32_t groups_per_block;     /* filter groups (warps) per thread block                   */
+    int32_t n_blocks;             /* blocks of contiguous output channels                     */
+    int32_t channels_per_chunk;   /* input channels staged per pipeline step                  */
+    int32_t n_chunks;
+    int32_t patterns_compiled;    /* size of the compiled pattern table the layer runs with   */
+    int32_t max_segment_slots;    /* longest per-(block, chunk) command segment               */
+    int64_t load_commands;        /* activation-patch loads in the stream (one per group and
+                                     input channel that group is connected to)                */
+    double  group_imbalance;      /* max over groups / mean over groups of surviving kernels  */
+} xgen_patconv_stats;
+
+/* Read-only view of the packed layout on the host, for inspection and tests.
+ * All pointers belong to the handle.
+ *
+ * The stream is an array of 32-byte command slots (8 words):
+ *   word 0  opcode:  p < patterns_compiled  -> kernel command with compiled pattern p
+ *                    patterns_compiled      -> LOAD: fetch the activation patch of one channel
+ *                    patterns_compiled + 1  -> END of this group's commands for the chunk
+ *   word 1  operand: kernel command: 8 * j (j = filter slot inside the group);
+ *                    LOAD: channel index inside the chunk
+ *   word 4..7  kernel command: the four kept weights in ascending tap order, fp32 bit
+ *              patterns (fp16 and int8 weights are widened exactly)
+ * Slots are ordered [block][chunk][group]: seg_off[(b * n_chunks + c) * (G + 1) + g]
+ * (G = groups_per_block) is the first slot of group g of block b in chunk c, and
+ * entry g = G is one past the segment.  Inside a group's run every LOAD is
+ * followed by the kernel commands of that channel, and the run ends with END.
+ * slot_oc[(b * G + g) * J + j] is the original output channel of filter slot j,
+ * or -1 for an empty slot. */
+typedef struct {
+    const uint32_t *slots;          int64_t n_slots;
+    const int32_t  *seg_off;        /* [n_blocks * n_chunks * (G + 1)]                         */
+    const int32_t  *slot_oc;        /* [n_blocks * G * J]                                      */
+    const uint16_t *compiled_masks; /* [patterns_compiled]                                     */
+} xgen_patconv_host_view;
+
+/*
+ * Pack one layer (paper Sec. 2.3, "Filter Kernel Reorder and Compact FKW
+ * Storage": patterns are known after training, so filters are regrouped and
+ * each filter's kernels reordered offline, and the weights are stored with one
+ * index per kernel rather than per weight).
+ *   dense_w_host    [c_out][c_in][3][3]: fp32 (XGEN_F32), IEEE fp16 bits
+ *                   (XGEN_F16_F32ACC) or int8 (XGEN_I8_I32).  Values at pruned
+ *                   positions are ignored; they need not be zero.
+ *   pattern_id_host [c_out][c_in]: index into desc->pattern_masks, or -1 for a
+ *                   removed kernel.
+ *   device          CUDA device ordinal to upload to, or -1 to build the host
+ *                   layout only (no CUDA call is made; such a handle cannot run).
+ *   out             receives the handle; release it with xgen_patconv_free.
+ * Synchronous.  Inputs are copied; the caller may free them on return.
+ * Errors: INVALID_ARG, BAD_PATTERN, UNSUPPORTED (pad != 1, stride not 1|2),
+ * SHAPE, ALLOC, CUDA.
+ */
+xgen_status xgen_patconv_pack(const xgen_patconv_desc *desc, const void *dense_w_host,
+                              const int16_t *pattern_id_host, int device,
+                              xgen_patconv_packed **out);
+
+/*
+ * Run the layer (paper Sec. 2.3, "Load Redundancy Elimination": tiled input,
+ * per-pattern code with static tap offsets; Sec. 2.2: bias and ReLU fused).
+ *   x_dev    [n][h][w][c_in]  NHWC, dtype's activation type, 16-byte aligned
+ *   bias_dev [c_out] fp32 (int32 for XGEN_I8_I32) or NULL for no bias
+ *   relu     non-zero applies max(.,0)
+ *   y_dev    [n][ho][wo][c_out] NHWC, 16-byte aligned, must not overlap x_dev;
+ *            ho, wo as xgen_patconv_out_shape reports
+ *   cuda_stream  a cudaStream_t passed as void* (NULL = default stream)
+ * Only enqueues work on the stream: no synchronisation, no allocation.  The
+ * caller keeps x, bias and y alive until the stream reaches that work.  The
+ * handle is not modified, so concurrent calls on different streams are allowed
+ * (for a shape prepared with xgen_patconv_plan, which uses a workspace owned by
+ * the handle, concurrent calls must be on one stream).
+ * Errors: INVALID_ARG, SHAPE (n,h,w < 1 or a tensor beyond 2^31-1 elements),
+ * CUDA (launch failure or host-only handle).
+ */
+xgen_status xgen_patconv_run(const xgen_patconv_packed *packed, const void *x_dev, int32_t n,
+                             int32_t h, int32_t w, const void *bias_dev, int32_t relu,
+                             void *y_dev, void *cuda_stream);
+
+/*
+ * Convenience for callers that hold host tensors: copies x (and bias) to the
+ * device, runs the layer, copies y back and waits.  Allocates and frees device
+ * buffers on every call.  Same tensor layouts as xgen_patconv_run, all
+ * pointers host memory.  Errors as xgen_patconv_run, plus ALLOC.
+ */
+xgen_status xgen_patconv_run_host(const xgen_patconv_packed *packed, const void *x_host, int32_t n,
+                                  int32_t h, int32_t w, const void *bias_host, int32_t relu,
+                                  void *y_host);
+
+/*
+ * Optional: prepare the handle for one input shape.  Layers with few output
+ * pixels do not fill the GPU with (pixel tile x filter block) work items; for
+ * such a shape this call lets later xgen_patconv_run calls split the input
+ * channels across thread blocks and reduce the partial sums (the paper does
+ * not discuss this; it is the cross-channel reduction of this implementation).
+ * It allocates a workspace owned by the handle, so it synchronises and must not
+ * be called while the handle is in use.  Without it every shape runs unsplit.
+ * Errors: INVALID_ARG, SHAPE, ALLOC, CUDA.
+ */
+xgen_status xgen_patconv_plan(xgen_patconv_packed *packed, int32_t n, int32_t h, int32_t w);
+
+/* Output extents for an h x w input: ho = (h + 2 - 3) / stride + 1, likewise wo. */
+xgen_status xgen_patconv_out_shape(const xgen_patconv_packed *packed, int32_t h, int32_t w,
+                                   int32_t *ho, int32_t *wo);
+
+/* Fill *stats (see xgen_patconv_stats). */
+xgen_status xgen_patconv_query(const xgen_patconv_packed *packed, xgen_patconv_stats *stats);
+
+/* Fill *view with pointers into the handle's host copy of the packed layout. */
+xgen_status xgen_patconv_view(const xgen_patconv_packed *packed, xgen_patconv_host_view *view);
+
+/* Synchronise the stream and report the first CUDA error seen on it, as a
+ * status (XGEN_OK, XGEN_ERR_CUDA).  The kernels contain no unbounded waits. */
+xgen_status xgen_patconv_last_status(const xgen_patconv_packed *packed, void *cuda_stream);
+
+/* Release the handle and its device memory.  NULL is allowed. */
+void xgen_patconv_free(xgen_patconv_packed *packed);
+
+/* Static, human-readable name of a status code. */
+const char *xgen_strerror(xgen_status status);
+
+/* Number of kernel launches this library has enqueued in this process. */
+int64_t xgen_patconv_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XGEN_PATCONV_H */
