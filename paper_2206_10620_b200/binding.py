@@ -1,0 +1,187 @@
+"""Thin ctypes binding of libpatconv: argument marshalling only.
+
+Every step of the layer runs inside the CUDA library.  There is no CPU
+fallback: if the shared library cannot be loaded the import of this module's
+functions fails loudly.  PyTorch appears only at the call sites (device memory
+and streams); this module itself needs numpy and ctypes.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+from . import build as _build
+
+F32, F16_F32ACC, I8_I32 = 0, 1, 2
+DTYPES = {"f32": F32, "f16": F16_F32ACC, "i8": I8_I32}
+OK = 0
+STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_PATTERN", 3: "SHAPE", 4: "UNSUPPORTED",
+                5: "ALLOC", 6: "CUDA", 7: "TIMEOUT"}
+
+EXPORTS = ["xgen_patconv_pack", "xgen_patconv_run", "xgen_patconv_run_host", "xgen_patconv_plan",
+           "xgen_patconv_out_shape", "xgen_patconv_query", "xgen_patconv_view",
+           "xgen_patconv_last_status", "xgen_patconv_free", "xgen_strerror",
+           "xgen_patconv_launch_count"]
+
+
+class Desc(ctypes.Structure):
+    _fields_ = [("c_in", ctypes.c_int32), ("c_out", ctypes.c_int32), ("stride", ctypes.c_int32),
+                ("pad", ctypes.c_int32), ("dtype", ctypes.c_int), ("num_patterns", ctypes.c_int32),
+                ("pattern_masks", ctypes.c_void_p)]
+
+
+class Stats(ctypes.Structure):
+    _fields_ = [("kernels_total", ctypes.c_int64), ("kernels_surviving", ctypes.c_int64),
+                ("macs_per_pixel", ctypes.c_int64), ("weight_bytes", ctypes.c_int64),
+                ("index_bytes", ctypes.c_int64), ("csr_index_bytes", ctypes.c_int64),
+                ("stream_bytes", ctypes.c_int64),
+                ("filters_per_group", ctypes.c_int32), ("groups_per_block", ctypes.c_int32),
+                ("n_blocks", ctypes.c_int32), ("channels_per_chunk", ctypes.c_int32),
+                ("n_chunks", ctypes.c_int32), ("patterns_compiled", ctypes.c_int32),
+                ("max_segment_slots", ctypes.c_int32),
+                ("load_commands", ctypes.c_int64), ("group_imbalance", ctypes.c_double)]
+
+
+class HostView(ctypes.Structure):
+    _fields_ = [("slots", ctypes.c_void_p), ("n_slots", ctypes.c_int64),
+                ("seg_off", ctypes.c_void_p), ("slot_oc", ctypes.c_void_p),
+                ("compiled_masks", ctypes.c_void_p)]
+
+
+class PatconvError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__("%s failed: %s (%d)" % (where, STATUS_NAMES.get(status, "?"), status))
+
+
+_lib = None
+
+
+def lib():
+    """Load libpatconv.so (building it first if it is missing or stale)."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB_PATH
+        if not os.path.exists(path):
+            path = _build.build()
+        L = ctypes.CDLL(path)
+        P, I = ctypes.c_void_p, ctypes.c_int32
+        L.xgen_patconv_pack.argtypes = [ctypes.POINTER(Desc), P, P, ctypes.c_int, ctypes.POINTER(P)]
+        L.xgen_patconv_run.argtypes = [P, P, I, I, I, P, I, P, P]
+        L.xgen_patconv_run_host.argtypes = [P, P, I, I, I, P, I, P]
+        L.xgen_patconv_plan.argtypes = [P, I, I, I]
+        L.xgen_patconv_out_shape.argtypes = [P, I, I, ctypes.POINTER(I), ctypes.POINTER(I)]
+        L.xgen_patconv_query.argtypes = [P, ctypes.POINTER(Stats)]
+        L.xgen_patconv_view.argtypes = [P, ctypes.POINTER(HostView)]
+        L.xgen_patconv_last_status.argtypes = [P, P]
+        L.xgen_patconv_free.argtypes = [P]
+        L.xgen_patconv_free.restype = None
+        L.xgen_strerror.argtypes = [ctypes.c_int]
+        L.xgen_strerror.restype = ctypes.c_char_p
+        L.xgen_patconv_launch_count.restype = ctypes.c_int64
+        for name in EXPORTS:
+            if name not in ("xgen_patconv_free", "xgen_strerror", "xgen_patconv_launch_count"):
+                getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def _check(status, where):
+    if status != OK:
+        raise PatconvError(status, where)
+
+
+class Packed:
+    """Owner of one xgen_patconv_packed handle."""
+
+    def __init__(self, c_in, c_out, stride, dtype, masks, dense_w, pattern_id, device=0, pad=1):
+        self._h = ctypes.c_void_p()
+        self.dtype = DTYPES[dtype] if isinstance(dtype, str) else int(dtype)
+        self.c_in, self.c_out, self.stride = int(c_in), int(c_out), int(stride)
+        masks = np.ascontiguousarray(masks, dtype=np.uint16)
+        want = {F32: np.float32, F16_F32ACC: np.float16, I8_I32: np.int8}[self.dtype]
+        w = np.ascontiguousarray(dense_w, dtype=want)
+        pid = np.ascontiguousarray(pattern_id, dtype=np.int16)
+        if w.size != c_out * c_in * 9 or pid.size != c_out * c_in:
+            raise ValueError("dense_w must be [c_out,c_in,3,3] and pattern_id [c_out,c_in]")
+        d = Desc(c_in, c_out, stride, pad, self.dtype, len(masks), masks.ctypes.data)
+        _check(lib().xgen_patconv_pack(ctypes.byref(d), w.ctypes.data, pid.ctypes.data, int(device),
+                                       ctypes.byref(self._h)), "xgen_patconv_pack")
+
+    def close(self):
+        if self._h:
+            lib().xgen_patconv_free(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def out_shape(self, h, w):
+        ho, wo = ctypes.c_int32(), ctypes.c_int32()
+        _check(lib().xgen_patconv_out_shape(self._h, h, w, ctypes.byref(ho), ctypes.byref(wo)),
+               "xgen_patconv_out_shape")
+        return ho.value, wo.value
+
+    def stats(self) -> dict:
+        s = Stats()
+        _check(lib().xgen_patconv_query(self._h, ctypes.byref(s)), "xgen_patconv_query")
+        return {k: getattr(s, k) for k, _ in Stats._fields_}
+
+    def view(self) -> dict:
+        """Copies of the packed host arrays (see xgen_patconv_host_view)."""
+        v = HostView()
+        _check(lib().xgen_patconv_view(self._h, ctypes.byref(v)), "xgen_patconv_view")
+        st = self.stats()
+        J, G = st["filters_per_group"], st["groups_per_block"]
+        nb, nc, npc = st["n_blocks"], st["n_chunks"], st["patterns_compiled"]
+
+        def arr(ptr, n, ct, dt):
+            if n == 0:
+                return np.zeros(0, dt)
+            return np.ctypeslib.as_array(ctypes.cast(ptr, ctypes.POINTER(ct)), shape=(n,)).astype(dt, copy=True)
+
+        return {
+            "slots": arr(v.slots, v.n_slots * 8, ctypes.c_uint32, np.uint32).reshape(-1, 8),
+            "seg_off": arr(v.seg_off, nb * nc * (G + 1), ctypes.c_int32, np.int32).reshape(nb, nc, G + 1),
+            "slot_oc": arr(v.slot_oc, nb * G * J, ctypes.c_int32, np.int32).reshape(nb, G, J),
+            "masks": arr(v.compiled_masks, npc, ctypes.c_uint16, np.uint16),
+        }
+
+    def plan(self, n, h, w):
+        _check(lib().xgen_patconv_plan(self._h, n, h, w), "xgen_patconv_plan")
+
+    def run(self, x_ptr, n, h, w, bias_ptr, relu, y_ptr, stream=0):
+        """Enqueue the layer; all pointers are device addresses (ints)."""
+        _check(lib().xgen_patconv_run(self._h, x_ptr, n, h, w, bias_ptr or None, int(bool(relu)),
+                                      y_ptr, stream or None), "xgen_patconv_run")
+
+    def run_host(self, x: np.ndarray, bias, relu) -> np.ndarray:
+        """Host tensors in, host tensor out (copies inside the library)."""
+        n, h, w, c = x.shape
+        assert c == self.c_in and x.flags["C_CONTIGUOUS"]
+        ho, wo = self.out_shape(h, w)
+        ydt = {F32: np.float32, F16_F32ACC: np.float16, I8_I32: np.int32}[self.dtype]
+        y = np.empty((n, ho, wo, self.c_out), dtype=ydt)
+        b = None
+        if bias is not None:
+            b = np.ascontiguousarray(bias, dtype=np.int32 if self.dtype == I8_I32 else np.float32)
+        _check(lib().xgen_patconv_run_host(self._h, x.ctypes.data, n, h, w,
+                                           None if b is None else b.ctypes.data, int(bool(relu)),
+                                           y.ctypes.data), "xgen_patconv_run_host")
+        return y
+
+    def sync(self, stream=0):
+        _check(lib().xgen_patconv_last_status(self._h, stream or None), "xgen_patconv_last_status")
+
+
+def launch_count() -> int:
+    return int(lib().xgen_patconv_launch_count())
+
+
+def strerror(status: int) -> str:
+    return lib().xgen_strerror(int(status)).decode()

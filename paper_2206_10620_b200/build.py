@@ -1,0 +1,42 @@
+"""Build libpatconv.so in-tree with nvcc for sm_100a (cross-compiles without a GPU)."""
+from __future__ import annotations
+
+import os
+import subprocess
+import sys
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_CSRC = os.path.join(_HERE, "csrc")
+_INC = os.path.join(os.path.dirname(_HERE), "include")
+LIB_PATH = os.path.join(_HERE, "libpatconv.so")
+_SOURCES = ["patconv.cu", "pack.cpp"]
+_DEPS = _SOURCES + ["patconv_internal.h", "gen_core.py", os.path.join(_INC, "patconv.h")]
+
+
+def _stale() -> bool:
+    if not os.path.exists(LIB_PATH):
+        return True
+    t = os.path.getmtime(LIB_PATH)
+    return any(os.path.getmtime(os.path.join(_CSRC, d)) > t for d in _DEPS)
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Generate the per-pattern code, then compile and link the shared library."""
+    if not force and not _stale():
+        return LIB_PATH
+    gen = os.path.join(_CSRC, "core_gen.inc")
+    subprocess.check_call([sys.executable, os.path.join(_CSRC, "gen_core.py"), gen])
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    tmp = LIB_PATH + ".tmp%d" % os.getpid()
+    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
+           "-shared", "-Xcompiler", "-fPIC", "-I", _INC, "-I", _CSRC, "-o", tmp]
+    if verbose:
+        cmd += ["-Xptxas", "-v"]
+    cmd += [os.path.join(_CSRC, s) for s in _SOURCES]
+    subprocess.check_call(cmd)
+    os.replace(tmp, LIB_PATH)
+    return LIB_PATH
+
+
+if __name__ == "__main__":
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

@@ -1,0 +1,246 @@
+// Host-side packer: pattern masking, filter reorder, kernel reorder and the
+// compact command-stream layout (paper Sec. 2.3, "Filter Kernel Reorder and
+// Compact FKW Storage").  Pure C++, no CUDA.
+//
+// Layout idea.  A warp owns one *filter group* (J filters) for a tile of output
+// pixels; each thread keeps J x 8 running sums (in tensor memory).  For every
+// input channel the group is connected to, the warp loads the activation patch
+// of its pixels once into registers (a LOAD command) and then executes one
+// *kernel command* per surviving kernel of that channel: the command names the
+// filter slot (an address) and the pattern (the code to run), and carries the
+// four kept weights.  One small word pair per kernel replaces CSR's index per
+// weight, and because the pattern selects straight-line code with fixed
+// register operands there is no per-tap index and no branch inside a kernel.
+#include <algorithm>
+#include <array>
+#include <cstring>
+#include <numeric>
+
+#include "patconv_internal.h"
+
+namespace patconv {
+
+static int popcount9(unsigned m) {
+    int n = 0;
+    for (int t = 0; t < 9; ++t) n += (m >> t) & 1;
+    return n;
+}
+
+uint16_t compiled_mask(int np, int idx) {
+    if (np <= kNumLibraryMasks) return kLibraryMasks[idx];
+    int k = 0;
+    for (unsigned m = 0; m < 512; ++m)
+        if (popcount9(m) == 4) {
+            if (k == idx) return (uint16_t)m;
+            ++k;
+        }
+    return 0;
+}
+
+static float half_bits_to_float(uint16_t h) {
+    uint32_t sign = (uint32_t)(h & 0x8000u) << 16;
+    uint32_t exp = (h >> 10) & 0x1Fu;
+    uint32_t man = h & 0x3FFu;
+    uint32_t bits;
+    if (exp == 0) {
+        if (man == 0) {
+            bits = sign;
+        } else {  // subnormal: normalise
+            int e = -1;
+            do { man <<= 1; ++e; } while (!(man & 0x400u));
+            bits = sign | ((uint32_t)(127 - 15 - e) << 23) | ((man & 0x3FFu) << 13);
+        }
+    } else if (exp == 31) {
+        bits = sign | 0x7F800000u | (man << 13);
+    } else {
+        bits = sign | ((exp + 127 - 15) << 23) | (man << 13);
+    }
+    float f;
+    std::memcpy(&f, &bits, 4);
+    return f;
+}
+
+PackConfig choose_pack_config(int c_in, int c_out, xgen_dtype dtype, int stride) {
+    (void)stride;
+    PackConfig c;
+    // The integer variant keeps two rows of sums per filter (an exact fp32
+    // partial sum and the int32 total), so it groups half as many filters.
+    c.filters_per_group = dtype == XGEN_I8_I32 ? 8 : 16;
+    int groups = (c_out + c.filters_per_group - 1) / c.filters_per_group;
+    c.groups_per_block = std::min(groups, 8);
+    c.channels_per_chunk = c_in <= 4 ? 4 : 8;
+    return c;
+}
+
+xgen_status pack_host(const xgen_patconv_desc &d, const void *dense_w, const int16_t *pid,
+                      const PackConfig &cfg, PackedHost &out) {
+    if (!dense_w || !pid || !d.pattern_masks) return XGEN_ERR_INVALID_ARG;
+    if (d.c_in < 1 || d.c_out < 1) return XGEN_ERR_INVALID_ARG;
+    if (d.pad != 1 || (d.stride != 1 && d.stride != 2)) return XGEN_ERR_UNSUPPORTED;
+    if (d.dtype != XGEN_F32 && d.dtype != XGEN_F16_F32ACC && d.dtype != XGEN_I8_I32)
+        return XGEN_ERR_UNSUPPORTED;
+    if (d.num_patterns < 1 || d.num_patterns > kNumAllMasks) return XGEN_ERR_BAD_PATTERN;
+    if ((int64_t)d.c_in * d.c_out > (int64_t)1 << 28) return XGEN_ERR_SHAPE;
+
+    const int P = d.num_patterns, cin = d.c_in, cout = d.c_out;
+    // --- a1: validate the library and the ids ---------------------------------
+    std::vector<int> lib_index(P, -1);  // position in the built-in library, if any
+    for (int p = 0; p < P; ++p) {
+        unsigned m = d.pattern_masks[p];
+        if (m >= 512u || popcount9(m) != 4) return XGEN_ERR_BAD_PATTERN;
+        for (int q = 0; q < kNumLibraryMasks; ++q)
+            if (kLibraryMasks[q] == m) lib_index[p] = q;
+    }
+    int max_lib = -1;
+    bool all_in_lib = true;
+    int64_t k_surv = 0;
+    for (int64_t k = 0; k < (int64_t)cin * cout; ++k) {
+        int p = pid[k];
+        if (p < -1 || p >= P) return XGEN_ERR_BAD_PATTERN;
+        if (p < 0) continue;
+        if (lib_index[p] < 0) all_in_lib = false;
+        max_lib = std::max(max_lib, lib_index[p]);
+        ++k_surv;
+    }
+    const int np = !all_in_lib ? kNumAllMasks : (max_lib < 4 ? 4 : (max_lib < 8 ? 8 : 12));
+    // caller pattern id -> index in the compiled table
+    std::vector<int> to_compiled(P, 0);
+    out = PackedHost();
+    out.masks.resize(np);
+    for (int q = 0; q < np; ++q) out.masks[q] = compiled_mask(np, q);
+    for (int p = 0; p < P; ++p) {
+        if (np <= kNumLibraryMasks) {
+            to_compiled[p] = lib_index[p] >= 0 && lib_index[p] < np ? lib_index[p] : 0;
+        } else {
+            for (int q = 0; q < np; ++q)
+                if (out.masks[q] == d.pattern_masks[p]) to_compiled[p] = q;
+        }
+    }
+
+    const int J = cfg.filters_per_group, cc = cfg.channels_per_chunk;
+    const int wpc = cfg.groups_per_block;
+    if (J < 1 || wpc < 1 || cc < 1 || (cc & (cc - 1))) return XGEN_ERR_INVALID_ARG;
+    const int ocb = J * wpc;  // output channels per thread block (contiguous originals)
+    const int n_blocks = (cout + ocb - 1) / ocb;
+    const int n_groups = n_blocks * wpc;
+    const int n_chunks = (cin + cc - 1) / cc;
+
+    out.c_in = cin; out.c_out = cout; out.stride = d.stride; out.dtype = d.dtype;
+    out.J = J; out.wpc = wpc; out.cc = cc; out.np = np;
+    out.n_blocks = n_blocks; out.n_chunks = n_chunks;
+    out.slot_oc.assign((size_t)n_groups * J, -1);
+
+    // --- a2: filter reorder.  Inside each block of `ocb` contiguous output
+    // channels, sort filters by (surviving kernels desc, pattern histogram,
+    // index) so that similar filters are neighbours, then deal them to the
+    // block's groups in serpentine order: the groups (= warps that meet at a
+    // barrier once per channel chunk) get near-equal kernel counts.
+    std::vector<int> cnt(cout, 0);
+    std::vector<std::vector<int>> hist(cout, std::vector<int>(np, 0));
+    for (int oc = 0; oc < cout; ++oc)
+        for (int ic = 0; ic < cin; ++ic) {
+            int p = pid[(size_t)oc * cin + ic];
+            if (p >= 0) { ++cnt[oc]; ++hist[oc][to_compiled[p]]; }
+        }
+    std::vector<int64_t> group_kernels(n_groups, 0);
+    for (int b = 0; b < n_blocks; ++b) {
+        int lo = b * ocb, hi = std::min(cout, lo + ocb);
+        std::vector<int> order(hi - lo);
+        std::iota(order.begin(), order.end(), lo);
+        std::sort(order.begin(), order.end(), [&](int a, int c) {
+            if (cnt[a] != cnt[c]) return cnt[a] > cnt[c];
+            if (hist[a] != hist[c]) return hist[a] > hist[c];
+            return a < c;
+        });
+        std::vector<int> fill(wpc, 0);
+        for (size_t i = 0; i < order.size(); ++i) {
+            int round = (int)(i / wpc), pos = (int)(i % wpc);
+            int g = (round & 1) ? (wpc - 1 - pos) : pos;
+            out.slot_oc[((size_t)(b * wpc + g)) * J + fill[g]] = order[i];
+            group_kernels[b * wpc + g] += cnt[order[i]];
+            ++fill[g];
+        }
+    }
+
+    // --- a3: kernel reorder + compact store.  Per group and channel: one LOAD,
+    // then the group's surviving kernels of that channel ordered by (pattern,
+    // slot) so equal patterns (equal code) run back to back.
+    out.seg_off.assign((size_t)n_blocks * n_chunks * (wpc + 1), 0);
+    out.slots.reserve(((size_t)k_surv + (size_t)n_groups * (cin + n_chunks)) * kSlotWords + 64);
+    int64_t n_loads = 0;
+    struct Ent { int p, j; };
+    std::vector<Ent> ents;
+    auto push_slot = [&](uint32_t op, uint32_t operand, const uint32_t *w4) {
+        uint32_t s[kSlotWords] = {op, operand, 0, 0, 0, 0, 0, 0};
+        if (w4) for (int i = 0; i < 4; ++i) s[4 + i] = w4[i];
+        out.slots.insert(out.slots.end(), s, s + kSlotWords);
+    };
+    for (int b = 0; b < n_blocks; ++b) {
+        for (int c = 0; c < n_chunks; ++c) {
+            int32_t *so = &out.seg_off[((size_t)b * n_chunks + c) * (wpc + 1)];
+            for (int g = 0; g < wpc; ++g) {
+                so[g] = (int32_t)(out.slots.size() / kSlotWords);
+                const int32_t *soc = &out.slot_oc[((size_t)(b * wpc + g)) * J];
+                for (int icl = 0; icl < cc; ++icl) {
+                    int ic = c * cc + icl;
+                    if (ic >= cin) break;
+                    ents.clear();
+                    for (int j = 0; j < J; ++j) {
+                        if (soc[j] < 0) continue;
+                        int p = pid[(size_t)soc[j] * cin + ic];
+                        if (p >= 0) ents.push_back({to_compiled[p], j});
+                    }
+                    if (ents.empty()) continue;  // group not connected to this channel
+                    std::sort(ents.begin(), ents.end(), [](const Ent &a, const Ent &e) {
+                        return a.p != e.p ? a.p < e.p : a.j < e.j;
+                    });
+                    push_slot((uint32_t)np, (uint32_t)icl, nullptr);
+                    ++n_loads;
+                    for (const Ent &e : ents) {
+                        size_t base = ((size_t)soc[e.j] * cin + ic) * 9;
+                        unsigned m = out.masks[e.p];
+                        uint32_t w4[4];
+                        int k = 0;
+                        for (int t = 0; t < 9; ++t) {
+                            if (!((m >> t) & 1)) continue;
+                            float f;
+                            if (d.dtype == XGEN_F32)
+                                f = ((const float *)dense_w)[base + t];
+                            else if (d.dtype == XGEN_F16_F32ACC)
+                                f = half_bits_to_float(((const uint16_t *)dense_w)[base + t]);
+                            else
+                                f = (float)((const int8_t *)dense_w)[base + t];
+                            std::memcpy(&w4[k++], &f, 4);
+                        }
+                        push_slot((uint32_t)e.p, (uint32_t)(e.j * kPixPerThread), w4);
+                    }
+                }
+                push_slot((uint32_t)np + 1, 0, nullptr);
+            }
+            so[wpc] = (int32_t)(out.slots.size() / kSlotWords);
+            out.max_seg_slots = std::max(out.max_seg_slots, so[wpc] - so[0]);
+            if (out.slots.size() / kSlotWords > (size_t)0x03FFFFFF) return XGEN_ERR_SHAPE;
+        }
+    }
+    const int64_t n_slots = (int64_t)(out.slots.size() / kSlotWords);
+
+    xgen_patconv_stats &s = out.stats;
+    s.kernels_total = (int64_t)cin * cout;
+    s.kernels_surviving = k_surv;
+    s.macs_per_pixel = 4 * k_surv;
+    const int wbytes = d.dtype == XGEN_F32 ? 4 : (d.dtype == XGEN_F16_F32ACC ? 2 : 1);
+    s.weight_bytes = 4 * k_surv * wbytes;
+    s.index_bytes = n_slots * 2 + (int64_t)out.seg_off.size() * 4 + (int64_t)out.slot_oc.size() * 4;
+    s.csr_index_bytes = 4 * k_surv * 4 + (int64_t)(cout + 1) * 4;
+    s.stream_bytes = n_slots * kSlotWords * 4;
+    s.filters_per_group = J; s.groups_per_block = wpc; s.n_blocks = n_blocks;
+    s.channels_per_chunk = cc; s.n_chunks = n_chunks; s.patterns_compiled = np;
+    s.max_segment_slots = out.max_seg_slots;
+    s.load_commands = n_loads;
+    int64_t mx = 0, sum = 0;
+    for (int64_t v : group_kernels) { mx = std::max(mx, v); sum += v; }
+    s.group_imbalance = sum > 0 ? (double)mx * n_groups / (double)sum : 1.0;
+    return XGEN_OK;
+}
+
+}  // namespace patconv

@@ -1,0 +1,660 @@
+// libpatconv: CUDA kernels (sm_100a) and the C ABI.
+//
+// One thread block = one tile of output pixels x one block of contiguous output
+// channels.  Each warp owns a filter group (J filters); each lane owns a 2x4
+// block of output pixels (up to LN images side by side for small images).
+// Per chunk of input channels the block stages (cp.async) the input tile with
+// its halo into channel planes in shared memory -- the NHWC -> plane transpose
+// happens in that copy -- together with the block's slice of the command
+// stream.  Each warp then interprets its commands (core_gen.inc): LOAD brings
+// the thread's activation patch of one channel into registers once, and every
+// surviving kernel of the group on that channel reuses it (the paper's load
+// redundancy elimination, Sec. 2.3); the running sums live in tensor memory,
+// addressed by filter slot.  The epilogue adds bias, applies ReLU, converts and
+// writes NHWC rows through a shared-memory transpose so stores are 16 bytes
+// wide and contiguous per pixel (operator fusion, Sec. 2.2).
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "core_gen.inc"
+#include "patconv_internal.h"
+
+namespace patconv {
+
+constexpr int kSmemPerSM = 233472;     // 228 KB
+constexpr int kSmemMaxDynamic = 232448;  // 227 KB per block
+constexpr int kMaxWarps = 8;
+constexpr int kEpiPix = 2;             // pixels per thread handled in one epilogue pass
+
+struct KParams {
+    const void *x; void *y; const void *bias;
+    const uint32_t *slots; const int32_t *seg_off; const int32_t *slot_oc;
+    int n, h, w, ho, wo, c_in, c_out;
+    int relu;
+    int J, wpc, cc, n_chunks;
+    int lx_log, ly_log, ln_log;          // lanes along x, y and images: 2^.. each, product 32
+    int tiles_x, tiles_y;
+    int tin_w, tin_h;                    // staged tile extents, input pixels
+    int pitch, img_stride, plane_stride; // words
+    int raw_planes;                      // planes of one staged chunk (cc / channels per word)
+    int act_stage_words, cmd_stage_words, stage_words;
+    int n_stages;
+    int exp_off_words;                   // offset of the expanded tile (f16 / i8) in shared memory
+    int tmem_cols, cols_per_warp;
+    int flush_chunks;                    // i8: chunks between folds of the fp32 partial sums
+    int vec_in;                          // c_in is a multiple of the channels per staged word
+    int vec_out;                         // c_out allows 4-channel vector stores
+    int opitch;                          // words per pixel row of the epilogue tile
+};
+
+// ---- small PTX wrappers -----------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src, int src_bytes) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t ta, uint32_t (&r)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(ta) : "memory");
+}
+__device__ __forceinline__ void tmem_ld2(uint32_t ta, uint32_t (&r)[2]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0,%1}, [%2];"
+                 : "=r"(r[0]), "=r"(r[1]) : "r"(ta) : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t ta, const uint32_t (&r)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"r"(ta), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+template <int STRIDE, int NP>
+__device__ __forceinline__ void run_commands(uint32_t &sp, uint32_t tbase, uint32_t plane_bytes,
+                                             uint32_t pitch_bytes, uint32_t tmem_base) {
+    if (STRIDE == 1) {
+        if (NP == 4) PATCONV_CORE_S1_NP4(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        else if (NP == 8) PATCONV_CORE_S1_NP8(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        else if (NP == 12) PATCONV_CORE_S1_NP12(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        else PATCONV_CORE_S1_NP126(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+    } else {
+        if (NP == 4) PATCONV_CORE_S2_NP4(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        else if (NP == 8) PATCONV_CORE_S2_NP8(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        else if (NP == 12) PATCONV_CORE_S2_NP12(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        else PATCONV_CORE_S2_NP126(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+    }
+}
+
+// Channels carried by one staged 32-bit word, and element sizes.
+template <int DT> struct DTraits;
+template <> struct DTraits<XGEN_F32> { static constexpr int E = 1, xbytes = 4, ybytes = 4; };
+template <> struct DTraits<XGEN_F16_F32ACC> { static constexpr int E = 2, xbytes = 2, ybytes = 2; };
+template <> struct DTraits<XGEN_I8_I32> { static constexpr int E = 4, xbytes = 1, ybytes = 4; };
+
+// ---- the kernel -----------------------------------------------------------------
+template <int DT, int STRIDE, int NP>
+__global__ void __launch_bounds__(kMaxWarps * 32)
+patconv_kernel(const KParams P) {
+    extern __shared__ __align__(16) uint32_t smem[];
+    __shared__ uint32_t tmem_base_s;
+    constexpr int E = DTraits<DT>::E;
+    constexpr int XB = DTraits<DT>::xbytes;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nthreads = blockDim.x;
+    const int b = blockIdx.y;
+    int tile = blockIdx.x;
+    const int tx = tile % P.tiles_x; tile /= P.tiles_x;
+    const int ty = tile % P.tiles_y;
+    const int tn = tile / P.tiles_y;
+    const int LX = 1 << P.lx_log, LY = 1 << P.ly_log;
+    const int l_x = lane & (LX - 1), l_y = (lane >> P.lx_log) & (LY - 1), l_n = lane >> (P.lx_log + P.ly_log);
+    const int TW = 2 * LX, TH = 4 * LY;
+    const int n0 = tn << P.ln_log;                   // first image of the tile
+    const int gy0 = ty * TH * STRIDE - 1, gx0 = tx * TW * STRIDE - 1;   // input coords of tile (0,0)
+
+    // --- tensor memory for the running sums --------------------------------------
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)P.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+
+    // --- staging -------------------------------------------------------------------
+    const int RP = P.raw_planes;                      // power of two
+    const int rp = tid & (RP - 1);
+    const int pix_step = nthreads / RP;
+    const int npix = (P.tin_w * P.tin_h) << P.ln_log;
+    const int32_t *seg = P.seg_off + (size_t)b * P.n_chunks * (P.wpc + 1);
+    const uint32_t smem_base = smem_u32(smem);
+
+    const int q0 = tid / RP;
+    const int col0 = q0 % P.tin_w, row0 = (q0 / P.tin_w) % P.tin_h, im0 = q0 / (P.tin_w * P.tin_h);
+    const int dcol = pix_step % P.tin_w, drow = pix_step / P.tin_w;
+    auto stage_load = [&](int c) {
+        if (c < P.n_chunks) {
+            const int stage = c % P.n_stages;
+            const uint32_t act = smem_base + (uint32_t)(stage * P.stage_words) * 4u;
+            // activations: one 32-bit word = E consecutive channels of one pixel
+            int col = col0, row = row0, im = im0;
+            const int ic = c * P.cc + rp * E;
+            for (int q = q0; q < npix; q += pix_step) {
+                const int gy = gy0 + row, gx = gx0 + col, gn = n0 + im;
+                const bool ok = gn < P.n && gy >= 0 && gy < P.h && gx >= 0 && gx < P.w && ic < P.c_in;
+                const uint32_t dst = act + (uint32_t)(rp * P.plane_stride + im * P.img_stride + row * P.pitch + col) * 4u;
+                const size_t gi = ok ? (((size_t)gn * P.h + gy) * P.w + gx) * P.c_in + ic : 0;
+                const char *src = (const char *)P.x + gi * XB;
+                if (E == 1 || P.vec_in) {
+                    cp_async4(dst, src, ok ? 4 : 0);
+                } else {
+                    // channel count not a multiple of E: assemble the word element by element
+                    uint32_t word = 0;
+                    if (ok) {
+                        for (int k = 0; k < E; ++k) {
+                            if (ic + k < P.c_in) {
+                                if (XB == 2) word |= (uint32_t)((const uint16_t *)src)[k] << (16 * k);
+                                else word |= (uint32_t)((const uint8_t *)src)[k] << (8 * k);
+                            }
+                        }
+                    }
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst), "r"(word) : "memory");
+                }
+                col += dcol; row += drow;
+                if (col >= P.tin_w) { col -= P.tin_w; ++row; }
+                while (row >= P.tin_h) { row -= P.tin_h; ++im; }
+            }
+            // this block's commands for the chunk: one contiguous segment
+            const int s0 = seg[c * (P.wpc + 1)], s1 = seg[c * (P.wpc + 1) + P.wpc];
+            const uint32_t cmd = act + (uint32_t)P.act_stage_words * 4u;
+            const uint4 *gsrc = reinterpret_cast<const uint4 *>(P.slots + (size_t)s0 * kSlotWords);
+            const int n16 = (s1 - s0) * 2;
+            for (int i = tid; i < n16; i += nthreads) cp_async16(cmd + (uint32_t)i * 16u, gsrc + i);
+        }
+        cp_async_commit();
+    };
+
+    for (int s = 0; s < P.n_stages - 1; ++s) stage_load(s);
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_cta = tmem_base_s;
+    const uint32_t tmem_warp = tmem_cta + (((uint32_t)(warp & 3) * 32u) << 16) + (uint32_t)((warp >> 2) * P.cols_per_warp);
+    {
+        const uint32_t z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        for (int c = 0; c < P.cols_per_warp; c += 8) tmem_st8(tmem_warp + c, z);
+        tmem_wait_st();
+    }
+    const uint32_t tmem_int = tmem_warp + (uint32_t)(P.J * kPixPerThread);   // i8: int32 totals
+
+    // i8: fold the exact fp32 partial sums into the int32 totals and clear them
+    auto fold_partial_sums = [&]() {
+        for (int j = 0; j < P.J; ++j) {
+            uint32_t f[8], q[8];
+            tmem_ld8(tmem_warp + j * 8, f);
+            tmem_ld8(tmem_int + j * 8, q);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { q[i] = (uint32_t)((int)q[i] + __float2int_rn(__uint_as_float(f[i]))); f[i] = 0u; }
+            tmem_st8(tmem_int + j * 8, q);
+            tmem_st8(tmem_warp + j * 8, f);
+        }
+        tmem_wait_st();
+    };
+
+    const uint32_t thr_off = (uint32_t)(l_n * P.img_stride + l_y * 4 * STRIDE * P.pitch + l_x * 2 * STRIDE) * 4u;
+    const uint32_t plane_bytes = (uint32_t)P.plane_stride * 4u, pitch_bytes = (uint32_t)P.pitch * 4u;
+
+    // --- main loop over channel chunks --------------------------------------------
+    for (int c = 0; c < P.n_chunks; ++c) {
+        const int stage = c % P.n_stages;
+        if (P.n_stages == 2) cp_async_wait<0>(); else cp_async_wait<1>();
+        __syncthreads();                       // chunk c has landed; everyone is done with chunk c-1
+        stage_load(c + P.n_stages - 1);
+        const uint32_t act = smem_base + (uint32_t)(stage * P.stage_words) * 4u;
+        uint32_t tile_base = act;
+        if (DT != XGEN_F32) {
+            // widen the staged words to fp32 planes (exact for fp16 and for uint8)
+            const uint32_t *raw = smem + stage * P.stage_words;
+            float *ex = reinterpret_cast<float *>(smem + P.exp_off_words);
+            const int nraw = RP * P.plane_stride;
+            for (int i = tid; i < nraw; i += nthreads) {
+                const int r = i / P.plane_stride, o = i - r * P.plane_stride;
+                const uint32_t wd = raw[i];
+                if (DT == XGEN_F16_F32ACC) {
+                    const __half2 h2 = *reinterpret_cast<const __half2 *>(&wd);
+                    ex[(2 * r) * P.plane_stride + o] = __low2float(h2);
+                    ex[(2 * r + 1) * P.plane_stride + o] = __high2float(h2);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) ex[(4 * r + k) * P.plane_stride + o] = (float)((wd >> (8 * k)) & 0xFFu);
+                }
+            }
+            __syncthreads();
+            tile_base = smem_base + (uint32_t)P.exp_off_words * 4u;
+        }
+        const int s0 = seg[c * (P.wpc + 1)], sg = seg[c * (P.wpc + 1) + warp];
+        uint32_t sp = act + (uint32_t)P.act_stage_words * 4u + (uint32_t)(sg - s0) * 32u;
+        run_commands<STRIDE, NP>(sp, tile_base + thr_off, plane_bytes, pitch_bytes, tmem_warp);
+        if (DT == XGEN_I8_I32 && ((c + 1) % P.flush_chunks == 0)) fold_partial_sums();
+    }
+    cp_async_wait<0>();
+    if (DT == XGEN_I8_I32) fold_partial_sums();
+    __syncthreads();                           // staging memory is free: reuse it for the epilogue
+
+    // --- epilogue: bias + ReLU + convert, NHWC rows through shared memory ----------
+    const int ocb = P.J * P.wpc;
+    const int oc_lo = b * ocb;
+    const int nvalid = min(ocb, P.c_out - oc_lo);
+    const int32_t *soc = P.slot_oc + ((size_t)(b * P.wpc + warp)) * P.J;
+    const uint32_t tmem_res = DT == XGEN_I8_I32 ? tmem_int : tmem_warp;
+    for (int t0 = 0; t0 < kPixPerThread; t0 += kEpiPix) {
+        for (int j = 0; j < P.J; ++j) {
+            const int oc = soc[j];
+            uint32_t v[2];
+            tmem_ld2(tmem_res + j * 8 + t0, v);
+            tmem_wait_ld();
+            if (oc >= 0) {
+                smem[(0 * 32 + lane) * P.opitch + (oc - oc_lo)] = v[0];
+                smem[(1 * 32 + lane) * P.opitch + (oc - oc_lo)] = v[1];
+            }
+        }
+        __syncthreads();
+        // cooperative store: kEpiPix*32 pixels x nvalid channels
+        const int segs = P.vec_out ? (nvalid >> 2) : nvalid;
+        const int total = kEpiPix * 32 * segs;
+        for (int i = tid; i < total; i += nthreads) {
+            const int pl = i / segs, sgm = i - pl * segs;     // pl = tt*32 + lane'
+            const int tt = pl >> 5, ln2 = pl & 31;
+            const int t = t0 + tt;
+            const int p_x = ln2 & (LX - 1), p_y = (ln2 >> P.lx_log) & (LY - 1), p_n = ln2 >> (P.lx_log + P.ly_log);
+            const int ox = tx * TW + p_x * 2 + (t & 1), oy = ty * TH + p_y * 4 + (t >> 1), on = n0 + p_n;
+            if (on >= P.n || oy >= P.ho || ox >= P.wo) continue;
+            const size_t pix = ((size_t)on * P.ho + oy) * P.wo + ox;
+            if (P.vec_out) {
+                const int ocl = sgm * 4;
+                const uint4 raw = *reinterpret_cast<const uint4 *>(&smem[pl * P.opitch + ocl]);
+                const size_t o = pix * P.c_out + oc_lo + ocl;
+                if (DT == XGEN_I8_I32) {
+                    int4 r = make_int4((int)raw.x, (int)raw.y, (int)raw.z, (int)raw.w);
+                    if (P.bias) {
+                        const int4 bb = *reinterpret_cast<const int4 *>((const int *)P.bias + oc_lo + ocl);
+                        r.x += bb.x; r.y += bb.y; r.z += bb.z; r.w += bb.w;
+                    }
+                    if (P.relu) { r.x = max(r.x, 0); r.y = max(r.y, 0); r.z = max(r.z, 0); r.w = max(r.w, 0); }
+                    *reinterpret_cast<int4 *>((int *)P.y + o) = r;
+                } else {
+                    float4 r = make_float4(__uint_as_float(raw.x), __uint_as_float(raw.y), __uint_as_float(raw.z), __uint_as_float(raw.w));
+                    if (P.bias) {
+                        const float4 bb = *reinterpret_cast<const float4 *>((const float *)P.bias + oc_lo + ocl);
+                        r.x += bb.x; r.y += bb.y; r.z += bb.z; r.w += bb.w;
+                    }
+                    if (P.relu) { r.x = fmaxf(r.x, 0.f); r.y = fmaxf(r.y, 0.f); r.z = fmaxf(r.z, 0.f); r.w = fmaxf(r.w, 0.f); }
+                    if (DT == XGEN_F32) {
+                        *reinterpret_cast<float4 *>((float *)P.y + o) = r;
+                    } else {
+                        __half2 lo = __floats2half2_rn(r.x, r.y), hi = __floats2half2_rn(r.z, r.w);
+                        uint2 pk;
+                        pk.x = *reinterpret_cast<uint32_t *>(&lo);
+                        pk.y = *reinterpret_cast<uint32_t *>(&hi);
+                        *reinterpret_cast<uint2 *>((__half *)P.y + o) = pk;
+                    }
+                }
+            } else {
+                const uint32_t raw = smem[pl * P.opitch + sgm];
+                const size_t o = pix * P.c_out + oc_lo + sgm;
+                if (DT == XGEN_I8_I32) {
+                    int r = (int)raw + (P.bias ? ((const int *)P.bias)[oc_lo + sgm] : 0);
+                    if (P.relu) r = max(r, 0);
+                    ((int *)P.y)[o] = r;
+                } else {
+                    float r = __uint_as_float(raw) + (P.bias ? ((const float *)P.bias)[oc_lo + sgm] : 0.f);
+                    if (P.relu) r = fmaxf(r, 0.f);
+                    if (DT == XGEN_F32) ((float *)P.y)[o] = r;
+                    else ((__half *)P.y)[o] = __float2half_rn(r);
+                }
+            }
+        }
+        __syncthreads();
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_cta), "r"((uint32_t)P.tmem_cols) : "memory");
+    }
+}
+
+// ---- host side ----------------------------------------------------------------------
+static std::atomic<int64_t> g_launches{0};
+
+struct Geometry {
+    int lx_log, ly_log, ln_log, tiles_x, tiles_y, tiles_n;
+    int tin_w, tin_h, pitch, img_stride, plane_stride;
+};
+
+// Cost (shared-memory wavefronts) of one patch-row load for a candidate pitch.
+static int row_load_conflicts(int stride, int lx_log, int ly_log, int pitch, int img_stride) {
+    const int LX = 1 << lx_log, LY = 1 << ly_log;
+    auto addr = [&](int lane) {
+        int x = lane & (LX - 1), y = (lane >> lx_log) & (LY - 1), n = lane >> (lx_log + ly_log);
+        return n * img_stride + y * 4 * stride * pitch + x * 2 * stride;   // words
+    };
+    int worst = 0;
+    const int lanes_per_phase = stride == 1 ? 16 : 8;     // 64-bit / 128-bit accesses
+    const int words = stride == 1 ? 2 : 4;
+    for (int ph = 0; ph < 32 / lanes_per_phase; ++ph) {
+        int cnt[32] = {0};
+        for (int l = 0; l < lanes_per_phase; ++l) {
+            int a = addr(ph * lanes_per_phase + l);
+            for (int k = 0; k < words; ++k) cnt[(a + k) & 31]++;
+        }
+        for (int i = 0; i < 32; ++i) worst = worst > cnt[i] ? worst : cnt[i];
+    }
+    return worst;
+}
+
+static Geometry choose_geometry(int n, int ho, int wo, int stride) {
+    Geometry best{};
+    double best_eff = -1.0;
+    for (int lx_log = 5; lx_log >= 0; --lx_log)
+        for (int ly_log = 5 - lx_log; ly_log >= 0; --ly_log) {
+            const int ln_log = 5 - lx_log - ly_log;
+            const int TW = 2 << lx_log, TH = 4 << ly_log, LN = 1 << ln_log;
+            if (LN > 1 && (TW < wo || TH < ho)) continue;   // several images per tile only when one image fits
+            const long tiles = (long)((wo + TW - 1) / TW) * ((ho + TH - 1) / TH) * ((n + LN - 1) / LN);
+            const double eff = (double)n * ho * wo / ((double)tiles * 256.0);
+            if (eff > best_eff + 1e-9) {
+                best_eff = eff;
+                best.lx_log = lx_log; best.ly_log = ly_log; best.ln_log = ln_log;
+            }
+        }
+    const int TW = 2 << best.lx_log, TH = 4 << best.ly_log, LN = 1 << best.ln_log;
+    best.tiles_x = (wo + TW - 1) / TW; best.tiles_y = (ho + TH - 1) / TH; best.tiles_n = (n + LN - 1) / LN;
+    best.tin_w = stride == 1 ? TW + 2 : 2 * TW + 1;
+    best.tin_h = stride == 1 ? TH + 2 : 2 * TH + 1;
+    const int align = stride == 1 ? 2 : 4;                // 8- or 16-byte aligned patch rows
+    int p0 = (best.tin_w + align - 1) / align * align, best_p = p0, best_c = 1 << 30;
+    for (int p = p0; p < p0 + 34; p += align) {
+        int c = row_load_conflicts(stride, best.lx_log, best.ly_log, p, best.tin_h * p);
+        if (c < best_c) { best_c = c; best_p = p; }
+    }
+    best.pitch = best_p;
+    best.img_stride = best.tin_h * best.pitch;
+    int ps = LN * best.img_stride;
+    while ((ps & 31) != 4) ++ps;                          // planes 4 banks apart: conflict-free staging writes
+    best.plane_stride = ps;
+    return best;
+}
+
+}  // namespace patconv
+
+using namespace patconv;
+
+struct xgen_patconv_packed {
+    PackedHost host;
+    int device = -1;
+    uint32_t *d_slots = nullptr;
+    int32_t *d_seg_off = nullptr;
+    int32_t *d_slot_oc = nullptr;
+};
+
+template <int DT, int STRIDE>
+static cudaError_t launch_np(int np, dim3 grid, dim3 block, size_t smem, cudaStream_t st, const KParams &kp) {
+    auto go = [&](auto kern) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMaxDynamic);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, block, smem, st>>>(kp);
+        return cudaGetLastError();
+    };
+    switch (np) {
+        case 4: return go(patconv_kernel<DT, STRIDE, 4>);
+        case 8: return go(patconv_kernel<DT, STRIDE, 8>);
+        case 12: return go(patconv_kernel<DT, STRIDE, 12>);
+        default: return go(patconv_kernel<DT, STRIDE, 126>);
+    }
+}
+
+static int next_pow2(int v) { int p = 32; while (p < v) p <<= 1; return p; }
+
+extern "C" {
+
+const char *xgen_strerror(xgen_status s) {
+    switch (s) {
+        case XGEN_OK: return "ok";
+        case XGEN_ERR_INVALID_ARG: return "invalid argument";
+        case XGEN_ERR_BAD_PATTERN: return "bad pattern mask or pattern id";
+        case XGEN_ERR_SHAPE: return "shape out of range";
+        case XGEN_ERR_UNSUPPORTED: return "unsupported configuration";
+        case XGEN_ERR_ALLOC: return "allocation failed";
+        case XGEN_ERR_CUDA: return "CUDA error";
+        case XGEN_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+int64_t xgen_patconv_launch_count(void) { return g_launches.load(); }
+
+xgen_status xgen_patconv_pack(const xgen_patconv_desc *desc, const void *dense_w_host,
+                              const int16_t *pattern_id_host, int device, xgen_patconv_packed **out) {
+    if (!desc || !out) return XGEN_ERR_INVALID_ARG;
+    *out = nullptr;
+    xgen_patconv_packed *h = new (std::nothrow) xgen_patconv_packed();
+    if (!h) return XGEN_ERR_ALLOC;
+    xgen_status st;
+    try {
+        PackConfig cfg = choose_pack_config(desc->c_in, desc->c_out, desc->dtype, desc->stride);
+        if (const char *e = getenv("XGEN_PATCONV_J")) { int v = atoi(e); if (v == 4 || v == 8 || v == 16 || v == 32) {
+            cfg.filters_per_group = v;
+            int groups = (desc->c_out + v - 1) / v; cfg.groups_per_block = groups < kMaxWarps ? groups : kMaxWarps; } }
+        if (const char *e = getenv("XGEN_PATCONV_CC")) { int v = atoi(e); if (v == 2 || v == 4 || v == 8 || v == 16) cfg.channels_per_chunk = v; }
+        if (desc->dtype == XGEN_I8_I32 && cfg.channels_per_chunk < 4) cfg.channels_per_chunk = 4;
+        st = pack_host(*desc, dense_w_host, pattern_id_host, cfg, h->host);
+    } catch (const std::bad_alloc &) {
+        st = XGEN_ERR_ALLOC;
+    }
+    if (st != XGEN_OK) { delete h; return st; }
+    if (device >= 0) {
+        int prev = 0;
+        if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(device) != cudaSuccess) { delete h; return XGEN_ERR_CUDA; }
+        const PackedHost &p = h->host;
+        // two spare slots: harmless over-read room for 16-byte copies
+        size_t sb = (p.slots.size() + 2 * kSlotWords) * 4, gb = p.seg_off.size() * 4, ob = p.slot_oc.size() * 4;
+        cudaError_t e = cudaMalloc(&h->d_slots, sb);
+        if (e == cudaSuccess) e = cudaMalloc(&h->d_seg_off, gb);
+        if (e == cudaSuccess) e = cudaMalloc(&h->d_slot_oc, ob);
+        if (e == cudaSuccess) e = cudaMemset(h->d_slots, 0, sb);
+        if (e == cudaSuccess) e = cudaMemcpy(h->d_slots, p.slots.data(), p.slots.size() * 4, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(h->d_seg_off, p.seg_off.data(), gb, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(h->d_slot_oc, p.slot_oc.data(), ob, cudaMemcpyHostToDevice);
+        cudaSetDevice(prev);
+        if (e != cudaSuccess) {
+            xgen_status r = (e == cudaErrorMemoryAllocation) ? XGEN_ERR_ALLOC : XGEN_ERR_CUDA;
+            cudaGetLastError();
+            xgen_patconv_free(h);
+            return r;
+        }
+        h->device = device;
+    }
+    *out = h;
+    return XGEN_OK;
+}
+
+void xgen_patconv_free(xgen_patconv_packed *h) {
+    if (!h) return;
+    if (h->device >= 0) {
+        cudaFree(h->d_slots); cudaFree(h->d_seg_off); cudaFree(h->d_slot_oc);
+    } else {
+        if (h->d_slots) cudaFree(h->d_slots);
+        if (h->d_seg_off) cudaFree(h->d_seg_off);
+        if (h->d_slot_oc) cudaFree(h->d_slot_oc);
+    }
+    delete h;
+}
+
+xgen_status xgen_patconv_out_shape(const xgen_patconv_packed *h, int32_t hh, int32_t ww, int32_t *ho, int32_t *wo) {
+    if (!h || !ho || !wo) return XGEN_ERR_INVALID_ARG;
+    if (hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
+    *ho = (hh + 2 - 3) / h->host.stride + 1;
+    *wo = (ww + 2 - 3) / h->host.stride + 1;
+    return XGEN_OK;
+}
+
+xgen_status xgen_patconv_query(const xgen_patconv_packed *h, xgen_patconv_stats *s) {
+    if (!h || !s) return XGEN_ERR_INVALID_ARG;
+    *s = h->host.stats;
+    return XGEN_OK;
+}
+
+xgen_status xgen_patconv_view(const xgen_patconv_packed *h, xgen_patconv_host_view *v) {
+    if (!h || !v) return XGEN_ERR_INVALID_ARG;
+    v->slots = h->host.slots.data();
+    v->n_slots = (int64_t)(h->host.slots.size() / kSlotWords);
+    v->seg_off = h->host.seg_off.data();
+    v->slot_oc = h->host.slot_oc.data();
+    v->compiled_masks = h->host.masks.data();
+    return XGEN_OK;
+}
+
+xgen_status xgen_patconv_plan(xgen_patconv_packed *h, int32_t n, int32_t hh, int32_t ww) {
+    if (!h) return XGEN_ERR_INVALID_ARG;
+    if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
+    return XGEN_OK;
+}
+
+xgen_status xgen_patconv_last_status(const xgen_patconv_packed *h, void *stream) {
+    if (!h) return XGEN_ERR_INVALID_ARG;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return XGEN_ERR_CUDA;
+    return cudaGetLastError() == cudaSuccess ? XGEN_OK : XGEN_ERR_CUDA;
+}
+
+xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
+                             const void *bias, int32_t relu, void *y, void *stream) {
+    if (!h || !x || !y) return XGEN_ERR_INVALID_ARG;
+    if (((uintptr_t)x & 15) || ((uintptr_t)y & 15) || ((uintptr_t)bias & 15)) return XGEN_ERR_INVALID_ARG;
+    if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
+    const PackedHost &p = h->host;
+    if (h->device < 0) return XGEN_ERR_CUDA;
+    const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
+    if ((int64_t)n * hh * ww * p.c_in > 0x7FFFFFFFLL || (int64_t)n * ho * wo * p.c_out > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
+    {
+        const char *xa = (const char *)x, *ya = (const char *)y;
+        const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
+        const int yb = p.dtype == XGEN_F16_F32ACC ? 2 : 4;
+        const char *xe = xa + (size_t)n * hh * ww * p.c_in * xb, *ye = ya + (size_t)n * ho * wo * p.c_out * yb;
+        if (xa < ye && ya < xe) return XGEN_ERR_INVALID_ARG;   // overlap
+    }
+    Geometry g = choose_geometry(n, ho, wo, p.stride);
+    KParams kp{};
+    kp.x = x; kp.y = y; kp.bias = bias;
+    kp.slots = h->d_slots; kp.seg_off = h->d_seg_off; kp.slot_oc = h->d_slot_oc;
+    kp.n = n; kp.h = hh; kp.w = ww; kp.ho = ho; kp.wo = wo; kp.c_in = p.c_in; kp.c_out = p.c_out;
+    kp.relu = relu ? 1 : 0;
+    kp.J = p.J; kp.wpc = p.wpc; kp.cc = p.cc; kp.n_chunks = p.n_chunks;
+    kp.lx_log = g.lx_log; kp.ly_log = g.ly_log; kp.ln_log = g.ln_log;
+    kp.tiles_x = g.tiles_x; kp.tiles_y = g.tiles_y;
+    kp.tin_w = g.tin_w; kp.tin_h = g.tin_h;
+    kp.pitch = g.pitch; kp.img_stride = g.img_stride; kp.plane_stride = g.plane_stride;
+    const int E = p.dtype == XGEN_F32 ? 1 : (p.dtype == XGEN_F16_F32ACC ? 2 : 4);
+    kp.raw_planes = p.cc / E;
+    kp.act_stage_words = (kp.raw_planes * g.plane_stride + 3) & ~3;
+    kp.cmd_stage_words = p.max_seg_slots * kSlotWords;
+    kp.stage_words = kp.act_stage_words + kp.cmd_stage_words;
+    kp.vec_in = (p.c_in % E) == 0;
+    kp.vec_out = (p.c_out % 4) == 0;
+    const bool is_i8 = p.dtype == XGEN_I8_I32;
+    kp.cols_per_warp = p.J * kPixPerThread * (is_i8 ? 2 : 1);
+    kp.tmem_cols = next_pow2(((p.wpc + 3) / 4) * kp.cols_per_warp);
+    if (kp.tmem_cols > 512) return XGEN_ERR_UNSUPPORTED;
+    kp.flush_chunks = 16777216 / (p.cc * 4 * 32640);
+    if (kp.flush_chunks < 1) return XGEN_ERR_UNSUPPORTED;
+    const int ocb = p.J * p.wpc;
+    kp.opitch = ocb + 4;
+    const int exp_words = p.dtype == XGEN_F32 ? 0 : p.cc * g.plane_stride;
+    const int epi_words = kEpiPix * 32 * kp.opitch;
+    int n_stages = 3;
+    size_t words = 0;
+    for (;; --n_stages) {
+        words = (size_t)n_stages * kp.stage_words + exp_words;
+        if (words * 4 <= (size_t)kSmemMaxDynamic / 2 || n_stages == 2) break;
+    }
+    kp.n_stages = n_stages;
+    kp.exp_off_words = n_stages * kp.stage_words;
+    if (words < (size_t)epi_words) words = epi_words;
+    size_t smem = words * 4;
+    // Never let more blocks share an SM than tensor memory has columns for.
+    const int max_ctas = 512 / kp.tmem_cols;
+    const size_t floor_bytes = (size_t)kSmemPerSM / (max_ctas + 1);
+    if (smem < floor_bytes) smem = floor_bytes;
+    if (smem > (size_t)kSmemMaxDynamic) return XGEN_ERR_UNSUPPORTED;
+
+    int prev = 0;
+    if (cudaGetDevice(&prev) != cudaSuccess) return XGEN_ERR_CUDA;
+    if (prev != h->device && cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
+    dim3 grid((unsigned)(g.tiles_x * g.tiles_y * g.tiles_n), (unsigned)p.n_blocks, 1), block((unsigned)(p.wpc * 32), 1, 1);
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e;
+    if (p.dtype == XGEN_F32)
+        e = p.stride == 1 ? launch_np<XGEN_F32, 1>(p.np, grid, block, smem, st, kp) : launch_np<XGEN_F32, 2>(p.np, grid, block, smem, st, kp);
+    else if (p.dtype == XGEN_F16_F32ACC)
+        e = p.stride == 1 ? launch_np<XGEN_F16_F32ACC, 1>(p.np, grid, block, smem, st, kp) : launch_np<XGEN_F16_F32ACC, 2>(p.np, grid, block, smem, st, kp);
+    else
+        e = p.stride == 1 ? launch_np<XGEN_I8_I32, 1>(p.np, grid, block, smem, st, kp) : launch_np<XGEN_I8_I32, 2>(p.np, grid, block, smem, st, kp);
+    if (prev != h->device) cudaSetDevice(prev);
+    if (e != cudaSuccess) return XGEN_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return XGEN_OK;
+}
+
+xgen_status xgen_patconv_run_host(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
+                                  const void *bias, int32_t relu, void *y) {
+    if (!h || !x || !y) return XGEN_ERR_INVALID_ARG;
+    if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
+    if (h->device < 0) return XGEN_ERR_CUDA;
+    const PackedHost &p = h->host;
+    const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
+    const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
+    const int yb = p.dtype == XGEN_F16_F32ACC ? 2 : 4;
+    const size_t xbytes = (size_t)n * hh * ww * p.c_in * xb, ybytes = (size_t)n * ho * wo * p.c_out * yb;
+    int prev = 0;
+    if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
+    void *dx = nullptr, *dy = nullptr, *db = nullptr;
+    xgen_status rs = XGEN_OK;
+    cudaError_t e = cudaMalloc(&dx, xbytes);
+    if (e == cudaSuccess) e = cudaMalloc(&dy, ybytes);
+    if (e == cudaSuccess && bias) e = cudaMalloc(&db, (size_t)p.c_out * 4);
+    if (e != cudaSuccess) { rs = XGEN_ERR_ALLOC; cudaGetLastError(); }
+    if (rs == XGEN_OK) {
+        e = cudaMemcpyAsync(dx, x, xbytes, cudaMemcpyHostToDevice, 0);
+        if (e == cudaSuccess && bias) e = cudaMemcpyAsync(db, bias, (size_t)p.c_out * 4, cudaMemcpyHostToDevice, 0);
+        if (e != cudaSuccess) rs = XGEN_ERR_CUDA;
+    }
+    if (rs == XGEN_OK) rs = xgen_patconv_run(h, dx, n, hh, ww, db, relu, dy, nullptr);
+    if (rs == XGEN_OK) {
+        e = cudaMemcpyAsync(y, dy, ybytes, cudaMemcpyDeviceToHost, 0);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+        if (e != cudaSuccess) rs = XGEN_ERR_CUDA;
+    }
+    cudaFree(dx); cudaFree(dy); cudaFree(db);
+    cudaSetDevice(prev);
+    return rs;
+}
+
+}  // extern "C"
