@@ -30,7 +30,7 @@
 namespace patconv {
 
 constexpr int kSmemPerSM = 233472;     // 228 KB
-constexpr int kSmemMaxDynamic = 232448;  // 227 KB per block
+constexpr int kSmemMaxDynamic = 232448 - 1024;  // 227 KB per block less static shared memory
 constexpr int kMaxWarps = 8;
 constexpr int kEpiPix = 2;             // pixels per thread handled in one epilogue pass
 
@@ -415,13 +415,20 @@ struct xgen_patconv_packed {
     int32_t *d_slot_oc = nullptr;
 };
 
+// With XGEN_PATCONV_LOG set, failed CUDA calls are named on stderr.
+static cudaError_t log_cuda(cudaError_t e, const char *what) {
+    if (e != cudaSuccess && getenv("XGEN_PATCONV_LOG"))
+        fprintf(stderr, "libpatconv: %s: %s\n", what, cudaGetErrorString(e));
+    return e;
+}
+
 template <int DT, int STRIDE>
 static cudaError_t launch_np(int np, dim3 grid, dim3 block, size_t smem, cudaStream_t st, const KParams &kp) {
     auto go = [&](auto kern) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMaxDynamic);
-        if (e != cudaSuccess) return e;
+        if (e != cudaSuccess) return log_cuda(e, "cudaFuncSetAttribute");
         kern<<<grid, block, smem, st>>>(kp);
-        return cudaGetLastError();
+        return log_cuda(cudaGetLastError(), "kernel launch");
     };
     switch (np) {
         case 4: return go(patconv_kernel<DT, STRIDE, 4>);

@@ -1,0 +1,127 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle,
+element by element on the same seeded inputs."""
+import numpy as np
+import pytest
+
+from paper_2206_10620_b200 import binding, workloads as wl
+from _gpu_util import compare, pack, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+def _layer(dtype, n, ci, co, h, w, stride=1, prune=0.5, lib=8, seed=1, idx=0):
+    xd = {"f32": "upm1", "f16": "relu_normal", "i8": "u01"}[dtype]
+    spec = wl.LayerSpec("t", n, ci, co, h, w, stride, dtype, prune, lib, "he", xd, 0.05, True, idx)
+    return wl.make_layer(spec, seed=seed)
+
+
+def test_config_single_layer():
+    d = wl.make_layer(wl.config_single_layer()[0])
+    pk = pack(d)
+    y = run_gpu(pk, d.x, d.bias, True)
+    compare(d, y)
+    assert binding.launch_count() >= 1
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "i8"])
+@pytest.mark.parametrize("stride", [1, 2])
+@pytest.mark.parametrize("shape", [
+    (2, 5, 7, 9, 11),        # odd everything: scalar stores, ragged channels
+    (3, 20, 40, 37, 19),     # several tiles and a ragged tail in both directions
+    (1, 16, 136, 70, 66),    # two blocks of output channels, the second ragged
+    (5, 24, 16, 7, 7),       # several small images in one tile
+    (2, 64, 32, 14, 14),
+])
+def test_shapes(dtype, stride, shape):
+    n, ci, co, h, w = shape
+    d = _layer(dtype, n, ci, co, h, w, stride, prune=0.5, lib=12, seed=n + ci)
+    pk = pack(d)
+    compare(d, run_gpu(pk, d.x, d.bias, True))
+    compare(d, run_gpu(pk, d.x, None, False), bias=None, relu=False)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "i8"])
+def test_first_layer_three_channels(dtype):
+    d = _layer(dtype, 1, 3, 64, 60, 60, prune=0.0)
+    compare(d, run_gpu(pack(d), d.x, d.bias, True))
+
+
+@pytest.mark.parametrize("prune", [0.0, 0.75, 0.875])
+@pytest.mark.parametrize("lib", [4, 12])
+def test_density_and_library(prune, lib):
+    d = _layer("f16", 2, 64, 64, 28, 28, prune=prune, lib=lib)
+    compare(d, run_gpu(pack(d), d.x, d.bias, True))
+
+
+def test_foreign_masks_universal_table():
+    d = _layer("f32", 1, 16, 32, 12, 12, lib=4)
+    d.masks = np.array([0x00F, 0x1E0, 0x145, 0x0AA], dtype=np.uint16)   # none contains the centre
+    pk = pack(d)
+    assert pk.stats()["patterns_compiled"] == 126
+    compare(d, run_gpu(pk, d.x, d.bias, True))
+
+
+def test_degenerate_layers():
+    d = _layer("f32", 1, 8, 16, 10, 10)
+    d.pid[:] = -1                                    # everything pruned: y = act(bias)
+    y = run_gpu(pack(d), d.x, d.bias, True)
+    assert np.array_equal(y, np.broadcast_to(np.maximum(d.bias, 0), y.shape))
+    d2 = _layer("f32", 1, 8, 16, 10, 10)
+    d2.pid[3, :] = -1                                # one filter with no kernel left
+    y2 = run_gpu(pack(d2), d2.x, d2.bias, False)
+    assert np.all(y2[..., 3] == d2.bias[3])
+    compare(d2, y2, relu=False)
+    d3 = _layer("f32", 1, 4, 8, 1, 1)                # 1x1 image: only the centre tap lands
+    compare(d3, run_gpu(pack(d3), d3.x, d3.bias, True))
+
+
+def test_pruned_weights_are_ignored_and_runs_are_deterministic():
+    d = _layer("f32", 1, 16, 32, 20, 20)
+    y0 = run_gpu(pack(d), d.x, d.bias, True)
+    w2 = d.w.copy()
+    keep = np.zeros((len(d.masks) + 1, 9), bool)
+    for p, m in enumerate(d.masks):
+        keep[p] = [(int(m) >> t) & 1 for t in range(9)]
+    sel = keep[d.pid].reshape(d.pid.shape + (3, 3))
+    w2[~sel] = 777.0
+    d.w = w2
+    pk = pack(d)
+    y1 = run_gpu(pk, d.x, d.bias, True)
+    y2 = run_gpu(pk, d.x, d.bias, True)
+    assert np.array_equal(y0, y1) and np.array_equal(y1, y2)
+
+
+def test_int8_extremes_and_long_reduction():
+    # 512 input channels: the exact-partial-sum fold runs several times
+    ci = 512
+    spec = wl.LayerSpec("t", 1, ci, 16, 6, 6, 1, "i8", 0.0, 8, "he", "u01", 0.05, True, 0)
+    d = wl.make_layer(spec)
+    d.x[:] = 255
+    for wv in (127, -128):
+        d.w[:] = wv
+        compare(d, run_gpu(pack(d), d.x, d.bias, False), relu=False)
+    d = wl.make_layer(spec)
+    compare(d, run_gpu(pack(d), d.x, d.bias, True))
+
+
+def test_run_host_entry_point():
+    d = _layer("f16", 2, 32, 48, 20, 20)
+    pk = pack(d)
+    compare(d, pk.run_host(d.x, d.bias, True))
+
+
+def test_argument_errors():
+    import torch
+    d = _layer("f32", 1, 8, 16, 10, 10)
+    pk = pack(d)
+    x = torch.zeros(1, 10, 10, 8, device="cuda")
+    y = torch.zeros(1, 10, 10, 16, device="cuda")
+    with pytest.raises(binding.PatconvError) as e:
+        pk.run(x.data_ptr() + 4, 1, 10, 10, 0, True, y.data_ptr())
+    assert e.value.status == 1
+    with pytest.raises(binding.PatconvError) as e:
+        pk.run(x.data_ptr(), 0, 10, 10, 0, True, y.data_ptr())
+    assert e.value.status == 3
+    with pytest.raises(binding.PatconvError) as e:
+        pk.run(x.data_ptr(), 1, 10, 10, 0, True, x.data_ptr())      # y overlaps x
+    assert e.value.status == 1
