@@ -72,8 +72,9 @@ PackConfig choose_pack_config(int c_in, int c_out, xgen_dtype dtype, int stride)
     return c;
 }
 
-xgen_status pack_host(const xgen_patconv_desc &d, const void *dense_w, const int16_t *pid,
+xgen_status pack_host(const xgen_patconv_desc &d, const void *dense_w, const int16_t *pid_in,
                       const PackConfig &cfg, PackedHost &out) {
+    const int16_t *pid = pid_in;
     if (!dense_w || !pid || !d.pattern_masks) return XGEN_ERR_INVALID_ARG;
     if (d.c_in < 1 || d.c_out < 1) return XGEN_ERR_INVALID_ARG;
     if (d.pad != 1 || (d.stride != 1 && d.stride != 2)) return XGEN_ERR_UNSUPPORTED;
@@ -117,6 +118,36 @@ xgen_status pack_host(const xgen_patconv_desc &d, const void *dense_w, const int
         }
     }
 
+    // Keep the survivors (compiled pattern id and the four kept weights, widened
+    // to fp32 exactly) so the layout can be rebuilt for another grouping later.
+    out.c_in = cin; out.c_out = cout; out.stride = d.stride; out.dtype = d.dtype; out.np = np;
+    out.kpat.assign((size_t)cin * cout, -1);
+    out.kw4.assign((size_t)cin * cout * 4, 0u);
+    for (int64_t k = 0; k < (int64_t)cin * cout; ++k) {
+        int p = pid[k];
+        if (p < 0) continue;
+        const int q = to_compiled[p];
+        out.kpat[k] = (int16_t)q;
+        unsigned m = out.masks[q];
+        int n = 0;
+        for (int t = 0; t < 9; ++t) {
+            if (!((m >> t) & 1)) continue;
+            float f;
+            if (d.dtype == XGEN_F32) f = ((const float *)dense_w)[k * 9 + t];
+            else if (d.dtype == XGEN_F16_F32ACC) f = half_bits_to_float(((const uint16_t *)dense_w)[k * 9 + t]);
+            else f = (float)((const int8_t *)dense_w)[k * 9 + t];
+            std::memcpy(&out.kw4[k * 4 + n++], &f, 4);
+        }
+    }
+    out.stats.kernels_total = (int64_t)cin * cout;
+    out.stats.kernels_surviving = k_surv;
+    return build_layout(out, cfg);
+}
+
+xgen_status build_layout(PackedHost &out, const PackConfig &cfg) {
+    const int cin = out.c_in, cout = out.c_out, np = out.np;
+    const int16_t *pid = out.kpat.data();           // compiled pattern ids from here on
+    const int64_t k_surv = out.stats.kernels_surviving;
     const int J = cfg.filters_per_group, cc = cfg.channels_per_chunk;
     const int wpc = cfg.groups_per_block;
     if (J < 1 || wpc < 1 || cc < 1 || (cc & (cc - 1))) return XGEN_ERR_INVALID_ARG;
@@ -125,8 +156,8 @@ xgen_status pack_host(const xgen_patconv_desc &d, const void *dense_w, const int
     const int n_groups = n_blocks * wpc;
     const int n_chunks = (cin + cc - 1) / cc;
 
-    out.c_in = cin; out.c_out = cout; out.stride = d.stride; out.dtype = d.dtype;
-    out.J = J; out.wpc = wpc; out.cc = cc; out.np = np;
+    out.J = J; out.wpc = wpc; out.cc = cc;
+    out.slots.clear(); out.max_seg_slots = 0;
     out.n_blocks = n_blocks; out.n_chunks = n_chunks;
     out.slot_oc.assign((size_t)n_groups * J, -1);
 
@@ -140,7 +171,7 @@ xgen_status pack_host(const xgen_patconv_desc &d, const void *dense_w, const int
     for (int oc = 0; oc < cout; ++oc)
         for (int ic = 0; ic < cin; ++ic) {
             int p = pid[(size_t)oc * cin + ic];
-            if (p >= 0) { ++cnt[oc]; ++hist[oc][to_compiled[p]]; }
+            if (p >= 0) { ++cnt[oc]; ++hist[oc][p]; }
         }
     std::vector<int64_t> group_kernels(n_groups, 0);
     for (int b = 0; b < n_blocks; ++b) {
@@ -188,7 +219,7 @@ xgen_status pack_host(const xgen_patconv_desc &d, const void *dense_w, const int
                     for (int j = 0; j < J; ++j) {
                         if (soc[j] < 0) continue;
                         int p = pid[(size_t)soc[j] * cin + ic];
-                        if (p >= 0) ents.push_back({to_compiled[p], j});
+                        if (p >= 0) ents.push_back({p, j});
                     }
                     if (ents.empty()) continue;  // group not connected to this channel
                     std::sort(ents.begin(), ents.end(), [](const Ent &a, const Ent &e) {
@@ -197,21 +228,7 @@ xgen_status pack_host(const xgen_patconv_desc &d, const void *dense_w, const int
                     push_slot((uint32_t)np, (uint32_t)icl, nullptr);
                     ++n_loads;
                     for (const Ent &e : ents) {
-                        size_t base = ((size_t)soc[e.j] * cin + ic) * 9;
-                        unsigned m = out.masks[e.p];
-                        uint32_t w4[4];
-                        int k = 0;
-                        for (int t = 0; t < 9; ++t) {
-                            if (!((m >> t) & 1)) continue;
-                            float f;
-                            if (d.dtype == XGEN_F32)
-                                f = ((const float *)dense_w)[base + t];
-                            else if (d.dtype == XGEN_F16_F32ACC)
-                                f = half_bits_to_float(((const uint16_t *)dense_w)[base + t]);
-                            else
-                                f = (float)((const int8_t *)dense_w)[base + t];
-                            std::memcpy(&w4[k++], &f, 4);
-                        }
+                        const uint32_t *w4 = &out.kw4[((size_t)soc[e.j] * cin + ic) * 4];
                         push_slot((uint32_t)e.p, (uint32_t)(e.j * kPixPerThread), w4);
                     }
                 }
@@ -225,10 +242,8 @@ xgen_status pack_host(const xgen_patconv_desc &d, const void *dense_w, const int
     const int64_t n_slots = (int64_t)(out.slots.size() / kSlotWords);
 
     xgen_patconv_stats &s = out.stats;
-    s.kernels_total = (int64_t)cin * cout;
-    s.kernels_surviving = k_surv;
     s.macs_per_pixel = 4 * k_surv;
-    const int wbytes = d.dtype == XGEN_F32 ? 4 : (d.dtype == XGEN_F16_F32ACC ? 2 : 1);
+    const int wbytes = out.dtype == XGEN_F32 ? 4 : (out.dtype == XGEN_F16_F32ACC ? 2 : 1);
     s.weight_bytes = 4 * k_surv * wbytes;
     s.index_bytes = n_slots * 2 + (int64_t)out.seg_off.size() * 4 + (int64_t)out.slot_oc.size() * 4;
     s.csr_index_bytes = 4 * k_surv * 4 + (int64_t)(cout + 1) * 4;

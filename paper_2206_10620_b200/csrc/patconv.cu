@@ -53,6 +53,10 @@ struct KParams {
     int vec_in;                          // c_in is a multiple of the channels per staged word
     int vec_out;                         // c_out allows 4-channel vector stores
     int opitch;                          // words per pixel row of the epilogue tile
+    int tab_off_words;                   // offset of the per-pixel staging table in shared memory
+    int chunks_per_split;                // grid.z splits the channel chunks; 0 = no split
+    uint32_t *partial;                   // split runs: [split][n*ho*wo*c_out] raw fp32 / int32 sums
+    size_t out_elems;                    // n*ho*wo*c_out
 };
 
 // ---- small PTX wrappers -----------------------------------------------------
@@ -144,24 +148,39 @@ patconv_kernel(const KParams P) {
     const int32_t *seg = P.seg_off + (size_t)b * P.n_chunks * (P.wpc + 1);
     const uint32_t smem_base = smem_u32(smem);
 
+    // Per-pixel staging table, built once: {element index of channel 0 of the input
+    // pixel, or -1 outside the image; word offset of the pixel inside a plane}.
+    int2 *tab = reinterpret_cast<int2 *>(smem + P.tab_off_words);
+    for (int q = tid; q < npix; q += nthreads) {
+        const int col = q % P.tin_w, t2 = q / P.tin_w;
+        const int row = t2 % P.tin_h, im = t2 / P.tin_h;
+        const int gy = gy0 + row, gx = gx0 + col, gn = n0 + im;
+        const bool ok = gn < P.n && gy >= 0 && gy < P.h && gx >= 0 && gx < P.w;
+        tab[q] = make_int2(ok ? ((gn * P.h + gy) * P.w + gx) * P.c_in : -1,
+                           im * P.img_stride + row * P.pitch + col);
+    }
+    __syncthreads();
+
+    const int c_begin = P.chunks_per_split ? (int)blockIdx.z * P.chunks_per_split : 0;
+    const int c_end = P.chunks_per_split ? min(P.n_chunks, c_begin + P.chunks_per_split) : P.n_chunks;
+
     const int q0 = tid / RP;
-    const int col0 = q0 % P.tin_w, row0 = (q0 / P.tin_w) % P.tin_h, im0 = q0 / (P.tin_w * P.tin_h);
-    const int dcol = pix_step % P.tin_w, drow = pix_step / P.tin_w;
     auto stage_load = [&](int c) {
-        if (c < P.n_chunks) {
-            const int stage = c % P.n_stages;
+        if (c < c_end) {
+            const int stage = (c - c_begin) % P.n_stages;
             const uint32_t act = smem_base + (uint32_t)(stage * P.stage_words) * 4u;
             // activations: one 32-bit word = E consecutive channels of one pixel
-            int col = col0, row = row0, im = im0;
             const int ic = c * P.cc + rp * E;
+            const bool ic_ok = ic < P.c_in;
+            const uint32_t plane = act + (uint32_t)(rp * P.plane_stride) * 4u;
+            const char *xc = (const char *)P.x + (size_t)ic * XB;
             for (int q = q0; q < npix; q += pix_step) {
-                const int gy = gy0 + row, gx = gx0 + col, gn = n0 + im;
-                const bool ok = gn < P.n && gy >= 0 && gy < P.h && gx >= 0 && gx < P.w && ic < P.c_in;
-                const uint32_t dst = act + (uint32_t)(rp * P.plane_stride + im * P.img_stride + row * P.pitch + col) * 4u;
-                const size_t gi = ok ? (((size_t)gn * P.h + gy) * P.w + gx) * P.c_in + ic : 0;
-                const char *src = (const char *)P.x + gi * XB;
+                const int2 t = tab[q];
+                const bool ok = ic_ok && t.x >= 0;
+                const uint32_t dst = plane + (uint32_t)t.y * 4u;
+                const char *src = xc + (size_t)(ok ? t.x : 0) * XB;
                 if (E == 1 || P.vec_in) {
-                    cp_async4(dst, src, ok ? 4 : 0);
+                    cp_async4(dst, ok ? src : (const char *)P.x, ok ? 4 : 0);
                 } else {
                     // channel count not a multiple of E: assemble the word element by element
                     uint32_t word = 0;
@@ -175,9 +194,6 @@ patconv_kernel(const KParams P) {
                     }
                     asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst), "r"(word) : "memory");
                 }
-                col += dcol; row += drow;
-                if (col >= P.tin_w) { col -= P.tin_w; ++row; }
-                while (row >= P.tin_h) { row -= P.tin_h; ++im; }
             }
             // this block's commands for the chunk: one contiguous segment
             const int s0 = seg[c * (P.wpc + 1)], s1 = seg[c * (P.wpc + 1) + P.wpc];
@@ -189,7 +205,7 @@ patconv_kernel(const KParams P) {
         cp_async_commit();
     };
 
-    for (int s = 0; s < P.n_stages - 1; ++s) stage_load(s);
+    for (int s = 0; s < P.n_stages - 1; ++s) stage_load(c_begin + s);
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -222,8 +238,8 @@ patconv_kernel(const KParams P) {
     const uint32_t plane_bytes = (uint32_t)P.plane_stride * 4u, pitch_bytes = (uint32_t)P.pitch * 4u;
 
     // --- main loop over channel chunks --------------------------------------------
-    for (int c = 0; c < P.n_chunks; ++c) {
-        const int stage = c % P.n_stages;
+    for (int c = c_begin; c < c_end; ++c) {
+        const int stage = (c - c_begin) % P.n_stages;
         if (P.n_stages == 2) cp_async_wait<0>(); else cp_async_wait<1>();
         __syncthreads();                       // chunk c has landed; everyone is done with chunk c-1
         stage_load(c + P.n_stages - 1);
@@ -231,19 +247,29 @@ patconv_kernel(const KParams P) {
         uint32_t tile_base = act;
         if (DT != XGEN_F32) {
             // widen the staged words to fp32 planes (exact for fp16 and for uint8)
-            const uint32_t *raw = smem + stage * P.stage_words;
             float *ex = reinterpret_cast<float *>(smem + P.exp_off_words);
-            const int nraw = RP * P.plane_stride;
-            for (int i = tid; i < nraw; i += nthreads) {
-                const int r = i / P.plane_stride, o = i - r * P.plane_stride;
-                const uint32_t wd = raw[i];
-                if (DT == XGEN_F16_F32ACC) {
-                    const __half2 h2 = *reinterpret_cast<const __half2 *>(&wd);
-                    ex[(2 * r) * P.plane_stride + o] = __low2float(h2);
-                    ex[(2 * r + 1) * P.plane_stride + o] = __high2float(h2);
-                } else {
+            const int quads = P.plane_stride >> 2;             // plane_stride is a multiple of 4
+            for (int r = 0; r < RP; ++r) {
+                const uint4 *raw = reinterpret_cast<const uint4 *>(smem + stage * P.stage_words + r * P.plane_stride);
+                for (int i = tid; i < quads; i += nthreads) {
+                    const uint4 wd = raw[i];
+                    const uint32_t w4[4] = {wd.x, wd.y, wd.z, wd.w};
+                    if (DT == XGEN_F16_F32ACC) {
+                        float lo[4], hi[4];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) ex[(4 * r + k) * P.plane_stride + o] = (float)((wd >> (8 * k)) & 0xFFu);
+                        for (int k = 0; k < 4; ++k) {
+                            const __half2 h2 = *reinterpret_cast<const __half2 *>(&w4[k]);
+                            lo[k] = __low2float(h2); hi[k] = __high2float(h2);
+                        }
+                        reinterpret_cast<float4 *>(ex + (2 * r) * P.plane_stride)[i] = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                        reinterpret_cast<float4 *>(ex + (2 * r + 1) * P.plane_stride)[i] = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            reinterpret_cast<float4 *>(ex + (4 * r + k) * P.plane_stride)[i] =
+                                make_float4((float)((w4[0] >> (8 * k)) & 0xFFu), (float)((w4[1] >> (8 * k)) & 0xFFu),
+                                            (float)((w4[2] >> (8 * k)) & 0xFFu), (float)((w4[3] >> (8 * k)) & 0xFFu));
+                    }
                 }
             }
             __syncthreads();
@@ -252,7 +278,7 @@ patconv_kernel(const KParams P) {
         const int s0 = seg[c * (P.wpc + 1)], sg = seg[c * (P.wpc + 1) + warp];
         uint32_t sp = act + (uint32_t)P.act_stage_words * 4u + (uint32_t)(sg - s0) * 32u;
         run_commands<STRIDE, NP>(sp, tile_base + thr_off, plane_bytes, pitch_bytes, tmem_warp);
-        if (DT == XGEN_I8_I32 && ((c + 1) % P.flush_chunks == 0)) fold_partial_sums();
+        if (DT == XGEN_I8_I32 && ((c - c_begin + 1) % P.flush_chunks == 0)) fold_partial_sums();
     }
     cp_async_wait<0>();
     if (DT == XGEN_I8_I32) fold_partial_sums();
@@ -287,6 +313,13 @@ patconv_kernel(const KParams P) {
             const int ox = tx * TW + p_x * 2 + (t & 1), oy = ty * TH + p_y * 4 + (t >> 1), on = n0 + p_n;
             if (on >= P.n || oy >= P.ho || ox >= P.wo) continue;
             const size_t pix = ((size_t)on * P.ho + oy) * P.wo + ox;
+            if (P.partial) {
+                // split run: raw sums to the workspace, no bias / ReLU / conversion
+                uint32_t *dst = P.partial + (size_t)blockIdx.z * P.out_elems + pix * P.c_out + oc_lo;
+                if (P.vec_out) *reinterpret_cast<uint4 *>(dst + sgm * 4) = *reinterpret_cast<const uint4 *>(&smem[pl * P.opitch + sgm * 4]);
+                else dst[sgm] = smem[pl * P.opitch + sgm];
+                continue;
+            }
             if (P.vec_out) {
                 const int ocl = sgm * 4;
                 const uint4 raw = *reinterpret_cast<const uint4 *>(&smem[pl * P.opitch + ocl]);
@@ -341,6 +374,53 @@ patconv_kernel(const KParams P) {
     }
 }
 
+// Split runs: y = act(bias + sum over splits of the raw partial sums), in a fixed
+// order (split 0, 1, ...), four channels per thread.
+template <int DT>
+__global__ void __launch_bounds__(256)
+patconv_reduce_kernel(const uint32_t *__restrict__ partial, int splits, size_t out_elems, int c_out,
+                      const void *__restrict__ bias, int relu, void *__restrict__ y, int vec) {
+    const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * (vec ? 4 : 1);
+    if (i >= out_elems) return;
+    const int oc = (int)(i % (size_t)c_out);
+    if (DT == XGEN_I8_I32) {
+        int r[4] = {0, 0, 0, 0};
+        for (int z = 0; z < splits; ++z) {
+            const uint32_t *src = partial + (size_t)z * out_elems + i;
+            if (vec) { const int4 v = *reinterpret_cast<const int4 *>(src); r[0] += v.x; r[1] += v.y; r[2] += v.z; r[3] += v.w; }
+            else r[0] += (int)src[0];
+        }
+        for (int k = 0; k < (vec ? 4 : 1); ++k) {
+            if (bias) r[k] += ((const int *)bias)[oc + k];
+            if (relu) r[k] = max(r[k], 0);
+            ((int *)y)[i + k] = r[k];
+        }
+    } else {
+        float r[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int z = 0; z < splits; ++z) {
+            const uint32_t *src = partial + (size_t)z * out_elems + i;
+            if (vec) { const float4 v = *reinterpret_cast<const float4 *>(src); r[0] += v.x; r[1] += v.y; r[2] += v.z; r[3] += v.w; }
+            else r[0] += __uint_as_float(src[0]);
+        }
+        for (int k = 0; k < (vec ? 4 : 1); ++k) {
+            if (bias) r[k] += ((const float *)bias)[oc + k];
+            if (relu) r[k] = fmaxf(r[k], 0.f);
+        }
+        if (DT == XGEN_F32) {
+            if (vec) *reinterpret_cast<float4 *>((float *)y + i) = make_float4(r[0], r[1], r[2], r[3]);
+            else ((float *)y)[i] = r[0];
+        } else {
+            if (vec) {
+                __half2 lo = __floats2half2_rn(r[0], r[1]), hi = __floats2half2_rn(r[2], r[3]);
+                uint2 pk;
+                pk.x = *reinterpret_cast<uint32_t *>(&lo);
+                pk.y = *reinterpret_cast<uint32_t *>(&hi);
+                *reinterpret_cast<uint2 *>((__half *)y + i) = pk;
+            } else ((__half *)y)[i] = __float2half_rn(r[0]);
+        }
+    }
+}
+
 // ---- host side ----------------------------------------------------------------------
 static std::atomic<int64_t> g_launches{0};
 
@@ -391,7 +471,7 @@ static Geometry choose_geometry(int n, int ho, int wo, int stride) {
     best.tin_h = stride == 1 ? TH + 2 : 2 * TH + 1;
     const int align = stride == 1 ? 2 : 4;                // 8- or 16-byte aligned patch rows
     int p0 = (best.tin_w + align - 1) / align * align, best_p = p0, best_c = 1 << 30;
-    for (int p = p0; p < p0 + 34; p += align) {
+    for (int p = p0; p <= p0 + 8; p += align) {
         int c = row_load_conflicts(stride, best.lx_log, best.ly_log, p, best.tin_h * p);
         if (c < best_c) { best_c = c; best_p = p; }
     }
@@ -413,7 +493,40 @@ struct xgen_patconv_packed {
     uint32_t *d_slots = nullptr;
     int32_t *d_seg_off = nullptr;
     int32_t *d_slot_oc = nullptr;
+    // set by xgen_patconv_plan: split the channel chunks of this shape across blocks
+    int plan_n = 0, plan_h = 0, plan_w = 0, plan_splits = 1, plan_cps = 0;
+    uint32_t *d_partial = nullptr;
+    size_t partial_bytes = 0;
 };
+
+static void free_device_layout(xgen_patconv_packed *h) {
+    if (h->d_slots) cudaFree(h->d_slots);
+    if (h->d_seg_off) cudaFree(h->d_seg_off);
+    if (h->d_slot_oc) cudaFree(h->d_slot_oc);
+    h->d_slots = nullptr; h->d_seg_off = nullptr; h->d_slot_oc = nullptr;
+}
+
+// Upload the host layout; the device must be current.
+static xgen_status upload_layout(xgen_patconv_packed *h) {
+    const PackedHost &p = h->host;
+    free_device_layout(h);
+    // two spare slots: harmless over-read room for 16-byte copies
+    size_t sb = (p.slots.size() + 2 * kSlotWords) * 4, gb = p.seg_off.size() * 4, ob = p.slot_oc.size() * 4;
+    cudaError_t e = cudaMalloc(&h->d_slots, sb);
+    if (e == cudaSuccess) e = cudaMalloc(&h->d_seg_off, gb);
+    if (e == cudaSuccess) e = cudaMalloc(&h->d_slot_oc, ob);
+    if (e == cudaSuccess) e = cudaMemset(h->d_slots, 0, sb);
+    if (e == cudaSuccess) e = cudaMemcpy(h->d_slots, p.slots.data(), p.slots.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(h->d_seg_off, p.seg_off.data(), gb, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(h->d_slot_oc, p.slot_oc.data(), ob, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        xgen_status r = (e == cudaErrorMemoryAllocation) ? XGEN_ERR_ALLOC : XGEN_ERR_CUDA;
+        cudaGetLastError();
+        free_device_layout(h);
+        return r;
+    }
+    return XGEN_OK;
+}
 
 // With XGEN_PATCONV_LOG set, failed CUDA calls are named on stderr.
 static cudaError_t log_cuda(cudaError_t e, const char *what) {
@@ -480,23 +593,9 @@ xgen_status xgen_patconv_pack(const xgen_patconv_desc *desc, const void *dense_w
     if (device >= 0) {
         int prev = 0;
         if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(device) != cudaSuccess) { delete h; return XGEN_ERR_CUDA; }
-        const PackedHost &p = h->host;
-        // two spare slots: harmless over-read room for 16-byte copies
-        size_t sb = (p.slots.size() + 2 * kSlotWords) * 4, gb = p.seg_off.size() * 4, ob = p.slot_oc.size() * 4;
-        cudaError_t e = cudaMalloc(&h->d_slots, sb);
-        if (e == cudaSuccess) e = cudaMalloc(&h->d_seg_off, gb);
-        if (e == cudaSuccess) e = cudaMalloc(&h->d_slot_oc, ob);
-        if (e == cudaSuccess) e = cudaMemset(h->d_slots, 0, sb);
-        if (e == cudaSuccess) e = cudaMemcpy(h->d_slots, p.slots.data(), p.slots.size() * 4, cudaMemcpyHostToDevice);
-        if (e == cudaSuccess) e = cudaMemcpy(h->d_seg_off, p.seg_off.data(), gb, cudaMemcpyHostToDevice);
-        if (e == cudaSuccess) e = cudaMemcpy(h->d_slot_oc, p.slot_oc.data(), ob, cudaMemcpyHostToDevice);
+        xgen_status us = upload_layout(h);
         cudaSetDevice(prev);
-        if (e != cudaSuccess) {
-            xgen_status r = (e == cudaErrorMemoryAllocation) ? XGEN_ERR_ALLOC : XGEN_ERR_CUDA;
-            cudaGetLastError();
-            xgen_patconv_free(h);
-            return r;
-        }
+        if (us != XGEN_OK) { delete h; return us; }
         h->device = device;
     }
     *out = h;
@@ -505,13 +604,8 @@ xgen_status xgen_patconv_pack(const xgen_patconv_desc *desc, const void *dense_w
 
 void xgen_patconv_free(xgen_patconv_packed *h) {
     if (!h) return;
-    if (h->device >= 0) {
-        cudaFree(h->d_slots); cudaFree(h->d_seg_off); cudaFree(h->d_slot_oc);
-    } else {
-        if (h->d_slots) cudaFree(h->d_slots);
-        if (h->d_seg_off) cudaFree(h->d_seg_off);
-        if (h->d_slot_oc) cudaFree(h->d_slot_oc);
-    }
+    free_device_layout(h);
+    if (h->d_partial) cudaFree(h->d_partial);
     delete h;
 }
 
@@ -542,6 +636,44 @@ xgen_status xgen_patconv_view(const xgen_patconv_packed *h, xgen_patconv_host_vi
 xgen_status xgen_patconv_plan(xgen_patconv_packed *h, int32_t n, int32_t hh, int32_t ww) {
     if (!h) return XGEN_ERR_INVALID_ARG;
     if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
+    if (h->device < 0) return XGEN_ERR_CUDA;
+    const PackedHost &p = h->host;
+    const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
+    if ((int64_t)n * ho * wo * p.c_out > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
+    const Geometry g = choose_geometry(n, ho, wo, p.stride);
+    const int64_t ctas = (int64_t)g.tiles_x * g.tiles_y * g.tiles_n * p.n_blocks;
+    const int cols_per_warp = p.J * kPixPerThread * (p.dtype == XGEN_I8_I32 ? 2 : 1);
+    const int warp_slots = 4 * (512 / cols_per_warp);                 // per SM, set by tensor memory
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
+    const int64_t target = (int64_t)sms * (warp_slots / p.wpc > 0 ? warp_slots / p.wpc : 1);
+    const size_t out_bytes = (size_t)n * ho * wo * p.c_out * 4;
+    // Splitting costs one write and one read of the fp32 output per split: cap it.
+    int64_t smax = (int64_t)((size_t)(24u << 20) / out_bytes);
+    if (smax > p.n_chunks / 2) smax = p.n_chunks / 2;
+    int64_t splits = (target + ctas - 1) / ctas;
+    if (splits > smax) splits = smax;
+    if (const char *e = getenv("XGEN_PATCONV_SPLIT")) { int v = atoi(e); if (v >= 1) splits = v < p.n_chunks ? v : p.n_chunks; }
+    if (splits < 1) splits = 1;
+    const int cps = (int)((p.n_chunks + splits - 1) / splits);
+    splits = (p.n_chunks + cps - 1) / cps;
+    int prev = 0;
+    if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
+    xgen_status rs = XGEN_OK;
+    if (cudaDeviceSynchronize() != cudaSuccess) rs = XGEN_ERR_CUDA;
+    if (rs == XGEN_OK && splits > 1) {
+        const size_t need = out_bytes * (size_t)splits;
+        if (need > h->partial_bytes) {
+            if (h->d_partial) cudaFree(h->d_partial);
+            h->d_partial = nullptr; h->partial_bytes = 0;
+            if (cudaMalloc(&h->d_partial, need) != cudaSuccess) { cudaGetLastError(); rs = XGEN_ERR_ALLOC; }
+            else h->partial_bytes = need;
+        }
+    }
+    cudaSetDevice(prev);
+    if (rs != XGEN_OK) { h->plan_splits = 1; h->plan_n = 0; return rs; }
+    h->plan_n = n; h->plan_h = hh; h->plan_w = ww;
+    h->plan_splits = (int)splits; h->plan_cps = cps;
     return XGEN_OK;
 }
 
@@ -604,8 +736,14 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_
     }
     kp.n_stages = n_stages;
     kp.exp_off_words = n_stages * kp.stage_words;
+    kp.tab_off_words = (int)((words + 1) & ~(size_t)1);
+    words = (size_t)kp.tab_off_words + 2 * (size_t)((g.tin_w * g.tin_h) << g.ln_log);
     if (words < (size_t)epi_words) words = epi_words;
     size_t smem = words * 4;
+    const bool split = h->plan_splits > 1 && h->plan_n == n && h->plan_h == hh && h->plan_w == ww && h->d_partial;
+    kp.out_elems = (size_t)n * ho * wo * p.c_out;
+    kp.chunks_per_split = split ? h->plan_cps : 0;
+    kp.partial = split ? h->d_partial : nullptr;
     // Never let more blocks share an SM than tensor memory has columns for.
     const int max_ctas = 512 / kp.tmem_cols;
     const size_t floor_bytes = (size_t)kSmemPerSM / (max_ctas + 1);
@@ -615,7 +753,7 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_
     int prev = 0;
     if (cudaGetDevice(&prev) != cudaSuccess) return XGEN_ERR_CUDA;
     if (prev != h->device && cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
-    dim3 grid((unsigned)(g.tiles_x * g.tiles_y * g.tiles_n), (unsigned)p.n_blocks, 1), block((unsigned)(p.wpc * 32), 1, 1);
+    dim3 grid((unsigned)(g.tiles_x * g.tiles_y * g.tiles_n), (unsigned)p.n_blocks, (unsigned)(split ? h->plan_splits : 1)), block((unsigned)(p.wpc * 32), 1, 1);
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e;
     if (p.dtype == XGEN_F32)
@@ -624,6 +762,19 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_
         e = p.stride == 1 ? launch_np<XGEN_F16_F32ACC, 1>(p.np, grid, block, smem, st, kp) : launch_np<XGEN_F16_F32ACC, 2>(p.np, grid, block, smem, st, kp);
     else
         e = p.stride == 1 ? launch_np<XGEN_I8_I32, 1>(p.np, grid, block, smem, st, kp) : launch_np<XGEN_I8_I32, 2>(p.np, grid, block, smem, st, kp);
+    if (e == cudaSuccess && split) {
+        const int vec = kp.vec_out;
+        const size_t items = vec ? kp.out_elems / 4 : kp.out_elems;
+        const unsigned blocks = (unsigned)((items + 255) / 256);
+        if (p.dtype == XGEN_F32)
+            patconv_reduce_kernel<XGEN_F32><<<blocks, 256, 0, st>>>(h->d_partial, h->plan_splits, kp.out_elems, p.c_out, bias, kp.relu, y, vec);
+        else if (p.dtype == XGEN_F16_F32ACC)
+            patconv_reduce_kernel<XGEN_F16_F32ACC><<<blocks, 256, 0, st>>>(h->d_partial, h->plan_splits, kp.out_elems, p.c_out, bias, kp.relu, y, vec);
+        else
+            patconv_reduce_kernel<XGEN_I8_I32><<<blocks, 256, 0, st>>>(h->d_partial, h->plan_splits, kp.out_elems, p.c_out, bias, kp.relu, y, vec);
+        e = log_cuda(cudaGetLastError(), "reduce launch");
+        if (e == cudaSuccess) g_launches.fetch_add(1);
+    }
     if (prev != h->device) cudaSetDevice(prev);
     if (e != cudaSuccess) return XGEN_ERR_CUDA;
     g_launches.fetch_add(1);

@@ -39,6 +39,8 @@ struct PackedHost {
     std::vector<int32_t> seg_off;                 // [n_blocks * n_chunks * (wpc + 1)]
     std::vector<int32_t> slot_oc;                 // [n_blocks * wpc * J], -1 = empty slot
     std::vector<uint16_t> masks;                  // [np]
+    std::vector<int16_t> kpat;                    // [c_out * c_in] compiled pattern id, -1 = removed
+    std::vector<uint32_t> kw4;                    // [c_out * c_in * 4] kept weights as fp32 bits
     xgen_patconv_stats stats{};
 };
 
@@ -48,5 +50,8 @@ PackConfig choose_pack_config(int c_in, int c_out, xgen_dtype dtype, int stride)
 // Validate the description and build the host image.  No CUDA call.
 xgen_status pack_host(const xgen_patconv_desc &desc, const void *dense_w, const int16_t *pid,
                       const PackConfig &cfg, PackedHost &out);
+
+// Rebuild slots / seg_off / slot_oc / stats of an already parsed layer for a grouping.
+xgen_status build_layout(PackedHost &p, const PackConfig &cfg);
 
 }  // namespace patconv

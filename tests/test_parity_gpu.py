@@ -125,3 +125,33 @@ def test_argument_errors():
     with pytest.raises(binding.PatconvError) as e:
         pk.run(x.data_ptr(), 1, 10, 10, 0, True, x.data_ptr())      # y overlaps x
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "i8"])
+@pytest.mark.parametrize("stride", [1, 2])
+def test_planned_shape_splits_input_channels(dtype, stride):
+    # few output pixels, many input channels: plan() splits the channel chunks across
+    # blocks and a second kernel reduces the partial sums
+    d = _layer(dtype, 1, 256, 72, 14, 14, stride, prune=0.6, lib=8, seed=11)
+    pk = pack(d)
+    pk.plan(1, 14, 14)
+    before = binding.launch_count()
+    y = run_gpu(pk, d.x, d.bias, True)
+    assert binding.launch_count() - before == 2          # split kernel + reduction
+    compare(d, y)
+    y2 = run_gpu(pk, d.x, d.bias, True)
+    assert np.array_equal(y, y2)                         # fixed reduction order
+    # another shape on the same handle runs unsplit
+    d2 = _layer(dtype, 1, 256, 72, 9, 9, stride, prune=0.6, lib=8, seed=11)
+    before = binding.launch_count()
+    y3 = run_gpu(pk, d2.x, d.bias, False)
+    assert binding.launch_count() - before == 1
+    d2.w, d2.pid, d2.masks = d.w, d.pid, d.masks
+    compare(d2, y3, bias=d.bias, relu=False)
+
+
+def test_planned_odd_channel_count():
+    d = _layer("f32", 2, 130, 37, 7, 7, 1, prune=0.3, lib=12, seed=4)
+    pk = pack(d)
+    pk.plan(2, 7, 7)
+    compare(d, run_gpu(pk, d.x, d.bias, True))
