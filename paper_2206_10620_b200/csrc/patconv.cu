@@ -89,19 +89,29 @@ __device__ __forceinline__ void tmem_st8(uint32_t ta, const uint32_t (&r)[8]) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// Stride-1 layers use the packed two-wide fp32 FMA unless built with -DPATCONV_F2=0.
+#ifndef PATCONV_F2
+#define PATCONV_F2 1
+#endif
+#if PATCONV_F2
+#define PATCONV_S1(np) PATCONV_CORE_S1_NP##np##_F2
+#else
+#define PATCONV_S1(np) PATCONV_CORE_S1_NP##np##_F1
+#endif
+
 template <int STRIDE, int NP>
-__device__ __forceinline__ void run_commands(uint32_t &sp, uint32_t tbase, uint32_t plane_bytes,
+__device__ __forceinline__ void run_commands(uint32_t sp, uint32_t tbase, uint32_t plane_bytes,
                                              uint32_t pitch_bytes, uint32_t tmem_base) {
     if (STRIDE == 1) {
-        if (NP == 4) PATCONV_CORE_S1_NP4(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
-        else if (NP == 8) PATCONV_CORE_S1_NP8(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
-        else if (NP == 12) PATCONV_CORE_S1_NP12(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
-        else PATCONV_CORE_S1_NP126(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        if (NP == 4) PATCONV_S1(4)(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        else if (NP == 8) PATCONV_S1(8)(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        else if (NP == 12) PATCONV_S1(12)(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        else PATCONV_S1(126)(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
     } else {
-        if (NP == 4) PATCONV_CORE_S2_NP4(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
-        else if (NP == 8) PATCONV_CORE_S2_NP8(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
-        else if (NP == 12) PATCONV_CORE_S2_NP12(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
-        else PATCONV_CORE_S2_NP126(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        if (NP == 4) PATCONV_CORE_S2_NP4_F1(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        else if (NP == 8) PATCONV_CORE_S2_NP8_F1(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        else if (NP == 12) PATCONV_CORE_S2_NP12_F1(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        else PATCONV_CORE_S2_NP126_F1(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
     }
 }
 
@@ -199,7 +209,7 @@ patconv_kernel(const KParams P) {
             const int s0 = seg[c * (P.wpc + 1)], s1 = seg[c * (P.wpc + 1) + P.wpc];
             const uint32_t cmd = act + (uint32_t)P.act_stage_words * 4u;
             const uint4 *gsrc = reinterpret_cast<const uint4 *>(P.slots + (size_t)s0 * kSlotWords);
-            const int n16 = (s1 - s0) * 2;
+            const int n16 = (s1 - s0 + 2) * 2;          // two look-ahead slots beyond the segment
             for (int i = tid; i < n16; i += nthreads) cp_async16(cmd + (uint32_t)i * 16u, gsrc + i);
         }
         cp_async_commit();
@@ -714,7 +724,7 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_
     const int E = p.dtype == XGEN_F32 ? 1 : (p.dtype == XGEN_F16_F32ACC ? 2 : 4);
     kp.raw_planes = p.cc / E;
     kp.act_stage_words = (kp.raw_planes * g.plane_stride + 3) & ~3;
-    kp.cmd_stage_words = p.max_seg_slots * kSlotWords;
+    kp.cmd_stage_words = (p.max_seg_slots + 2) * kSlotWords;
     kp.stage_words = kp.act_stage_words + kp.cmd_stage_words;
     kp.vec_in = (p.c_in % E) == 0;
     kp.vec_out = (p.c_out % 4) == 0;
