@@ -30,9 +30,11 @@ every block emitted once per set.  While command i runs from set A:
   * command i+2 is read from shared memory into set A once command i's weights
     are consumed;
   * the block ends with an indirect branch on set B's opcode (brx.idx).
-The packer never places two kernel commands of one filter back to back, and
-every fetch of a row is preceded by tcgen05.wait::st, so a row is never read
-while a write to it is in flight.  The stream segment is staged with two valid
+Between two LOADs every kernel command addresses a different filter, so the
+row fetched ahead by a kernel command is never one with a write in flight; a
+LOAD (and the block's exit) waits for all writes (tcgen05.wait::st) before it
+fetches ahead, which covers a filter that ends one channel and starts the
+next.  A row fetched ahead for a LOAD or END command is never used.  The stream segment is staged with two valid
 spare slots so the look-ahead never reads undefined data.
 
 Operands of every block, in order:
@@ -94,18 +96,20 @@ def gen_block(np_, stride, f2):
     L.append(" brx.idx opA, tsA;")
 
     for S, O in (("A", "B"), ("B", "A")):
-        def prefetch_next():
-            return [" tcgen05.wait::ld.sync.aligned;",          # my own row has arrived
-                    " add.u32 ta%s, %%4, pay%s;" % (O, O),
-                    " tcgen05.wait::st.sync.aligned;",          # no write to any row is in flight
-                    " tcgen05.ld.sync.aligned.32x32b.x8.b32 %s, [ta%s];" % (accs(O), O)]
+        def prefetch_next(fence):
+            r = [" tcgen05.wait::ld.sync.aligned;",             # my own row has arrived
+                 " add.u32 ta%s, %%4, pay%s;" % (O, O)]
+            if fence:
+                r.append(" tcgen05.wait::st.sync.aligned;")     # no write to any row is in flight
+            r.append(" tcgen05.ld.sync.aligned.32x32b.x8.b32 %s, [ta%s];" % (accs(O), O))
+            return r
 
         def refill_and_go():
             return fetch(S, 0) + [" add.u32 %0, %0, 32;", " brx.idx op%s, ts%s;" % (O, O)]
 
         for pi, m in enumerate(masks):
             L.append(" K%s%d:" % (S, pi))
-            L += prefetch_next()
+            L += prefetch_next(False)
             taps = [t for t in range(9) if (m >> t) & 1]
             if f2:
                 for k in range(4):
@@ -130,7 +134,7 @@ def gen_block(np_, stride, f2):
             L += refill_and_go()
 
         L.append(" LOAD%s:" % S)
-        L += prefetch_next()
+        L += prefetch_next(True)
         L.append(" mad.lo.u32 ad, pay%s, %%2, %%1;" % S)
         for r in range(rows):
             if stride == 1:
