@@ -32,7 +32,6 @@ namespace patconv {
 constexpr int kSmemPerSM = 233472;     // 228 KB
 constexpr int kSmemMaxDynamic = 232448 - 1024;  // 227 KB per block less static shared memory
 constexpr int kMaxWarps = 8;
-constexpr int kEpiPix = 2;             // pixels per thread handled in one epilogue pass
 
 struct KParams {
     const void *x; void *y; const void *bias;
@@ -54,6 +53,9 @@ struct KParams {
     int vec_out;                         // c_out allows 4-channel vector stores
     int opitch;                          // words per pixel row of the epilogue tile
     int tab_off_words;                   // offset of the per-pixel staging table in shared memory
+    int ptab_off_words;                  // offset of the output-pixel table (256 entries)
+    int epi_pix;                         // pixels per thread handled in one epilogue pass (2, 4 or 8)
+    int segs_log;                        // log2 of the 16-byte segments per pixel row, or -1
     int chunks_per_split;                // grid.z splits the channel chunks; 0 = no split
     uint32_t *partial;                   // split runs: [split][n*ho*wo*c_out] raw fp32 / int32 sums
     size_t out_elems;                    // n*ho*wo*c_out
@@ -81,6 +83,10 @@ __device__ __forceinline__ void tmem_ld8(uint32_t ta, uint32_t (&r)[8]) {
 __device__ __forceinline__ void tmem_ld2(uint32_t ta, uint32_t (&r)[2]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0,%1}, [%2];"
                  : "=r"(r[0]), "=r"(r[1]) : "r"(ta) : "memory");
+}
+__device__ __forceinline__ void tmem_ld4(uint32_t ta, uint32_t (&r)[4]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(ta) : "memory");
 }
 __device__ __forceinline__ void tmem_st8(uint32_t ta, const uint32_t (&r)[8]) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
@@ -168,6 +174,14 @@ patconv_kernel(const KParams P) {
         const bool ok = gn < P.n && gy >= 0 && gy < P.h && gx >= 0 && gx < P.w;
         tab[q] = make_int2(ok ? ((gn * P.h + gy) * P.w + gx) * P.c_in : -1,
                            im * P.img_stride + row * P.pitch + col);
+    }
+    // Output-pixel table: linear pixel index of (pixel t of lane l), or -1 outside the output.
+    int *ptab = reinterpret_cast<int *>(smem + P.ptab_off_words);
+    for (int i = tid; i < 256; i += nthreads) {
+        const int t = i >> 5, l2 = i & 31;
+        const int p_x = l2 & (LX - 1), p_y = (l2 >> P.lx_log) & (LY - 1), p_n = l2 >> (P.lx_log + P.ly_log);
+        const int ox = tx * TW + p_x * 2 + (t & 1), oy = ty * TH + p_y * 4 + (t >> 1), on = n0 + p_n;
+        ptab[i] = (on < P.n && oy < P.ho && ox < P.wo) ? (on * P.ho + oy) * P.wo + ox : -1;
     }
     __syncthreads();
 
@@ -300,29 +314,33 @@ patconv_kernel(const KParams P) {
     const int nvalid = min(ocb, P.c_out - oc_lo);
     const int32_t *soc = P.slot_oc + ((size_t)(b * P.wpc + warp)) * P.J;
     const uint32_t tmem_res = DT == XGEN_I8_I32 ? tmem_int : tmem_warp;
-    for (int t0 = 0; t0 < kPixPerThread; t0 += kEpiPix) {
+    const int EP = P.epi_pix;
+    for (int t0 = 0; t0 < kPixPerThread; t0 += EP) {
         for (int j = 0; j < P.J; ++j) {
             const int oc = soc[j];
-            uint32_t v[2];
-            tmem_ld2(tmem_res + j * 8 + t0, v);
+            uint32_t v[8];
+            if (EP == 8) { tmem_ld8(tmem_res + j * 8, v); }
+            else if (EP == 4) { uint32_t q[4]; tmem_ld4(tmem_res + j * 8 + t0, q); v[0] = q[0]; v[1] = q[1]; v[2] = q[2]; v[3] = q[3]; }
+            else { uint32_t q[2]; tmem_ld2(tmem_res + j * 8 + t0, q); v[0] = q[0]; v[1] = q[1]; }
             tmem_wait_ld();
             if (oc >= 0) {
-                smem[(0 * 32 + lane) * P.opitch + (oc - oc_lo)] = v[0];
-                smem[(1 * 32 + lane) * P.opitch + (oc - oc_lo)] = v[1];
+                uint32_t *dst = smem + lane * P.opitch + (oc - oc_lo);
+#pragma unroll
+                for (int tt = 0; tt < 8; ++tt)
+                    if (tt < EP) dst[tt * 32 * P.opitch] = v[tt];
             }
         }
         __syncthreads();
-        // cooperative store: kEpiPix*32 pixels x nvalid channels
+        // cooperative store: EP*32 pixels x nvalid channels
         const int segs = P.vec_out ? (nvalid >> 2) : nvalid;
-        const int total = kEpiPix * 32 * segs;
+        const int total = EP * 32 * segs;
         for (int i = tid; i < total; i += nthreads) {
-            const int pl = i / segs, sgm = i - pl * segs;     // pl = tt*32 + lane'
-            const int tt = pl >> 5, ln2 = pl & 31;
-            const int t = t0 + tt;
-            const int p_x = ln2 & (LX - 1), p_y = (ln2 >> P.lx_log) & (LY - 1), p_n = ln2 >> (P.lx_log + P.ly_log);
-            const int ox = tx * TW + p_x * 2 + (t & 1), oy = ty * TH + p_y * 4 + (t >> 1), on = n0 + p_n;
-            if (on >= P.n || oy >= P.ho || ox >= P.wo) continue;
-            const size_t pix = ((size_t)on * P.ho + oy) * P.wo + ox;
+            int pl, sgm;                                      // pl = tt*32 + lane'
+            if (P.segs_log >= 0 && segs == (1 << P.segs_log)) { pl = i >> P.segs_log; sgm = i & (segs - 1); }
+            else { pl = i / segs; sgm = i - pl * segs; }
+            const int pidx = ptab[t0 * 32 + pl];
+            if (pidx < 0) continue;
+            const size_t pix = (size_t)pidx;
             if (P.partial) {
                 // split run: raw sums to the workspace, no bias / ReLU / conversion
                 uint32_t *dst = P.partial + (size_t)blockIdx.z * P.out_elems + pix * P.c_out + oc_lo;
@@ -737,25 +755,42 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_
     const int ocb = p.J * p.wpc;
     kp.opitch = ocb + 4;
     const int exp_words = p.dtype == XGEN_F32 ? 0 : p.cc * g.plane_stride;
-    const int epi_words = kEpiPix * 32 * kp.opitch;
+    const int npix_tile = (g.tin_w * g.tin_h) << g.ln_log;
+    const int max_ctas = 512 / kp.tmem_cols;          // blocks per SM that tensor memory has columns for
+    // Pick the stage count: three stages unless two let more blocks share an SM.
+    auto smem_words = [&](int stages, int ep) {
+        size_t w = (size_t)stages * kp.stage_words + exp_words;
+        const size_t epi = (size_t)ep * 32 * kp.opitch;
+        if (w < epi) w = epi;
+        return ((w + 1) & ~(size_t)1) + 2 * (size_t)npix_tile + 256;
+    };
+    auto occupancy = [&](size_t words) {
+        int o = (int)((size_t)kSmemPerSM / (words * 4 + 1040));
+        return o < max_ctas ? o : max_ctas;
+    };
     int n_stages = 3;
-    size_t words = 0;
-    for (;; --n_stages) {
-        words = (size_t)n_stages * kp.stage_words + exp_words;
-        if (words * 4 <= (size_t)kSmemMaxDynamic / 2 || n_stages == 2) break;
-    }
+    if (smem_words(3, 2) * 4 > (size_t)kSmemMaxDynamic || occupancy(smem_words(2, 2)) > occupancy(smem_words(3, 2))) n_stages = 2;
     kp.n_stages = n_stages;
     kp.exp_off_words = n_stages * kp.stage_words;
-    kp.tab_off_words = (int)((words + 1) & ~(size_t)1);
-    words = (size_t)kp.tab_off_words + 2 * (size_t)((g.tin_w * g.tin_h) << g.ln_log);
-    if (words < (size_t)epi_words) words = epi_words;
+    // The epilogue tile reuses the staging memory: as many pixels per pass as fit for free.
+    int ep = 2;
+    for (int cand = 8; cand > 2; cand >>= 1)
+        if (smem_words(n_stages, cand) * 4 <= (size_t)kSmemMaxDynamic && occupancy(smem_words(n_stages, cand)) >= occupancy(smem_words(n_stages, 2))) { ep = cand; break; }
+    kp.epi_pix = ep;
+    size_t words = smem_words(n_stages, ep);
+    kp.ptab_off_words = (int)(words - 256);
+    kp.tab_off_words = kp.ptab_off_words - 2 * npix_tile;
+    {
+        const int segs = kp.vec_out ? (ocb >> 2) : ocb;
+        kp.segs_log = -1;
+        for (int l = 0; l < 12; ++l) if ((1 << l) == segs) kp.segs_log = l;
+    }
     size_t smem = words * 4;
     const bool split = h->plan_splits > 1 && h->plan_n == n && h->plan_h == hh && h->plan_w == ww && h->d_partial;
     kp.out_elems = (size_t)n * ho * wo * p.c_out;
     kp.chunks_per_split = split ? h->plan_cps : 0;
     kp.partial = split ? h->d_partial : nullptr;
     // Never let more blocks share an SM than tensor memory has columns for.
-    const int max_ctas = 512 / kp.tmem_cols;
     const size_t floor_bytes = (size_t)kSmemPerSM / (max_ctas + 1);
     if (smem < floor_bytes) smem = floor_bytes;
     if (smem > (size_t)kSmemMaxDynamic) return XGEN_ERR_UNSUPPORTED;
