@@ -39,6 +39,26 @@ UNIT = "GFLOP/s"
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 
 
+def rank_seed(rank: int) -> int:
+    """Every rank draws its own image (weak scaling: the batch is sharded by rank)."""
+    return wl.BASE_SEED + rank
+
+
+def max_over_ranks(x: float, dist, device) -> float:
+    """The job's time is the slowest rank's (all-reduce MAX; identity for one rank)."""
+    if dist is None:
+        return float(x)
+    import torch
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gflops(useful_macs_per_rank: int, world: int, ms: float) -> float:
+    """Useful GFLOP/s of all ranks together over the slowest rank's time."""
+    return 2.0 * useful_macs_per_rank * world / (ms * 1e-3) / 1e9
+
+
 def workload(name="vgg16"):
     return wl.CONFIGS[name]()
 
@@ -157,7 +177,7 @@ def run_gpu(args):
     layers = []
     tdt = {"f32": torch.float32, "f16": torch.float16, "i8": torch.int32}
     for s in specs:
-        d = wl.make_layer(s, seed=wl.BASE_SEED + rank)       # each rank its own image
+        d = wl.make_layer(s, seed=rank_seed(rank))
         pk = binding.Packed(s.c_in, s.c_out, s.stride, s.dtype, d.masks, d.w, d.pid, device=local)
         pk.plan(s.n, s.h, s.w)
         x = torch.from_numpy(d.x).to(dev)
@@ -195,14 +215,10 @@ def run_gpu(args):
     launches = binding.launch_count() - launches0
     clocks = sampler.stop()
     ms_steps = [a.elapsed_time(b) for a, b in ev]
-    ms = float(np.mean(ms_steps))
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(float(np.mean(ms_steps)), dist, dev)
     useful = sum(s.useful_macs() for s in specs)
     dense = sum(s.dense_macs() for s in specs)
-    value = 2.0 * useful * world / (ms * 1e-3) / 1e9
+    value = whole_job_gflops(useful, world, ms)
 
     # --- per-layer device times (L2 flushed before each layer) for the roofline
     hbm, hbm_src = measured_hbm_gbs()
@@ -251,10 +267,7 @@ def run_gpu(args):
             pk.run_host(d.x, d.bias, s.relu)
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_s], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks(e2e_s, dist, dev)
     e2e = {"value": 2.0 * useful * world / e2e_s / 1e9, "unit": UNIT,
            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_s * 1e3}
 
