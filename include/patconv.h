@@ -88,7 +88,8 @@ typedef struct {
  *   word 0  opcode:  p < patterns_compiled  -> kernel command with compiled pattern p
  *                    patterns_compiled      -> LOAD: fetch the activation patch of one channel
  *                    patterns_compiled + 1  -> END of this group's commands for the chunk
- *   word 1  operand: kernel command: 8 * j (j = filter slot inside the group);
+ *   word 1  operand: kernel command: T * j (j = filter slot inside the group; T = 16 at
+ *                    stride 1, 8 at stride 2: the output pixels one thread owns);
  *                    LOAD: channel index inside the chunk
  *   word 4..7  kernel command: the four kept weights in ascending tap order, fp32 bit
  *              patterns (fp16 and int8 weights are widened exactly)

@@ -9,32 +9,29 @@ PTX block that interprets a warp's command stream from shared memory.
 
 Commands are 32-byte slots {opcode, operand, -, -, w0, w1, w2, w3}:
   opcode p < NP : kernel command.  The operand is the tensor-memory column of
-                  the addressed filter's 8 running sums (2x4 output pixels of
-                  this thread).  The block for pattern p multiplies the four
-                  weights with the 4 taps x 8 pixels of the register-resident
+                  the addressed filter's running sums (one per output pixel of
+                  this thread: 4x4 pixels at stride 1, 2x4 at stride 2).  The
+                  block for pattern p multiplies the four weights with the 4
+                  taps of every pixel, read from the register-resident
                   activation patch; tap offsets are immediate register names.
   opcode NP     : LOAD.  The operand is the channel inside the staged chunk;
-                  the thread's patch (2x4 pixels plus halo) is read from the
+                  the thread's patch (its pixels plus halo) is read from the
                   staged tile into registers.
   opcode NP + 1 : END of the warp's commands for this chunk.
 
 The running sums live in tensor memory because the filter a command addresses
-is data: tensor-memory columns can be addressed at run time, registers cannot.
-The pattern selects code, so nothing inside a kernel command is indexed or
-branches.
+is data: tensor-memory columns can be addressed at run time, registers cannot
+(a row round trip is about 40 cycles).  The pattern selects code, so nothing
+inside a kernel command is indexed or branches.
 
-The interpreter is software-pipelined over two register sets (A and B), with
-every block emitted once per set.  While command i runs from set A:
-  * command i+1 is already decoded in set B, and its row of sums is fetched
-    from tensor memory (tcgen05.ld) before command i's arithmetic starts;
-  * command i+2 is read from shared memory into set A once command i's weights
-    are consumed;
-  * the block ends with an indirect branch on set B's opcode (brx.idx).
-Between two LOADs every kernel command addresses a different filter, so the
-row fetched ahead by a kernel command is never one with a write in flight; a
-LOAD (and the block's exit) waits for all writes (tcgen05.wait::st) before it
-fetches ahead, which covers a filter that ends one channel and starts the
-next.  A row fetched ahead for a LOAD or END command is never used.  The stream segment is staged with two valid
+Command decoding is software-pipelined over two register sets (A and B), with
+every block emitted once per set: while command i runs from set A, command i+1
+is already decoded in set B, command i+2 is read from shared memory into set A
+once command i's weights are consumed, and the block ends with an indirect
+branch on set B's opcode (brx.idx).  Between two LOADs every kernel command
+addresses a different filter; a LOAD and the block's exit wait for all
+tensor-memory writes (tcgen05.wait::st), which covers a filter that ends one
+channel and starts the next.  The stream segment is staged with two valid
 spare slots so the look-ahead never reads undefined data.
 
 Operands of every block, in order:
@@ -55,27 +52,30 @@ def table(np_):
 
 
 def gen_block(np_, stride, f2):
-    """f2: use packed two-wide fp32 FMAs (fma.rn.f32x2); stride 1 only."""
+    """One interpreter block.  Stride 1: a thread owns 4x4 output pixels (16 running
+    sums per filter, patch 6x6); stride 2: 2x4 pixels (8 sums, patch 9x5).
+    f2: packed two-wide fp32 FMAs (fma.rn.f32x2), stride 1 only."""
     assert not (f2 and stride != 1)
     masks = table(np_)
-    rows, cols = (6, 4) if stride == 1 else (9, 5)
+    bw, bh = (4, 4) if stride == 1 else (2, 4)
+    T = bw * bh
+    rows = (bh - 1) * stride + 3
+    cols = (bw - 1) * stride + 3
     npatch = rows * cols
+    npair = cols - 1
     L = ["{"]
-    L.append(" .reg .b32 opA, payA, taA, opB, payB, taB, ad;")
-    L.append(" .reg .f32 wA<4>, wB<4>, aA<8>, aB<8>, p<%d>;" % npatch)
+    L.append(" .reg .b32 opA, payA, opB, payB, ta, ad;")
+    L.append(" .reg .f32 wA<4>, wB<4>, a<%d>, p<%d>;" % (T, npatch if not f2 else cols))
     if f2:
-        L.append(" .reg .b64 q<%d>, acc<4>, wd<4>;" % (rows * 3))
+        L.append(" .reg .b64 q<%d>, acc<%d>, wd<4>;" % (rows * npair, T // 2))
     # Registers written on one path and read on another must be defined on every
     # path into the branch tables, or register allocation degrades badly.
     if f2:
-        for i in range(rows * 3):
+        for i in range(rows * npair):
             L.append(" mov.b64 q%d, 0;" % i)
     else:
         for i in range(npatch):
             L.append(" mov.f32 p%d, 0f00000000;" % i)
-    for i in range(8):
-        L.append(" mov.f32 aB%d, 0f00000000;" % i)
-    L.append(" mov.b32 taB, %4;")
     for S in "AB":
         L.append(" ts%s: .branchtargets %s;" % (
             S, ",".join("K%s%d" % (S, i) for i in range(len(masks))) + ",LOAD%s,END%s" % (S, S)))
@@ -84,69 +84,61 @@ def gen_block(np_, stride, f2):
         return [" ld.shared.v2.b32 {op%s, pay%s}, [%%0+%d];" % (S, S, off),
                 " ld.shared.v4.f32 {w%s0,w%s1,w%s2,w%s3}, [%%0+%d];" % (S, S, S, S, off + 16)]
 
-    def accs(S):
-        return "{" + ",".join("a%s%d" % (S, i) for i in range(8)) + "}"
+    accs = "{" + ",".join("a%d" % i for i in range(T)) + "}"
 
-    # prologue: commands 0 and 1 decoded, row of command 0 requested
+    # prologue: commands 0 and 1 decoded
     L += fetch("A", 0) + fetch("B", 32)
     L.append(" add.u32 %0, %0, 64;")
-    L.append(" add.u32 taA, %4, payA;")
-    L.append(" tcgen05.wait::st.sync.aligned;")
-    L.append(" tcgen05.ld.sync.aligned.32x32b.x8.b32 %s, [taA];" % accs("A"))
     L.append(" brx.idx opA, tsA;")
 
     for S, O in (("A", "B"), ("B", "A")):
-        def prefetch_next(fence):
-            r = [" tcgen05.wait::ld.sync.aligned;",             # my own row has arrived
-                 " add.u32 ta%s, %%4, pay%s;" % (O, O)]
-            if fence:
-                r.append(" tcgen05.wait::st.sync.aligned;")     # no write to any row is in flight
-            r.append(" tcgen05.ld.sync.aligned.32x32b.x8.b32 %s, [ta%s];" % (accs(O), O))
-            return r
-
         def refill_and_go():
             return fetch(S, 0) + [" add.u32 %0, %0, 32;", " brx.idx op%s, ts%s;" % (O, O)]
 
         for pi, m in enumerate(masks):
             L.append(" K%s%d:" % (S, pi))
-            L += prefetch_next(False)
+            L.append(" add.u32 ta, %%4, pay%s;" % S)
+            L.append(" tcgen05.ld.sync.aligned.32x32b.x%d.b32 %s, [ta];" % (T, accs))
             taps = [t for t in range(9) if (m >> t) & 1]
             if f2:
                 for k in range(4):
                     L.append(" mov.b64 wd%d, {w%s%d, w%s%d};" % (k, S, k, S, k))
-                for py in range(4):
-                    L.append(" mov.b64 acc%d, {a%s%d, a%s%d};" % (py, S, 2 * py, S, 2 * py + 1))
+            L.append(" tcgen05.wait::ld.sync.aligned;")
+            if f2:
+                for n in range(T // 2):
+                    L.append(" mov.b64 acc%d, {a%d, a%d};" % (n, 2 * n, 2 * n + 1))
                 for k, t in enumerate(taps):
                     dy, dx = divmod(t, 3)
-                    for py in range(4):
-                        L.append(" fma.rn.f32x2 acc%d, wd%d, q%d, acc%d;" % (py, k, (py + dy) * 3 + dx, py))
-                for py in range(4):
-                    L.append(" mov.b64 {a%s%d, a%s%d}, acc%d;" % (S, 2 * py, S, 2 * py + 1, py))
+                    for py in range(bh):
+                        for h in range(bw // 2):
+                            L.append(" fma.rn.f32x2 acc%d, wd%d, q%d, acc%d;" % (
+                                py * (bw // 2) + h, k, (py + dy) * npair + dx + 2 * h, py * (bw // 2) + h))
+                for n in range(T // 2):
+                    L.append(" mov.b64 {a%d, a%d}, acc%d;" % (2 * n, 2 * n + 1, n))
             else:
                 for k, t in enumerate(taps):
                     dy, dx = divmod(t, 3)
-                    for py in range(4):
-                        for px in range(2):
+                    for py in range(bh):
+                        for px in range(bw):
                             pr = (py * stride + dy) * cols + px * stride + dx
-                            a = py * 2 + px
-                            L.append(" fma.rn.f32 a%s%d, w%s%d, p%d, a%s%d;" % (S, a, S, k, pr, S, a))
-            L.append(" tcgen05.st.sync.aligned.32x32b.x8.b32 [ta%s], %s;" % (S, accs(S)))
+                            a = py * bw + px
+                            L.append(" fma.rn.f32 a%d, w%s%d, p%d, a%d;" % (a, S, k, pr, a))
+            L.append(" tcgen05.st.sync.aligned.32x32b.x%d.b32 [ta], %s;" % (T, accs))
             L += refill_and_go()
 
         L.append(" LOAD%s:" % S)
-        L += prefetch_next(True)
+        L.append(" tcgen05.wait::st.sync.aligned;")          # no write to any row is in flight
         L.append(" mad.lo.u32 ad, pay%s, %%2, %%1;" % S)
         for r in range(rows):
             if stride == 1:
                 if f2:
-                    L.append(" ld.shared.v2.f32 {p0,p1}, [ad];")
-                    L.append(" ld.shared.v2.f32 {p2,p3}, [ad+8];")
-                    L.append(" mov.b64 q%d, {p0,p1};" % (r * 3))
-                    L.append(" mov.b64 q%d, {p1,p2};" % (r * 3 + 1))
-                    L.append(" mov.b64 q%d, {p2,p3};" % (r * 3 + 2))
+                    L.append(" ld.shared.v4.f32 {p0,p1,p2,p3}, [ad];")
+                    L.append(" ld.shared.v2.f32 {p4,p5}, [ad+16];")
+                    for c in range(npair):
+                        L.append(" mov.b64 q%d, {p%d,p%d};" % (r * npair + c, c, c + 1))
                 else:
-                    L.append(" ld.shared.v2.f32 {p%d,p%d}, [ad];" % (r * 4, r * 4 + 1))
-                    L.append(" ld.shared.v2.f32 {p%d,p%d}, [ad+8];" % (r * 4 + 2, r * 4 + 3))
+                    L.append(" ld.shared.v4.f32 {p%d,p%d,p%d,p%d}, [ad];" % tuple(r * 6 + i for i in range(4)))
+                    L.append(" ld.shared.v2.f32 {p%d,p%d}, [ad+16];" % (r * 6 + 4, r * 6 + 5))
             else:
                 L.append(" ld.shared.v4.f32 {p%d,p%d,p%d,p%d}, [ad];" % tuple(r * 5 + i for i in range(4)))
                 L.append(" ld.shared.f32 p%d, [ad+16];" % (r * 5 + 4))
@@ -157,7 +149,6 @@ def gen_block(np_, stride, f2):
         L.append(" END%s:" % S)
         L.append(" bra.uni DONE;")
     L.append(" DONE:")
-    L.append(" tcgen05.wait::ld.sync.aligned;")
     L.append(" tcgen05.wait::st.sync.aligned;")
     L.append("}")
     return L

@@ -61,14 +61,17 @@ static float half_bits_to_float(uint16_t h) {
 }
 
 PackConfig choose_pack_config(int c_in, int c_out, xgen_dtype dtype, int stride) {
-    (void)stride;
     PackConfig c;
-    // The integer variant keeps two rows of sums per filter (an exact fp32
-    // partial sum and the int32 total), so it groups half as many filters.
-    c.filters_per_group = dtype == XGEN_I8_I32 ? 8 : 16;
-    int groups = (c_out + c.filters_per_group - 1) / c.filters_per_group;
-    c.groups_per_block = std::min(groups, 8);
     c.channels_per_chunk = c_in <= 4 ? 4 : 8;
+    // A warp's running sums take J x (pixels per thread) tensor-memory columns, and an SM
+    // has 4 x 512 of them: 128 columns per warp lets 16 warps share an SM.  Long integer
+    // layers keep a second row per filter (int32 totals), so they group half as many.
+    const int n_chunks = (c_in + c.channels_per_chunk - 1) / c.channels_per_chunk;
+    const bool fold = dtype == XGEN_I8_I32 && n_chunks > 16777216 / (c.channels_per_chunk * 4 * 32640);
+    c.filters_per_group = 128 / pix_per_thread(stride);
+    if (fold && stride == 2) c.filters_per_group /= 2;
+    int groups = (c_out + c.filters_per_group - 1) / c.filters_per_group;
+    c.groups_per_block = std::min(groups, fold && stride == 1 ? 8 : 16);
     return c;
 }
 
@@ -229,7 +232,7 @@ xgen_status build_layout(PackedHost &out, const PackConfig &cfg) {
                     ++n_loads;
                     for (const Ent &e : ents) {
                         const uint32_t *w4 = &out.kw4[((size_t)soc[e.j] * cin + ic) * 4];
-                        push_slot((uint32_t)e.p, (uint32_t)(e.j * kPixPerThread), w4);
+                        push_slot((uint32_t)e.p, (uint32_t)(e.j * pix_per_thread(out.stride)), w4);
                     }
                 }
                 push_slot((uint32_t)np + 1, 0, nullptr);

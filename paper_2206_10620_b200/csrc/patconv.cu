@@ -1,8 +1,9 @@
 // libpatconv: CUDA kernels (sm_100a) and the C ABI.
 //
 // One thread block = one tile of output pixels x one block of contiguous output
-// channels.  Each warp owns a filter group (J filters); each lane owns a 2x4
-// block of output pixels (up to LN images side by side for small images).
+// channels.  Each warp owns a filter group (J filters); each lane owns a
+// 4x4 block of output pixels (2x4 at stride 2; up to LN images side by side for
+// small images).
 // Per chunk of input channels the block stages (cp.async) the input tile with
 // its halo into channel planes in shared memory -- the NHWC -> plane transpose
 // happens in that copy -- together with the block's slice of the command
@@ -31,7 +32,7 @@ namespace patconv {
 
 constexpr int kSmemPerSM = 233472;     // 228 KB
 constexpr int kSmemMaxDynamic = 232448 - 1024;  // 227 KB per block less static shared memory
-constexpr int kMaxWarps = 8;
+constexpr int kMaxWarps = 16;
 
 struct KParams {
     const void *x; void *y; const void *bias;
@@ -53,8 +54,9 @@ struct KParams {
     int vec_out;                         // c_out allows 4-channel vector stores
     int opitch;                          // words per pixel row of the epilogue tile
     int tab_off_words;                   // offset of the per-pixel staging table in shared memory
-    int ptab_off_words;                  // offset of the output-pixel table (256 entries)
-    int epi_pix;                         // pixels per thread handled in one epilogue pass (2, 4 or 8)
+    int ptab_off_words;                  // offset of the output-pixel table (32 lanes x pixels per thread)
+    int epi_pix;                         // pixels per thread handled in one epilogue pass (2, 4, 8 or 16)
+    int fold;                            // i8: keep int32 totals in a second row and fold periodically
     int segs_log;                        // log2 of the 16-byte segments per pixel row, or -1
     int chunks_per_split;                // grid.z splits the channel chunks; 0 = no split
     uint32_t *partial;                   // split runs: [split][n*ho*wo*c_out] raw fp32 / int32 sums
@@ -135,6 +137,8 @@ patconv_kernel(const KParams P) {
     __shared__ uint32_t tmem_base_s;
     constexpr int E = DTraits<DT>::E;
     constexpr int XB = DTraits<DT>::xbytes;
+    constexpr int BW = STRIDE == 1 ? 4 : 2, BH = 4;   // output pixels per thread: BW x BH
+    constexpr int T = BW * BH;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nthreads = blockDim.x;
@@ -145,7 +149,7 @@ patconv_kernel(const KParams P) {
     const int tn = tile / P.tiles_y;
     const int LX = 1 << P.lx_log, LY = 1 << P.ly_log;
     const int l_x = lane & (LX - 1), l_y = (lane >> P.lx_log) & (LY - 1), l_n = lane >> (P.lx_log + P.ly_log);
-    const int TW = 2 * LX, TH = 4 * LY;
+    const int TW = BW * LX, TH = BH * LY;
     const int n0 = tn << P.ln_log;                   // first image of the tile
     const int gy0 = ty * TH * STRIDE - 1, gx0 = tx * TW * STRIDE - 1;   // input coords of tile (0,0)
 
@@ -177,10 +181,10 @@ patconv_kernel(const KParams P) {
     }
     // Output-pixel table: linear pixel index of (pixel t of lane l), or -1 outside the output.
     int *ptab = reinterpret_cast<int *>(smem + P.ptab_off_words);
-    for (int i = tid; i < 256; i += nthreads) {
+    for (int i = tid; i < 32 * T; i += nthreads) {
         const int t = i >> 5, l2 = i & 31;
         const int p_x = l2 & (LX - 1), p_y = (l2 >> P.lx_log) & (LY - 1), p_n = l2 >> (P.lx_log + P.ly_log);
-        const int ox = tx * TW + p_x * 2 + (t & 1), oy = ty * TH + p_y * 4 + (t >> 1), on = n0 + p_n;
+        const int ox = tx * TW + p_x * BW + (t % BW), oy = ty * TH + p_y * BH + (t / BW), on = n0 + p_n;
         ptab[i] = (on < P.n && oy < P.ho && ox < P.wo) ? (on * P.ho + oy) * P.wo + ox : -1;
     }
     __syncthreads();
@@ -241,24 +245,36 @@ patconv_kernel(const KParams P) {
         for (int c = 0; c < P.cols_per_warp; c += 8) tmem_st8(tmem_warp + c, z);
         tmem_wait_st();
     }
-    const uint32_t tmem_int = tmem_warp + (uint32_t)(P.J * kPixPerThread);   // i8: int32 totals
+    const uint32_t tmem_int = tmem_warp + (uint32_t)(P.J * T);   // i8 with folding: int32 totals
 
     // i8: fold the exact fp32 partial sums into the int32 totals and clear them
     auto fold_partial_sums = [&]() {
-        for (int j = 0; j < P.J; ++j) {
+        for (int c8 = 0; c8 < P.J * T; c8 += 8) {
             uint32_t f[8], q[8];
-            tmem_ld8(tmem_warp + j * 8, f);
-            tmem_ld8(tmem_int + j * 8, q);
+            tmem_ld8(tmem_warp + c8, f);
+            tmem_ld8(tmem_int + c8, q);
             tmem_wait_ld();
 #pragma unroll
             for (int i = 0; i < 8; ++i) { q[i] = (uint32_t)((int)q[i] + __float2int_rn(__uint_as_float(f[i]))); f[i] = 0u; }
-            tmem_st8(tmem_int + j * 8, q);
-            tmem_st8(tmem_warp + j * 8, f);
+            tmem_st8(tmem_int + c8, q);
+            tmem_st8(tmem_warp + c8, f);
+        }
+        tmem_wait_st();
+    };
+    // i8 without folding (few channels): the fp32 sums are exact integers; convert in place
+    auto sums_to_int = [&]() {
+        for (int c8 = 0; c8 < P.J * T; c8 += 8) {
+            uint32_t f[8];
+            tmem_ld8(tmem_warp + c8, f);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 8; ++i) f[i] = (uint32_t)__float2int_rn(__uint_as_float(f[i]));
+            tmem_st8(tmem_warp + c8, f);
         }
         tmem_wait_st();
     };
 
-    const uint32_t thr_off = (uint32_t)(l_n * P.img_stride + l_y * 4 * STRIDE * P.pitch + l_x * 2 * STRIDE) * 4u;
+    const uint32_t thr_off = (uint32_t)(l_n * P.img_stride + l_y * BH * STRIDE * P.pitch + l_x * BW * STRIDE) * 4u;
     const uint32_t plane_bytes = (uint32_t)P.plane_stride * 4u, pitch_bytes = (uint32_t)P.pitch * 4u;
 
     // --- main loop over channel chunks --------------------------------------------
@@ -302,10 +318,10 @@ patconv_kernel(const KParams P) {
         const int s0 = seg[c * (P.wpc + 1)], sg = seg[c * (P.wpc + 1) + warp];
         uint32_t sp = act + (uint32_t)P.act_stage_words * 4u + (uint32_t)(sg - s0) * 32u;
         run_commands<STRIDE, NP>(sp, tile_base + thr_off, plane_bytes, pitch_bytes, tmem_warp);
-        if (DT == XGEN_I8_I32 && ((c - c_begin + 1) % P.flush_chunks == 0)) fold_partial_sums();
+        if (DT == XGEN_I8_I32 && P.fold && ((c - c_begin + 1) % P.flush_chunks == 0)) fold_partial_sums();
     }
     cp_async_wait<0>();
-    if (DT == XGEN_I8_I32) fold_partial_sums();
+    if (DT == XGEN_I8_I32) { if (P.fold) fold_partial_sums(); else sums_to_int(); }
     __syncthreads();                           // staging memory is free: reuse it for the epilogue
 
     // --- epilogue: bias + ReLU + convert, NHWC rows through shared memory ----------
@@ -313,20 +329,29 @@ patconv_kernel(const KParams P) {
     const int oc_lo = b * ocb;
     const int nvalid = min(ocb, P.c_out - oc_lo);
     const int32_t *soc = P.slot_oc + ((size_t)(b * P.wpc + warp)) * P.J;
-    const uint32_t tmem_res = DT == XGEN_I8_I32 ? tmem_int : tmem_warp;
+    const uint32_t tmem_res = (DT == XGEN_I8_I32 && P.fold) ? tmem_int : tmem_warp;
     const int EP = P.epi_pix;
-    for (int t0 = 0; t0 < kPixPerThread; t0 += EP) {
+    for (int t0 = 0; t0 < T; t0 += EP) {
         for (int j = 0; j < P.J; ++j) {
             const int oc = soc[j];
-            uint32_t v[8];
-            if (EP == 8) { tmem_ld8(tmem_res + j * 8, v); }
-            else if (EP == 4) { uint32_t q[4]; tmem_ld4(tmem_res + j * 8 + t0, q); v[0] = q[0]; v[1] = q[1]; v[2] = q[2]; v[3] = q[3]; }
-            else { uint32_t q[2]; tmem_ld2(tmem_res + j * 8 + t0, q); v[0] = q[0]; v[1] = q[1]; }
+            uint32_t v[16];
+            if (EP >= 8) {
+                uint32_t q[8];
+                tmem_ld8(tmem_res + j * T + t0, q);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[i] = q[i];
+                if (EP == 16) {
+                    tmem_ld8(tmem_res + j * T + t0 + 8, q);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) v[8 + i] = q[i];
+                }
+            } else if (EP == 4) { uint32_t q[4]; tmem_ld4(tmem_res + j * T + t0, q); v[0] = q[0]; v[1] = q[1]; v[2] = q[2]; v[3] = q[3]; }
+            else { uint32_t q[2]; tmem_ld2(tmem_res + j * T + t0, q); v[0] = q[0]; v[1] = q[1]; }
             tmem_wait_ld();
             if (oc >= 0) {
                 uint32_t *dst = smem + lane * P.opitch + (oc - oc_lo);
 #pragma unroll
-                for (int tt = 0; tt < 8; ++tt)
+                for (int tt = 0; tt < 16; ++tt)
                     if (tt < EP) dst[tt * 32 * P.opitch] = v[tt];
             }
         }
@@ -452,26 +477,28 @@ patconv_reduce_kernel(const uint32_t *__restrict__ partial, int splits, size_t o
 // ---- host side ----------------------------------------------------------------------
 static std::atomic<int64_t> g_launches{0};
 
+static inline int pixels_per_thread_x(int stride) { return stride == 1 ? 4 : 2; }
+static inline int pixels_per_thread(int stride) { return 4 * pixels_per_thread_x(stride); }
+
 struct Geometry {
     int lx_log, ly_log, ln_log, tiles_x, tiles_y, tiles_n;
     int tin_w, tin_h, pitch, img_stride, plane_stride;
 };
 
-// Cost (shared-memory wavefronts) of one patch-row load for a candidate pitch.
+// Worst bank multiplicity of the 128-bit patch-row load for a candidate pitch.
 static int row_load_conflicts(int stride, int lx_log, int ly_log, int pitch, int img_stride) {
     const int LX = 1 << lx_log, LY = 1 << ly_log;
+    const int bw = pixels_per_thread_x(stride);
     auto addr = [&](int lane) {
         int x = lane & (LX - 1), y = (lane >> lx_log) & (LY - 1), n = lane >> (lx_log + ly_log);
-        return n * img_stride + y * 4 * stride * pitch + x * 2 * stride;   // words
+        return n * img_stride + y * 4 * stride * pitch + x * bw * stride;   // words
     };
     int worst = 0;
-    const int lanes_per_phase = stride == 1 ? 16 : 8;     // 64-bit / 128-bit accesses
-    const int words = stride == 1 ? 2 : 4;
-    for (int ph = 0; ph < 32 / lanes_per_phase; ++ph) {
+    for (int ph = 0; ph < 4; ++ph) {                      // 128-bit accesses: 8 lanes per wavefront
         int cnt[32] = {0};
-        for (int l = 0; l < lanes_per_phase; ++l) {
-            int a = addr(ph * lanes_per_phase + l);
-            for (int k = 0; k < words; ++k) cnt[(a + k) & 31]++;
+        for (int l = 0; l < 8; ++l) {
+            int a = addr(ph * 8 + l);
+            for (int k = 0; k < 4; ++k) cnt[(a + k) & 31]++;
         }
         for (int i = 0; i < 32; ++i) worst = worst > cnt[i] ? worst : cnt[i];
     }
@@ -481,23 +508,24 @@ static int row_load_conflicts(int stride, int lx_log, int ly_log, int pitch, int
 static Geometry choose_geometry(int n, int ho, int wo, int stride) {
     Geometry best{};
     double best_eff = -1.0;
+    const int bw = pixels_per_thread_x(stride), bh = 4;
     for (int lx_log = 5; lx_log >= 0; --lx_log)
         for (int ly_log = 5 - lx_log; ly_log >= 0; --ly_log) {
             const int ln_log = 5 - lx_log - ly_log;
-            const int TW = 2 << lx_log, TH = 4 << ly_log, LN = 1 << ln_log;
+            const int TW = bw << lx_log, TH = bh << ly_log, LN = 1 << ln_log;
             if (LN > 1 && (TW < wo || TH < ho)) continue;   // several images per tile only when one image fits
             const long tiles = (long)((wo + TW - 1) / TW) * ((ho + TH - 1) / TH) * ((n + LN - 1) / LN);
-            const double eff = (double)n * ho * wo / ((double)tiles * 256.0);
+            const double eff = (double)n * ho * wo / ((double)tiles * 32.0 * bw * bh);
             if (eff > best_eff + 1e-9) {
                 best_eff = eff;
                 best.lx_log = lx_log; best.ly_log = ly_log; best.ln_log = ln_log;
             }
         }
-    const int TW = 2 << best.lx_log, TH = 4 << best.ly_log, LN = 1 << best.ln_log;
+    const int TW = bw << best.lx_log, TH = bh << best.ly_log, LN = 1 << best.ln_log;
     best.tiles_x = (wo + TW - 1) / TW; best.tiles_y = (ho + TH - 1) / TH; best.tiles_n = (n + LN - 1) / LN;
     best.tin_w = stride == 1 ? TW + 2 : 2 * TW + 1;
     best.tin_h = stride == 1 ? TH + 2 : 2 * TH + 1;
-    const int align = stride == 1 ? 2 : 4;                // 8- or 16-byte aligned patch rows
+    const int align = 4;                                  // 16-byte aligned patch rows
     int p0 = (best.tin_w + align - 1) / align * align, best_p = p0, best_c = 1 << 30;
     for (int p = p0; p <= p0 + 8; p += align) {
         int c = row_load_conflicts(stride, best.lx_log, best.ly_log, p, best.tin_h * p);
@@ -611,6 +639,8 @@ xgen_status xgen_patconv_pack(const xgen_patconv_desc *desc, const void *dense_w
         if (const char *e = getenv("XGEN_PATCONV_J")) { int v = atoi(e); if (v == 4 || v == 8 || v == 16 || v == 32) {
             cfg.filters_per_group = v;
             int groups = (desc->c_out + v - 1) / v; cfg.groups_per_block = groups < kMaxWarps ? groups : kMaxWarps; } }
+        if (const char *e = getenv("XGEN_PATCONV_WPC")) { int v = atoi(e); if (v >= 1 && v <= kMaxWarps) {
+            int groups = (desc->c_out + cfg.filters_per_group - 1) / cfg.filters_per_group; cfg.groups_per_block = groups < v ? groups : v; } }
         if (const char *e = getenv("XGEN_PATCONV_CC")) { int v = atoi(e); if (v == 2 || v == 4 || v == 8 || v == 16) cfg.channels_per_chunk = v; }
         if (desc->dtype == XGEN_I8_I32 && cfg.channels_per_chunk < 4) cfg.channels_per_chunk = 4;
         st = pack_host(*desc, dense_w_host, pattern_id_host, cfg, h->host);
@@ -670,7 +700,8 @@ xgen_status xgen_patconv_plan(xgen_patconv_packed *h, int32_t n, int32_t hh, int
     if ((int64_t)n * ho * wo * p.c_out > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
     const Geometry g = choose_geometry(n, ho, wo, p.stride);
     const int64_t ctas = (int64_t)g.tiles_x * g.tiles_y * g.tiles_n * p.n_blocks;
-    const int cols_per_warp = p.J * kPixPerThread * (p.dtype == XGEN_I8_I32 ? 2 : 1);
+    const int flush_chunks_plan = 16777216 / (p.cc * 4 * 32640);
+    const int cols_per_warp = p.J * pixels_per_thread(p.stride) * ((p.dtype == XGEN_I8_I32 && p.n_chunks > flush_chunks_plan) ? 2 : 1);
     const int warp_slots = 4 * (512 / cols_per_warp);                 // per SM, set by tensor memory
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
@@ -747,11 +778,13 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_
     kp.vec_in = (p.c_in % E) == 0;
     kp.vec_out = (p.c_out % 4) == 0;
     const bool is_i8 = p.dtype == XGEN_I8_I32;
-    kp.cols_per_warp = p.J * kPixPerThread * (is_i8 ? 2 : 1);
-    kp.tmem_cols = next_pow2(((p.wpc + 3) / 4) * kp.cols_per_warp);
-    if (kp.tmem_cols > 512) return XGEN_ERR_UNSUPPORTED;
+    const int T = pixels_per_thread(p.stride);
     kp.flush_chunks = 16777216 / (p.cc * 4 * 32640);
     if (kp.flush_chunks < 1) return XGEN_ERR_UNSUPPORTED;
+    kp.fold = (is_i8 && p.n_chunks > kp.flush_chunks) ? 1 : 0;
+    kp.cols_per_warp = p.J * T * (kp.fold ? 2 : 1);
+    kp.tmem_cols = next_pow2(((p.wpc + 3) / 4) * kp.cols_per_warp);
+    if (kp.tmem_cols > 512) return XGEN_ERR_UNSUPPORTED;
     const int ocb = p.J * p.wpc;
     kp.opitch = ocb + 4;
     const int exp_words = p.dtype == XGEN_F32 ? 0 : p.cc * g.plane_stride;
@@ -762,7 +795,7 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_
         size_t w = (size_t)stages * kp.stage_words + exp_words;
         const size_t epi = (size_t)ep * 32 * kp.opitch;
         if (w < epi) w = epi;
-        return ((w + 1) & ~(size_t)1) + 2 * (size_t)npix_tile + 256;
+        return ((w + 1) & ~(size_t)1) + 2 * (size_t)npix_tile + 32 * (size_t)T;
     };
     auto occupancy = [&](size_t words) {
         int o = (int)((size_t)kSmemPerSM / (words * 4 + 1040));
@@ -774,11 +807,11 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_
     kp.exp_off_words = n_stages * kp.stage_words;
     // The epilogue tile reuses the staging memory: as many pixels per pass as fit for free.
     int ep = 2;
-    for (int cand = 8; cand > 2; cand >>= 1)
+    for (int cand = T; cand > 2; cand >>= 1)
         if (smem_words(n_stages, cand) * 4 <= (size_t)kSmemMaxDynamic && occupancy(smem_words(n_stages, cand)) >= occupancy(smem_words(n_stages, 2))) { ep = cand; break; }
     kp.epi_pix = ep;
     size_t words = smem_words(n_stages, ep);
-    kp.ptab_off_words = (int)(words - 256);
+    kp.ptab_off_words = (int)(words - 32 * T);
     kp.tab_off_words = kp.ptab_off_words - 2 * npix_tile;
     {
         const int segs = kp.vec_out ? (ocb >> 2) : ocb;

@@ -8,7 +8,9 @@
 namespace patconv {
 
 constexpr int kSlotWords = 8;   // one command slot = 32 bytes
-constexpr int kPixPerThread = 8;  // a thread owns a 2 (x) by 4 (y) block of output pixels
+// A thread owns a 4x4 block of output pixels at stride 1 and a 2x4 block at stride 2;
+// a filter's running sums take that many tensor-memory columns.
+constexpr int pix_per_thread(int stride) { return stride == 1 ? 16 : 8; }
 
 // The twelve tap sets of the built-in library (bit 3*dy+dx = tap kept): four 2x2
 // blocks holding the centre, four T shapes, four edge-plus-centre.  Layers whose

@@ -15,7 +15,7 @@ def _masked_dense(d):
     return np.where(sel, d.w.astype(np.float64), 0.0)
 
 
-def _walk(pk, c_in, c_out):
+def _walk(pk, c_in, c_out, stride=1):
     """Rebuild [c_out,c_in,9] from the stream; also return counters."""
     st, v = pk.stats(), pk.view()
     J, G, cc = st["filters_per_group"], st["groups_per_block"], st["channels_per_chunk"]
@@ -37,8 +37,9 @@ def _walk(pk, c_in, c_out):
                         loads += 1
                         last_key = None
                     else:
-                        assert op < npc and ic is not None and operand % 8 == 0
-                        j = operand // 8
+                        T = 16 if stride == 1 else 8
+                        assert op < npc and ic is not None and operand % T == 0
+                        j = operand // T
                         oc = int(v["slot_oc"][b, g, j])
                         assert 0 <= oc < c_out
                         key = (op, j)
@@ -52,13 +53,14 @@ def _walk(pk, c_in, c_out):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "f16", "i8"])
-@pytest.mark.parametrize("shape", [(5, 7), (16, 32), (40, 150), (3, 64)])
-def test_stream_rebuilds_masked_tensor(dtype, shape):
+@pytest.mark.parametrize("stride", [1, 2])
+@pytest.mark.parametrize("shape", [(5, 7), (16, 32), (40, 150), (3, 64), (300, 20)])
+def test_stream_rebuilds_masked_tensor(dtype, stride, shape):
     ci, co = shape
-    spec = wl.LayerSpec("t", 1, ci, co, 4, 4, 1, dtype, 0.45, 12, 0.5, "upm1", 0.1, True, 2)
+    spec = wl.LayerSpec("t", 1, ci, co, 4, 4, stride, dtype, 0.45, 12, 0.5, "upm1", 0.1, True, 2)
     d = wl.make_layer(spec, seed=9)
-    pk = binding.Packed(ci, co, 1, dtype, d.masks, d.w, d.pid, device=-1)
-    dense, seen, loads = _walk(pk, ci, co)
+    pk = binding.Packed(ci, co, stride, dtype, d.masks, d.w, d.pid, device=-1)
+    dense, seen, loads = _walk(pk, ci, co, stride)
     np.testing.assert_array_equal(dense.reshape(co, ci, 3, 3), _masked_dense(d))
     np.testing.assert_array_equal(seen, (d.pid >= 0).astype(int))          # each survivor exactly once
     st = pk.stats()
