@@ -31,7 +31,7 @@
 namespace patconv {
 
 constexpr int kSmemPerSM = 233472;     // 228 KB
-constexpr int kSmemMaxDynamic = 232448 - 1024;  // 227 KB per block less static shared memory
+constexpr int kSmemMaxDynamic = 232448 - 2048;  // 227 KB per block less static shared memory
 constexpr int kMaxWarps = 16;
 
 struct KParams {
@@ -135,6 +135,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32)
 patconv_kernel(const KParams P) {
     extern __shared__ __align__(16) uint32_t smem[];
     __shared__ uint32_t tmem_base_s;
+    __shared__ int soc_s[kMaxWarps * 16];           // original output channel of every filter slot of this block
     constexpr int E = DTraits<DT>::E;
     constexpr int XB = DTraits<DT>::xbytes;
     constexpr int BW = STRIDE == 1 ? 4 : 2, BH = 4;   // output pixels per thread: BW x BH
@@ -179,6 +180,7 @@ patconv_kernel(const KParams P) {
         tab[q] = make_int2(ok ? ((gn * P.h + gy) * P.w + gx) * P.c_in : -1,
                            im * P.img_stride + row * P.pitch + col);
     }
+    for (int i = tid; i < P.wpc * P.J; i += nthreads) soc_s[i] = P.slot_oc[(size_t)blockIdx.y * P.wpc * P.J + i];
     // Output-pixel table: linear pixel index of (pixel t of lane l), or -1 outside the output.
     int *ptab = reinterpret_cast<int *>(smem + P.ptab_off_words);
     for (int i = tid; i < 32 * T; i += nthreads) {
@@ -201,16 +203,24 @@ patconv_kernel(const KParams P) {
             const int ic = c * P.cc + rp * E;
             const bool ic_ok = ic < P.c_in;
             const uint32_t plane = act + (uint32_t)(rp * P.plane_stride) * 4u;
-            const char *xc = (const char *)P.x + (size_t)ic * XB;
-            for (int q = q0; q < npix; q += pix_step) {
-                const int2 t = tab[q];
-                const bool ok = ic_ok && t.x >= 0;
-                const uint32_t dst = plane + (uint32_t)t.y * 4u;
-                const char *src = xc + (size_t)(ok ? t.x : 0) * XB;
-                if (E == 1 || P.vec_in) {
-                    cp_async4(dst, ok ? src : (const char *)P.x, ok ? 4 : 0);
-                } else {
-                    // channel count not a multiple of E: assemble the word element by element
+            const char *xc = (const char *)P.x + (size_t)(ic_ok ? ic : 0) * XB;
+            if (E == 1 || P.vec_in) {
+                auto copy1 = [&](const int2 t) {
+                    const bool ok = ic_ok && t.x >= 0;
+                    cp_async4(plane + (uint32_t)t.y * 4u, xc + (size_t)(ok ? t.x : 0) * XB, ok ? 4 : 0);
+                };
+                int q = q0;
+                for (; q + 3 * pix_step < npix; q += 4 * pix_step) {      // four independent copies in flight
+                    const int2 t0 = tab[q], t1 = tab[q + pix_step], t2 = tab[q + 2 * pix_step], t3 = tab[q + 3 * pix_step];
+                    copy1(t0); copy1(t1); copy1(t2); copy1(t3);
+                }
+                for (; q < npix; q += pix_step) copy1(tab[q]);
+            } else {
+                // channel count not a multiple of E: assemble the word element by element
+                for (int q = q0; q < npix; q += pix_step) {
+                    const int2 t = tab[q];
+                    const bool ok = ic_ok && t.x >= 0;
+                    const char *src = xc + (size_t)(ok ? t.x : 0) * XB;
                     uint32_t word = 0;
                     if (ok) {
                         for (int k = 0; k < E; ++k) {
@@ -220,7 +230,7 @@ patconv_kernel(const KParams P) {
                             }
                         }
                     }
-                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst), "r"(word) : "memory");
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(plane + (uint32_t)t.y * 4u), "r"(word) : "memory");
                 }
             }
             // this block's commands for the chunk: one contiguous segment
@@ -328,7 +338,7 @@ patconv_kernel(const KParams P) {
     const int ocb = P.J * P.wpc;
     const int oc_lo = b * ocb;
     const int nvalid = min(ocb, P.c_out - oc_lo);
-    const int32_t *soc = P.slot_oc + ((size_t)(b * P.wpc + warp)) * P.J;
+    const int *soc = soc_s + warp * P.J;
     const uint32_t tmem_res = (DT == XGEN_I8_I32 && P.fold) ? tmem_int : tmem_warp;
     const int EP = P.epi_pix;
     for (int t0 = 0; t0 < T; t0 += EP) {
@@ -358,6 +368,58 @@ patconv_kernel(const KParams P) {
         __syncthreads();
         // cooperative store: EP*32 pixels x nvalid channels
         const int segs = P.vec_out ? (nvalid >> 2) : nvalid;
+        if (P.vec_out && segs > 0 && (nthreads % segs) == 0) {
+            // every thread keeps one 4-channel column: bias and offsets are loop-invariant
+            const int sgm = tid % segs, dpl = nthreads / segs;
+            const int ocl = sgm * 4;
+            uint4 bb = make_uint4(0u, 0u, 0u, 0u);
+            if (P.bias && !P.partial) bb = *reinterpret_cast<const uint4 *>((const uint32_t *)P.bias + oc_lo + ocl);
+            const int *pt = ptab + t0 * 32;
+            const uint32_t *srow = smem + ocl;
+            const size_t col = (size_t)oc_lo + ocl;
+            uint32_t *part = P.partial ? P.partial + (size_t)blockIdx.z * P.out_elems + col : nullptr;
+            auto emit = [&](const int pidx, const uint4 raw) {
+                const size_t o = (size_t)pidx * P.c_out;
+                if (part) { *reinterpret_cast<uint4 *>(part + o) = raw; return; }
+                if (DT == XGEN_I8_I32) {
+                    int4 r = make_int4((int)raw.x + (int)bb.x, (int)raw.y + (int)bb.y, (int)raw.z + (int)bb.z, (int)raw.w + (int)bb.w);
+                    if (P.relu) { r.x = max(r.x, 0); r.y = max(r.y, 0); r.z = max(r.z, 0); r.w = max(r.w, 0); }
+                    *reinterpret_cast<int4 *>((int *)P.y + o + col) = r;
+                } else {
+                    float4 r = make_float4(__uint_as_float(raw.x) + __uint_as_float(bb.x), __uint_as_float(raw.y) + __uint_as_float(bb.y),
+                                           __uint_as_float(raw.z) + __uint_as_float(bb.z), __uint_as_float(raw.w) + __uint_as_float(bb.w));
+                    if (P.relu) { r.x = fmaxf(r.x, 0.f); r.y = fmaxf(r.y, 0.f); r.z = fmaxf(r.z, 0.f); r.w = fmaxf(r.w, 0.f); }
+                    if (DT == XGEN_F32) {
+                        *reinterpret_cast<float4 *>((float *)P.y + o + col) = r;
+                    } else {
+                        __half2 lo = __floats2half2_rn(r.x, r.y), hi = __floats2half2_rn(r.z, r.w);
+                        uint2 pk;
+                        pk.x = *reinterpret_cast<uint32_t *>(&lo);
+                        pk.y = *reinterpret_cast<uint32_t *>(&hi);
+                        *reinterpret_cast<uint2 *>((__half *)P.y + o + col) = pk;
+                    }
+                }
+            };
+            const int npl = EP * 32;
+            int pl = tid / segs;
+            for (; pl + 3 * dpl < npl; pl += 4 * dpl) {           // four rows in flight
+                const int i0 = pt[pl], i1 = pt[pl + dpl], i2 = pt[pl + 2 * dpl], i3 = pt[pl + 3 * dpl];
+                const uint4 r0 = *reinterpret_cast<const uint4 *>(srow + pl * P.opitch);
+                const uint4 r1 = *reinterpret_cast<const uint4 *>(srow + (pl + dpl) * P.opitch);
+                const uint4 r2 = *reinterpret_cast<const uint4 *>(srow + (pl + 2 * dpl) * P.opitch);
+                const uint4 r3 = *reinterpret_cast<const uint4 *>(srow + (pl + 3 * dpl) * P.opitch);
+                if (i0 >= 0) emit(i0, r0);
+                if (i1 >= 0) emit(i1, r1);
+                if (i2 >= 0) emit(i2, r2);
+                if (i3 >= 0) emit(i3, r3);
+            }
+            for (; pl < npl; pl += dpl) {
+                const int i0 = pt[pl];
+                if (i0 >= 0) emit(i0, *reinterpret_cast<const uint4 *>(srow + pl * P.opitch));
+            }
+            __syncthreads();
+            continue;
+        }
         const int total = EP * 32 * segs;
         for (int i = tid; i < total; i += nthreads) {
             int pl, sgm;                                      // pl = tt*32 + lane'
@@ -798,7 +860,7 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_
         return ((w + 1) & ~(size_t)1) + 2 * (size_t)npix_tile + 32 * (size_t)T;
     };
     auto occupancy = [&](size_t words) {
-        int o = (int)((size_t)kSmemPerSM / (words * 4 + 1040));
+        int o = (int)((size_t)kSmemPerSM / (words * 4 + 2112));     // + static and per-block reserved shared memory
         return o < max_ctas ? o : max_ctas;
     };
     int n_stages = 3;
