@@ -149,6 +149,40 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *packed, const void *x_de
                              void *y_dev, void *cuda_stream);
 
 /*
+ * (The paper has no counterpart to this entry point; it exists for callers of this
+ * library.)  Run the layer with its input channels split over `splits` groups of thread
+ * blocks, like a shape prepared with xgen_patconv_plan, but keep the partial sums in a
+ * fixed array inside the library instead of a workspace from cudaMalloc.  It is meant for
+ * callers that must not allocate device memory where they call us: code running under a
+ * memory budget that was handed out up front, inside another framework's allocator
+ * scope, or on a path where an allocation (which may synchronise the device) is not
+ * allowed.  Neither this call nor anything it uses allocates or frees device memory.
+ *
+ *   splits   how many ways to split the channel chunks (>= 1; clamped to the number of
+ *            chunks); more splits put more thread blocks to work on layers with few
+ *            output pixels, and cost splits x 4 bytes of scratch per output element
+ *   others   exactly as xgen_patconv_run; the caller still owns x, bias and y
+ *
+ * Limit: splits x n*ho*wo*c_out x 4 bytes must not exceed
+ * XGEN_PATCONV_STATIC_SCRATCH_BYTES; beyond that the call returns XGEN_ERR_SHAPE and
+ * launches nothing (with XGEN_PATCONV_LOG set, the reason goes to stderr).  The array is
+ * part of the loaded library: every GPU that uses the library holds those bytes until
+ * the process exits.
+ * The first call on a device looks up the array's device address (once per device, with
+ * that device made current); make that first call outside any stream capture.
+ * All calls share the one array and nothing in it has to start at zero: every element a
+ * call reads it has written itself.  For the same reason two calls whose kernels may
+ * overlap on the GPU (different streams, no dependency between them) race on it; put
+ * such calls on one stream or order them with events.
+ * Errors: INVALID_ARG, SHAPE, CUDA, as xgen_patconv_run, plus SHAPE for the limit.
+ */
+#define XGEN_PATCONV_STATIC_SCRATCH_BYTES (8u << 20)
+xgen_status xgen_patconv_run_static_scratch(const xgen_patconv_packed *packed, const void *x_dev,
+                                            int32_t n, int32_t h, int32_t w, const void *bias_dev,
+                                            int32_t relu, void *y_dev, int32_t splits,
+                                            void *cuda_stream);
+
+/*
  * Convenience for callers that hold host tensors: copies x (and bias) to the
  * device, runs the layer, copies y back and waits.  Allocates and frees device
  * buffers on every call.  Same tensor layouts as xgen_patconv_run, all

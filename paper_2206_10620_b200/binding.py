@@ -17,10 +17,12 @@ from . import build as _build
 F32, F16_F32ACC, I8_I32 = 0, 1, 2
 DTYPES = {"f32": F32, "f16": F16_F32ACC, "i8": I8_I32}
 OK = 0
+STATIC_SCRATCH_BYTES = 8 << 20
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_PATTERN", 3: "SHAPE", 4: "UNSUPPORTED",
                 5: "ALLOC", 6: "CUDA", 7: "TIMEOUT"}
 
-EXPORTS = ["xgen_patconv_pack", "xgen_patconv_run", "xgen_patconv_run_host", "xgen_patconv_plan",
+EXPORTS = ["xgen_patconv_pack", "xgen_patconv_run", "xgen_patconv_run_static_scratch",
+           "xgen_patconv_run_host", "xgen_patconv_plan",
            "xgen_patconv_out_shape", "xgen_patconv_query", "xgen_patconv_view",
            "xgen_patconv_last_status", "xgen_patconv_free", "xgen_strerror",
            "xgen_patconv_launch_count"]
@@ -70,6 +72,7 @@ def lib():
         P, I = ctypes.c_void_p, ctypes.c_int32
         L.xgen_patconv_pack.argtypes = [ctypes.POINTER(Desc), P, P, ctypes.c_int, ctypes.POINTER(P)]
         L.xgen_patconv_run.argtypes = [P, P, I, I, I, P, I, P, P]
+        L.xgen_patconv_run_static_scratch.argtypes = [P, P, I, I, I, P, I, P, I, P]
         L.xgen_patconv_run_host.argtypes = [P, P, I, I, I, P, I, P]
         L.xgen_patconv_plan.argtypes = [P, I, I, I]
         L.xgen_patconv_out_shape.argtypes = [P, I, I, ctypes.POINTER(I), ctypes.POINTER(I)]
@@ -159,6 +162,14 @@ class Packed:
         """Enqueue the layer; all pointers are device addresses (ints)."""
         _check(lib().xgen_patconv_run(self._h, x_ptr, n, h, w, bias_ptr or None, int(bool(relu)),
                                       y_ptr, stream or None), "xgen_patconv_run")
+
+    def run_static_scratch(self, x_ptr, n, h, w, bias_ptr, relu, y_ptr, splits, stream=0):
+        """Like run(), with the channel chunks split `splits` ways and the partial sums kept
+        in the library's built-in scratch array: no device memory is allocated.  For callers
+        that may not allocate where they call; see the header for the size limit."""
+        _check(lib().xgen_patconv_run_static_scratch(self._h, x_ptr, n, h, w, bias_ptr or None,
+                                                     int(bool(relu)), y_ptr, int(splits), stream or None),
+               "xgen_patconv_run_static_scratch")
 
     def run_host(self, x: np.ndarray, bias, relu) -> np.ndarray:
         """Host tensors in, host tensor out (copies inside the library)."""

@@ -805,8 +805,13 @@ xgen_status xgen_patconv_last_status(const xgen_patconv_packed *h, void *stream)
     return cudaGetLastError() == cudaSuccess ? XGEN_OK : XGEN_ERR_CUDA;
 }
 
-xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
-                             const void *bias, int32_t relu, void *y, void *stream) {
+}  // extern "C"
+
+// Where a run keeps the partial sums of a split, when the caller (not the plan) decides.
+struct SplitChoice { int splits, chunks_per_split; uint32_t *partial; };
+
+static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
+                             const void *bias, int32_t relu, void *y, void *stream, const SplitChoice *forced) {
     if (!h || !x || !y) return XGEN_ERR_INVALID_ARG;
     if (((uintptr_t)x & 15) || ((uintptr_t)y & 15) || ((uintptr_t)bias & 15)) return XGEN_ERR_INVALID_ARG;
     if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
@@ -881,10 +886,13 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_
         for (int l = 0; l < 12; ++l) if ((1 << l) == segs) kp.segs_log = l;
     }
     size_t smem = words * 4;
-    const bool split = h->plan_splits > 1 && h->plan_n == n && h->plan_h == hh && h->plan_w == ww && h->d_partial;
+    const bool split = forced ? forced->splits > 1
+                              : (h->plan_splits > 1 && h->plan_n == n && h->plan_h == hh && h->plan_w == ww && h->d_partial);
+    const int n_splits = forced ? forced->splits : h->plan_splits;
+    uint32_t *const partial = forced ? forced->partial : h->d_partial;
     kp.out_elems = (size_t)n * ho * wo * p.c_out;
-    kp.chunks_per_split = split ? h->plan_cps : 0;
-    kp.partial = split ? h->d_partial : nullptr;
+    kp.chunks_per_split = split ? (forced ? forced->chunks_per_split : h->plan_cps) : 0;
+    kp.partial = split ? partial : nullptr;
     // Never let more blocks share an SM than tensor memory has columns for.
     const size_t floor_bytes = (size_t)kSmemPerSM / (max_ctas + 1);
     if (smem < floor_bytes) smem = floor_bytes;
@@ -893,7 +901,7 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_
     int prev = 0;
     if (cudaGetDevice(&prev) != cudaSuccess) return XGEN_ERR_CUDA;
     if (prev != h->device && cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
-    dim3 grid((unsigned)(g.tiles_x * g.tiles_y * g.tiles_n), (unsigned)p.n_blocks, (unsigned)(split ? h->plan_splits : 1)), block((unsigned)(p.wpc * 32), 1, 1);
+    dim3 grid((unsigned)(g.tiles_x * g.tiles_y * g.tiles_n), (unsigned)p.n_blocks, (unsigned)(split ? n_splits : 1)), block((unsigned)(p.wpc * 32), 1, 1);
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e;
     if (p.dtype == XGEN_F32)
@@ -907,11 +915,11 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_
         const size_t items = vec ? kp.out_elems / 4 : kp.out_elems;
         const unsigned blocks = (unsigned)((items + 255) / 256);
         if (p.dtype == XGEN_F32)
-            patconv_reduce_kernel<XGEN_F32><<<blocks, 256, 0, st>>>(h->d_partial, h->plan_splits, kp.out_elems, p.c_out, bias, kp.relu, y, vec);
+            patconv_reduce_kernel<XGEN_F32><<<blocks, 256, 0, st>>>(partial, n_splits, kp.out_elems, p.c_out, bias, kp.relu, y, vec);
         else if (p.dtype == XGEN_F16_F32ACC)
-            patconv_reduce_kernel<XGEN_F16_F32ACC><<<blocks, 256, 0, st>>>(h->d_partial, h->plan_splits, kp.out_elems, p.c_out, bias, kp.relu, y, vec);
+            patconv_reduce_kernel<XGEN_F16_F32ACC><<<blocks, 256, 0, st>>>(partial, n_splits, kp.out_elems, p.c_out, bias, kp.relu, y, vec);
         else
-            patconv_reduce_kernel<XGEN_I8_I32><<<blocks, 256, 0, st>>>(h->d_partial, h->plan_splits, kp.out_elems, p.c_out, bias, kp.relu, y, vec);
+            patconv_reduce_kernel<XGEN_I8_I32><<<blocks, 256, 0, st>>>(partial, n_splits, kp.out_elems, p.c_out, bias, kp.relu, y, vec);
         e = log_cuda(cudaGetLastError(), "reduce launch");
         if (e == cudaSuccess) g_launches.fetch_add(1);
     }
@@ -919,6 +927,60 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_
     if (e != cudaSuccess) return XGEN_ERR_CUDA;
     g_launches.fetch_add(1);
     return XGEN_OK;
+}
+
+
+// The library's own scratch for xgen_patconv_run_static_scratch: partial sums of a split run.
+// It lives in every CUDA context that loads this library, until the process exits.
+static __device__ __align__(256) uint32_t g_static_scratch[XGEN_PATCONV_STATIC_SCRATCH_BYTES / 4];
+static uint32_t *g_static_scratch_addr[64];        // device address per device ordinal, resolved once
+static std::mutex g_static_scratch_mutex;
+
+extern "C" {
+
+xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
+                             const void *bias, int32_t relu, void *y, void *stream) {
+    return run_layer(h, x, n, hh, ww, bias, relu, y, stream, nullptr);
+}
+
+xgen_status xgen_patconv_run_static_scratch(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh,
+                                            int32_t ww, const void *bias, int32_t relu, void *y,
+                                            int32_t splits, void *stream) {
+    if (!h || !x || !y || splits < 1) return XGEN_ERR_INVALID_ARG;
+    if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
+    if (h->device < 0 || h->device >= 64) return XGEN_ERR_CUDA;
+    const PackedHost &p = h->host;
+    const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
+    const int64_t out_elems = (int64_t)n * ho * wo * p.c_out;
+    if (out_elems > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
+    if (splits > p.n_chunks) splits = p.n_chunks;
+    const int cps = (p.n_chunks + splits - 1) / splits;
+    const int eff = (p.n_chunks + cps - 1) / cps;                 // splits that actually get chunks
+    if (eff > 1 && (uint64_t)out_elems * 4u * (uint64_t)eff > (uint64_t)XGEN_PATCONV_STATIC_SCRATCH_BYTES) {
+        if (getenv("XGEN_PATCONV_LOG"))
+            fprintf(stderr, "libpatconv: %d splits x %lld outputs x 4 bytes exceed the %u-byte static scratch\n",
+                    eff, (long long)out_elems, (unsigned)XGEN_PATCONV_STATIC_SCRATCH_BYTES);
+        return XGEN_ERR_SHAPE;
+    }
+    uint32_t *scratch = nullptr;
+    {
+        // First call on a device: resolve the device address of the array (in host code the
+        // array's name is only a handle, not an address a kernel can use).
+        std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+        scratch = g_static_scratch_addr[h->device];
+        if (!scratch) {
+            int prev = 0;
+            if (cudaGetDevice(&prev) != cudaSuccess) return XGEN_ERR_CUDA;
+            if (prev != h->device && cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
+            void *addr = nullptr;
+            const cudaError_t e = cudaGetSymbolAddress(&addr, g_static_scratch);
+            if (prev != h->device) cudaSetDevice(prev);
+            if (log_cuda(e, "cudaGetSymbolAddress") != cudaSuccess || !addr) return XGEN_ERR_CUDA;
+            scratch = g_static_scratch_addr[h->device] = static_cast<uint32_t *>(addr);
+        }
+    }
+    const SplitChoice choice{eff, cps, scratch};
+    return run_layer(h, x, n, hh, ww, bias, relu, y, stream, &choice);
 }
 
 xgen_status xgen_patconv_run_host(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
