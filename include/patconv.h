@@ -78,7 +78,8 @@ typedef struct {
     int32_t max_segment_slots;    /* longest per-(block, chunk) command segment               */
     int64_t load_commands;        /* activation-patch loads in the stream (one per group and
                                      input channel that group is connected to)                */
-    double  group_imbalance;      /* max over groups / mean over groups of surviving kernels  */
+    double  group_imbalance;      /* worst thread block: max / mean of surviving kernels over
+                                     the block's groups (its warps wait for each other)       */
 } xgen_patconv_stats;
 
 /* Read-only view of the packed layout on the host, for inspection and tests.

@@ -2,8 +2,8 @@
 // compact command-stream layout (paper Sec. 2.3, "Filter Kernel Reorder and
 // Compact FKW Storage").  Pure C++, no CUDA.
 //
-// Layout idea.  A warp owns one *filter group* (J filters) for a tile of output
-// pixels; each thread keeps J x 8 running sums (in tensor memory).  For every
+// Layout idea.  A warp owns one *filter group* (J consecutive output channels) for a
+// tile of output pixels; each thread keeps J x 8 running sums (in tensor memory).  For every
 // input channel the group is connected to, the warp loads the activation patch
 // of its pixels once into registers (a LOAD command) and then executes one
 // *kernel command* per surviving kernel of that channel: the command names the
@@ -154,8 +154,7 @@ xgen_status build_layout(PackedHost &out, const PackConfig &cfg) {
     const int J = cfg.filters_per_group, cc = cfg.channels_per_chunk;
     const int wpc = cfg.groups_per_block;
     if (J < 1 || wpc < 1 || cc < 1 || (cc & (cc - 1))) return XGEN_ERR_INVALID_ARG;
-    const int ocb = J * wpc;  // output channels per thread block (contiguous originals)
-    const int n_blocks = (cout + ocb - 1) / ocb;
+    const int n_blocks = ((cout + J - 1) / J + wpc - 1) / wpc;
     const int n_groups = n_blocks * wpc;
     const int n_chunks = (cin + cc - 1) / cc;
 
@@ -164,36 +163,35 @@ xgen_status build_layout(PackedHost &out, const PackConfig &cfg) {
     out.n_blocks = n_blocks; out.n_chunks = n_chunks;
     out.slot_oc.assign((size_t)n_groups * J, -1);
 
-    // --- a2: filter reorder.  Inside each block of `ocb` contiguous output
-    // channels, sort filters by (surviving kernels desc, pattern histogram,
-    // index) so that similar filters are neighbours, then deal them to the
-    // block's groups in serpentine order: the groups (= warps that meet at a
-    // barrier once per channel chunk) get near-equal kernel counts.
-    std::vector<int> cnt(cout, 0);
-    std::vector<std::vector<int>> hist(cout, std::vector<int>(np, 0));
+    // --- a2: filter reorder.  A filter group is a run of J consecutive output
+    // channels (so a thread can store a pixel's J results as one contiguous piece);
+    // what is reordered is which groups share a thread block.  Groups are sorted by
+    // (surviving kernels desc, pattern histogram, index) and taken wpc at a time: the
+    // warps of a block, which meet at a barrier once per channel chunk, then carry
+    // similar numbers of kernels.
+    const int n_runs = (cout + J - 1) / J;
+    std::vector<int> cnt(n_runs, 0);
+    std::vector<std::vector<int>> hist(n_runs, std::vector<int>(np, 0));
     for (int oc = 0; oc < cout; ++oc)
         for (int ic = 0; ic < cin; ++ic) {
             int p = pid[(size_t)oc * cin + ic];
-            if (p >= 0) { ++cnt[oc]; ++hist[oc][p]; }
+            if (p >= 0) { ++cnt[oc / J]; ++hist[oc / J][p]; }
         }
+    std::vector<int> order(n_runs);
+    std::iota(order.begin(), order.end(), 0);
+    std::sort(order.begin(), order.end(), [&](int a, int c) {
+        if (cnt[a] != cnt[c]) return cnt[a] > cnt[c];
+        if (hist[a] != hist[c]) return hist[a] > hist[c];
+        return a < c;
+    });
     std::vector<int64_t> group_kernels(n_groups, 0);
-    for (int b = 0; b < n_blocks; ++b) {
-        int lo = b * ocb, hi = std::min(cout, lo + ocb);
-        std::vector<int> order(hi - lo);
-        std::iota(order.begin(), order.end(), lo);
-        std::sort(order.begin(), order.end(), [&](int a, int c) {
-            if (cnt[a] != cnt[c]) return cnt[a] > cnt[c];
-            if (hist[a] != hist[c]) return hist[a] > hist[c];
-            return a < c;
-        });
-        std::vector<int> fill(wpc, 0);
-        for (size_t i = 0; i < order.size(); ++i) {
-            int round = (int)(i / wpc), pos = (int)(i % wpc);
-            int g = (round & 1) ? (wpc - 1 - pos) : pos;
-            out.slot_oc[((size_t)(b * wpc + g)) * J + fill[g]] = order[i];
-            group_kernels[b * wpc + g] += cnt[order[i]];
-            ++fill[g];
+    for (int i = 0; i < n_runs; ++i) {
+        const int g = i;                                   // block i / wpc, warp i % wpc
+        for (int j = 0; j < J; ++j) {
+            const int oc = order[i] * J + j;
+            out.slot_oc[(size_t)g * J + j] = oc < cout ? oc : -1;
         }
+        group_kernels[g] = cnt[order[i]];
     }
 
     // --- a3: kernel reorder + compact store.  Per group and channel: one LOAD,
@@ -255,9 +253,14 @@ xgen_status build_layout(PackedHost &out, const PackConfig &cfg) {
     s.channels_per_chunk = cc; s.n_chunks = n_chunks; s.patterns_compiled = np;
     s.max_segment_slots = out.max_seg_slots;
     s.load_commands = n_loads;
-    int64_t mx = 0, sum = 0;
-    for (int64_t v : group_kernels) { mx = std::max(mx, v); sum += v; }
-    s.group_imbalance = sum > 0 ? (double)mx * n_groups / (double)sum : 1.0;
+    // Warps of one block wait for each other: what matters is the spread inside a block.
+    double worst = 1.0;
+    for (int b = 0; b < n_blocks; ++b) {
+        int64_t mx = 0, sum = 0, n = 0;
+        for (int g = b * wpc; g < (b + 1) * wpc && g < n_runs; ++g) { mx = std::max(mx, group_kernels[g]); sum += group_kernels[g]; ++n; }
+        if (sum > 0) worst = std::max(worst, (double)mx * (double)n / (double)sum);
+    }
+    s.group_imbalance = worst;
     return XGEN_OK;
 }
 

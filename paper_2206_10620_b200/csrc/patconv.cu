@@ -12,8 +12,9 @@
 // surviving kernel of the group on that channel reuses it (the paper's load
 // redundancy elimination, Sec. 2.3); the running sums live in tensor memory,
 // addressed by filter slot.  The epilogue adds bias, applies ReLU, converts and
-// writes NHWC rows through a shared-memory transpose so stores are 16 bytes
-// wide and contiguous per pixel (operator fusion, Sec. 2.2).
+// stores straight from tensor memory: a group is a run of consecutive output
+// channels, so a thread writes 32 contiguous bytes per pixel (operator fusion,
+// Sec. 2.2).
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
@@ -51,13 +52,10 @@ struct KParams {
     int tmem_cols, cols_per_warp;
     int flush_chunks;                    // i8: chunks between folds of the fp32 partial sums
     int vec_in;                          // c_in is a multiple of the channels per staged word
-    int vec_out;                         // c_out allows 4-channel vector stores
-    int opitch;                          // words per pixel row of the epilogue tile
+    int vec_out;                         // widest aligned store of an 8-channel piece: 8 or 4 words, 0 = scalar
     int tab_off_words;                   // offset of the per-pixel staging table in shared memory
     int ptab_off_words;                  // offset of the output-pixel table (32 lanes x pixels per thread)
-    int epi_pix;                         // pixels per thread handled in one epilogue pass (2, 4, 8 or 16)
     int fold;                            // i8: keep int32 totals in a second row and fold periodically
-    int segs_log;                        // log2 of the 16-byte segments per pixel row, or -1
     int chunks_per_split;                // grid.z splits the channel chunks; 0 = no split
     uint32_t *partial;                   // split runs: [split][n*ho*wo*c_out] raw fp32 / int32 sums
     size_t out_elems;                    // n*ho*wo*c_out
@@ -332,154 +330,78 @@ patconv_kernel(const KParams P) {
     }
     cp_async_wait<0>();
     if (DT == XGEN_I8_I32) { if (P.fold) fold_partial_sums(); else sums_to_int(); }
-    __syncthreads();                           // staging memory is free: reuse it for the epilogue
 
-    // --- epilogue: bias + ReLU + convert, NHWC rows through shared memory ----------
-    const int ocb = P.J * P.wpc;
-    const int oc_lo = b * ocb;
-    const int nvalid = min(ocb, P.c_out - oc_lo);
+    // --- epilogue: bias + ReLU + convert, straight from tensor memory to NHWC -------
+    // A group is a run of J consecutive output channels, so for one pixel a thread holds
+    // 8 adjacent channels per 8 filter slots: 32 bytes (16 for fp16) it can store as one
+    // piece.  No shared memory, no block-wide barrier: every warp drains on its own.
     const int *soc = soc_s + warp * P.J;
     const uint32_t tmem_res = (DT == XGEN_I8_I32 && P.fold) ? tmem_int : tmem_warp;
-    const int EP = P.epi_pix;
-    for (int t0 = 0; t0 < T; t0 += EP) {
-        for (int j = 0; j < P.J; ++j) {
-            const int oc = soc[j];
-            uint32_t v[16];
-            if (EP >= 8) {
-                uint32_t q[8];
-                tmem_ld8(tmem_res + j * T + t0, q);
+    const int oc_base = soc[0];
+    if (oc_base >= 0) {
+        const int *pt = ptab + lane;
+        uint32_t *const part = P.partial ? P.partial + (size_t)blockIdx.z * P.out_elems : nullptr;
+        for (int j0 = 0; j0 < P.J; j0 += 8) {
+            const int oc0 = oc_base + j0;
+            if (oc0 >= P.c_out) break;
+            const int nv = min(8, P.c_out - oc0);                 // valid channels of this piece
+            uint32_t bb[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) v[i] = q[i];
-                if (EP == 16) {
-                    tmem_ld8(tmem_res + j * T + t0 + 8, q);
+            for (int k = 0; k < 8; ++k) bb[k] = (P.bias && !part && k < nv) ? ((const uint32_t *)P.bias)[oc0 + k] : 0u;
+            for (int t0 = 0; t0 < T; t0 += 4) {
+                uint32_t v[8][4];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) v[8 + i] = q[i];
+                for (int k = 0; k < 8; ++k) {
+                    if (j0 + k < P.J) tmem_ld4(tmem_res + (j0 + k) * T + t0, v[k]);
+                    else { v[k][0] = v[k][1] = v[k][2] = v[k][3] = 0u; }
                 }
-            } else if (EP == 4) { uint32_t q[4]; tmem_ld4(tmem_res + j * T + t0, q); v[0] = q[0]; v[1] = q[1]; v[2] = q[2]; v[3] = q[3]; }
-            else { uint32_t q[2]; tmem_ld2(tmem_res + j * T + t0, q); v[0] = q[0]; v[1] = q[1]; }
-            tmem_wait_ld();
-            if (oc >= 0) {
-                uint32_t *dst = smem + lane * P.opitch + (oc - oc_lo);
+                tmem_wait_ld();
 #pragma unroll
-                for (int tt = 0; tt < 16; ++tt)
-                    if (tt < EP) dst[tt * 32 * P.opitch] = v[tt];
-            }
-        }
-        __syncthreads();
-        // cooperative store: EP*32 pixels x nvalid channels
-        const int segs = P.vec_out ? (nvalid >> 2) : nvalid;
-        if (P.vec_out && segs > 0 && (nthreads % segs) == 0) {
-            // every thread keeps one 4-channel column: bias and offsets are loop-invariant
-            const int sgm = tid % segs, dpl = nthreads / segs;
-            const int ocl = sgm * 4;
-            uint4 bb = make_uint4(0u, 0u, 0u, 0u);
-            if (P.bias && !P.partial) bb = *reinterpret_cast<const uint4 *>((const uint32_t *)P.bias + oc_lo + ocl);
-            const int *pt = ptab + t0 * 32;
-            const uint32_t *srow = smem + ocl;
-            const size_t col = (size_t)oc_lo + ocl;
-            uint32_t *part = P.partial ? P.partial + (size_t)blockIdx.z * P.out_elems + col : nullptr;
-            auto emit = [&](const int pidx, const uint4 raw) {
-                const size_t o = (size_t)pidx * P.c_out;
-                if (part) { *reinterpret_cast<uint4 *>(part + o) = raw; return; }
-                if (DT == XGEN_I8_I32) {
-                    int4 r = make_int4((int)raw.x + (int)bb.x, (int)raw.y + (int)bb.y, (int)raw.z + (int)bb.z, (int)raw.w + (int)bb.w);
-                    if (P.relu) { r.x = max(r.x, 0); r.y = max(r.y, 0); r.z = max(r.z, 0); r.w = max(r.w, 0); }
-                    *reinterpret_cast<int4 *>((int *)P.y + o + col) = r;
-                } else {
-                    float4 r = make_float4(__uint_as_float(raw.x) + __uint_as_float(bb.x), __uint_as_float(raw.y) + __uint_as_float(bb.y),
-                                           __uint_as_float(raw.z) + __uint_as_float(bb.z), __uint_as_float(raw.w) + __uint_as_float(bb.w));
-                    if (P.relu) { r.x = fmaxf(r.x, 0.f); r.y = fmaxf(r.y, 0.f); r.z = fmaxf(r.z, 0.f); r.w = fmaxf(r.w, 0.f); }
-                    if (DT == XGEN_F32) {
-                        *reinterpret_cast<float4 *>((float *)P.y + o + col) = r;
+                for (int tt = 0; tt < 4; ++tt) {
+                    const int pidx = pt[(t0 + tt) * 32];
+                    if (pidx < 0) continue;
+                    const size_t o = (size_t)pidx * P.c_out + oc0;
+                    uint32_t r[8];
+                    if (part) {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) r[k] = v[k][tt];
+                    } else if (DT == XGEN_I8_I32) {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) { int q = (int)v[k][tt] + (int)bb[k]; if (P.relu) q = max(q, 0); r[k] = (uint32_t)q; }
                     } else {
-                        __half2 lo = __floats2half2_rn(r.x, r.y), hi = __floats2half2_rn(r.z, r.w);
-                        uint2 pk;
-                        pk.x = *reinterpret_cast<uint32_t *>(&lo);
-                        pk.y = *reinterpret_cast<uint32_t *>(&hi);
-                        *reinterpret_cast<uint2 *>((__half *)P.y + o + col) = pk;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) { float q = __uint_as_float(v[k][tt]) + __uint_as_float(bb[k]); if (P.relu) q = fmaxf(q, 0.f); r[k] = __float_as_uint(q); }
                     }
-                }
-            };
-            const int npl = EP * 32;
-            int pl = tid / segs;
-            for (; pl + 3 * dpl < npl; pl += 4 * dpl) {           // four rows in flight
-                const int i0 = pt[pl], i1 = pt[pl + dpl], i2 = pt[pl + 2 * dpl], i3 = pt[pl + 3 * dpl];
-                const uint4 r0 = *reinterpret_cast<const uint4 *>(srow + pl * P.opitch);
-                const uint4 r1 = *reinterpret_cast<const uint4 *>(srow + (pl + dpl) * P.opitch);
-                const uint4 r2 = *reinterpret_cast<const uint4 *>(srow + (pl + 2 * dpl) * P.opitch);
-                const uint4 r3 = *reinterpret_cast<const uint4 *>(srow + (pl + 3 * dpl) * P.opitch);
-                if (i0 >= 0) emit(i0, r0);
-                if (i1 >= 0) emit(i1, r1);
-                if (i2 >= 0) emit(i2, r2);
-                if (i3 >= 0) emit(i3, r3);
-            }
-            for (; pl < npl; pl += dpl) {
-                const int i0 = pt[pl];
-                if (i0 >= 0) emit(i0, *reinterpret_cast<const uint4 *>(srow + pl * P.opitch));
-            }
-            __syncthreads();
-            continue;
-        }
-        const int total = EP * 32 * segs;
-        for (int i = tid; i < total; i += nthreads) {
-            int pl, sgm;                                      // pl = tt*32 + lane'
-            if (P.segs_log >= 0 && segs == (1 << P.segs_log)) { pl = i >> P.segs_log; sgm = i & (segs - 1); }
-            else { pl = i / segs; sgm = i - pl * segs; }
-            const int pidx = ptab[t0 * 32 + pl];
-            if (pidx < 0) continue;
-            const size_t pix = (size_t)pidx;
-            if (P.partial) {
-                // split run: raw sums to the workspace, no bias / ReLU / conversion
-                uint32_t *dst = P.partial + (size_t)blockIdx.z * P.out_elems + pix * P.c_out + oc_lo;
-                if (P.vec_out) *reinterpret_cast<uint4 *>(dst + sgm * 4) = *reinterpret_cast<const uint4 *>(&smem[pl * P.opitch + sgm * 4]);
-                else dst[sgm] = smem[pl * P.opitch + sgm];
-                continue;
-            }
-            if (P.vec_out) {
-                const int ocl = sgm * 4;
-                const uint4 raw = *reinterpret_cast<const uint4 *>(&smem[pl * P.opitch + ocl]);
-                const size_t o = pix * P.c_out + oc_lo + ocl;
-                if (DT == XGEN_I8_I32) {
-                    int4 r = make_int4((int)raw.x, (int)raw.y, (int)raw.z, (int)raw.w);
-                    if (P.bias) {
-                        const int4 bb = *reinterpret_cast<const int4 *>((const int *)P.bias + oc_lo + ocl);
-                        r.x += bb.x; r.y += bb.y; r.z += bb.z; r.w += bb.w;
-                    }
-                    if (P.relu) { r.x = max(r.x, 0); r.y = max(r.y, 0); r.z = max(r.z, 0); r.w = max(r.w, 0); }
-                    *reinterpret_cast<int4 *>((int *)P.y + o) = r;
-                } else {
-                    float4 r = make_float4(__uint_as_float(raw.x), __uint_as_float(raw.y), __uint_as_float(raw.z), __uint_as_float(raw.w));
-                    if (P.bias) {
-                        const float4 bb = *reinterpret_cast<const float4 *>((const float *)P.bias + oc_lo + ocl);
-                        r.x += bb.x; r.y += bb.y; r.z += bb.z; r.w += bb.w;
-                    }
-                    if (P.relu) { r.x = fmaxf(r.x, 0.f); r.y = fmaxf(r.y, 0.f); r.z = fmaxf(r.z, 0.f); r.w = fmaxf(r.w, 0.f); }
-                    if (DT == XGEN_F32) {
-                        *reinterpret_cast<float4 *>((float *)P.y + o) = r;
+                    if (part || DT != XGEN_F16_F32ACC) {
+                        uint32_t *dst = (part ? part : (uint32_t *)P.y) + o;
+                        if (nv == 8 && P.vec_out == 8) {
+                            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
+                        } else if (nv == 8 && P.vec_out == 4) {
+                            *reinterpret_cast<uint4 *>(dst) = make_uint4(r[0], r[1], r[2], r[3]);
+                            *reinterpret_cast<uint4 *>(dst + 4) = make_uint4(r[4], r[5], r[6], r[7]);
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) if (k < nv) dst[k] = r[k];
+                        }
                     } else {
-                        __half2 lo = __floats2half2_rn(r.x, r.y), hi = __floats2half2_rn(r.z, r.w);
-                        uint2 pk;
-                        pk.x = *reinterpret_cast<uint32_t *>(&lo);
-                        pk.y = *reinterpret_cast<uint32_t *>(&hi);
-                        *reinterpret_cast<uint2 *>((__half *)P.y + o) = pk;
+                        __half *dst = (__half *)P.y + o;
+                        if (nv == 8 && P.vec_out >= 4 && (P.c_out & 7) == 0) {
+                            uint4 pk;
+                            __half2 h0 = __floats2half2_rn(__uint_as_float(r[0]), __uint_as_float(r[1]));
+                            __half2 h1 = __floats2half2_rn(__uint_as_float(r[2]), __uint_as_float(r[3]));
+                            __half2 h2 = __floats2half2_rn(__uint_as_float(r[4]), __uint_as_float(r[5]));
+                            __half2 h3 = __floats2half2_rn(__uint_as_float(r[6]), __uint_as_float(r[7]));
+                            pk.x = *reinterpret_cast<uint32_t *>(&h0); pk.y = *reinterpret_cast<uint32_t *>(&h1);
+                            pk.z = *reinterpret_cast<uint32_t *>(&h2); pk.w = *reinterpret_cast<uint32_t *>(&h3);
+                            *reinterpret_cast<uint4 *>(dst) = pk;
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) if (k < nv) dst[k] = __float2half_rn(__uint_as_float(r[k]));
+                        }
                     }
-                }
-            } else {
-                const uint32_t raw = smem[pl * P.opitch + sgm];
-                const size_t o = pix * P.c_out + oc_lo + sgm;
-                if (DT == XGEN_I8_I32) {
-                    int r = (int)raw + (P.bias ? ((const int *)P.bias)[oc_lo + sgm] : 0);
-                    if (P.relu) r = max(r, 0);
-                    ((int *)P.y)[o] = r;
-                } else {
-                    float r = __uint_as_float(raw) + (P.bias ? ((const float *)P.bias)[oc_lo + sgm] : 0.f);
-                    if (P.relu) r = fmaxf(r, 0.f);
-                    if (DT == XGEN_F32) ((float *)P.y)[o] = r;
-                    else ((__half *)P.y)[o] = __float2half_rn(r);
                 }
             }
         }
-        __syncthreads();
     }
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -843,7 +765,8 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     kp.cmd_stage_words = (p.max_seg_slots + 2) * kSlotWords;
     kp.stage_words = kp.act_stage_words + kp.cmd_stage_words;
     kp.vec_in = (p.c_in % E) == 0;
-    kp.vec_out = (p.c_out % 4) == 0;
+    // widest aligned store per 8-channel piece: 8 words (32-byte aligned rows), 4, or scalar
+    kp.vec_out = ((p.c_out % 8) == 0 && ((uintptr_t)y & 31) == 0) ? 8 : ((p.c_out % 4) == 0 ? 4 : 0);
     const bool is_i8 = p.dtype == XGEN_I8_I32;
     const int T = pixels_per_thread(p.stride);
     kp.flush_chunks = 16777216 / (p.cc * 4 * 32640);
@@ -852,16 +775,12 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     kp.cols_per_warp = p.J * T * (kp.fold ? 2 : 1);
     kp.tmem_cols = next_pow2(((p.wpc + 3) / 4) * kp.cols_per_warp);
     if (kp.tmem_cols > 512) return XGEN_ERR_UNSUPPORTED;
-    const int ocb = p.J * p.wpc;
-    kp.opitch = ocb + 4;
     const int exp_words = p.dtype == XGEN_F32 ? 0 : p.cc * g.plane_stride;
     const int npix_tile = (g.tin_w * g.tin_h) << g.ln_log;
     const int max_ctas = 512 / kp.tmem_cols;          // blocks per SM that tensor memory has columns for
     // Pick the stage count: three stages unless two let more blocks share an SM.
-    auto smem_words = [&](int stages, int ep) {
+    auto smem_words = [&](int stages) {
         size_t w = (size_t)stages * kp.stage_words + exp_words;
-        const size_t epi = (size_t)ep * 32 * kp.opitch;
-        if (w < epi) w = epi;
         return ((w + 1) & ~(size_t)1) + 2 * (size_t)npix_tile + 32 * (size_t)T;
     };
     auto occupancy = [&](size_t words) {
@@ -869,22 +788,12 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
         return o < max_ctas ? o : max_ctas;
     };
     int n_stages = 3;
-    if (smem_words(3, 2) * 4 > (size_t)kSmemMaxDynamic || occupancy(smem_words(2, 2)) > occupancy(smem_words(3, 2))) n_stages = 2;
+    if (smem_words(3) * 4 > (size_t)kSmemMaxDynamic || occupancy(smem_words(2)) > occupancy(smem_words(3))) n_stages = 2;
     kp.n_stages = n_stages;
     kp.exp_off_words = n_stages * kp.stage_words;
-    // The epilogue tile reuses the staging memory: as many pixels per pass as fit for free.
-    int ep = 2;
-    for (int cand = T; cand > 2; cand >>= 1)
-        if (smem_words(n_stages, cand) * 4 <= (size_t)kSmemMaxDynamic && occupancy(smem_words(n_stages, cand)) >= occupancy(smem_words(n_stages, 2))) { ep = cand; break; }
-    kp.epi_pix = ep;
-    size_t words = smem_words(n_stages, ep);
+    size_t words = smem_words(n_stages);
     kp.ptab_off_words = (int)(words - 32 * T);
     kp.tab_off_words = kp.ptab_off_words - 2 * npix_tile;
-    {
-        const int segs = kp.vec_out ? (ocb >> 2) : ocb;
-        kp.segs_log = -1;
-        for (int l = 0; l < 12; ++l) if ((1 << l) == segs) kp.segs_log = l;
-    }
     size_t smem = words * 4;
     const bool split = forced ? forced->splits > 1
                               : (h->plan_splits > 1 && h->plan_n == n && h->plan_h == hh && h->plan_w == ww && h->d_partial);
@@ -911,7 +820,7 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     else
         e = p.stride == 1 ? launch_np<XGEN_I8_I32, 1>(p.np, grid, block, smem, st, kp) : launch_np<XGEN_I8_I32, 2>(p.np, grid, block, smem, st, kp);
     if (e == cudaSuccess && split) {
-        const int vec = kp.vec_out;
+        const int vec = kp.vec_out >= 4 ? 1 : 0;
         const size_t items = vec ? kp.out_elems / 4 : kp.out_elems;
         const unsigned blocks = (unsigned)((items + 255) / 256);
         if (p.dtype == XGEN_F32)

@@ -70,12 +70,15 @@ def test_stream_rebuilds_masked_tensor(dtype, stride, shape):
     v = pk.view()
     oc = v["slot_oc"].ravel()
     assert sorted(oc[oc >= 0].tolist()) == list(range(co))               # a bijection onto the filters
-    # blocks hold contiguous original channels
-    J, G = st["filters_per_group"], st["groups_per_block"]
-    for b in range(st["n_blocks"]):
-        blk = v["slot_oc"][b].ravel()
-        blk = blk[blk >= 0]
-        assert blk.min() == b * J * G and blk.max() == min(co, (b + 1) * J * G) - 1
+    # every group is an aligned run of J consecutive output channels
+    J = st["filters_per_group"]
+    for grp in v["slot_oc"].reshape(-1, J):
+        if grp[0] < 0:
+            assert (grp < 0).all()
+            continue
+        assert grp[0] % J == 0
+        for j in range(J):
+            assert grp[j] == (grp[0] + j if grp[0] + j < co else -1)
 
 
 def test_index_overhead_below_csr_and_balance():
