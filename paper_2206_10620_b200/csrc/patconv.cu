@@ -19,6 +19,7 @@
 #include <cuda_runtime.h>
 
 #include <atomic>
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -689,13 +690,28 @@ xgen_status xgen_patconv_plan(xgen_patconv_packed *h, int32_t n, int32_t hh, int
     const int warp_slots = 4 * (512 / cols_per_warp);                 // per SM, set by tensor memory
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
-    const int64_t target = (int64_t)sms * (warp_slots / p.wpc > 0 ? warp_slots / p.wpc : 1);
     const size_t out_bytes = (size_t)n * ho * wo * p.c_out * 4;
-    // Splitting costs one write and one read of the fp32 output per split: cap it.
-    int64_t smax = (int64_t)((size_t)(24u << 20) / out_bytes);
-    if (smax > p.n_chunks / 2) smax = p.n_chunks / 2;
-    int64_t splits = (target + ctas - 1) / ctas;
-    if (splits > smax) splits = smax;
+    // Pick the split count with a small cost model (microseconds): blocks run in waves of
+    // (SMs x blocks per SM); a block costs a fixed prologue + epilogue plus its share of the
+    // multiply-adds at the rate one busy SM sustains; a split adds one write and one read of
+    // the fp32 output per part, plus a second launch.
+    const double blocks_per_wave = (double)sms * (warp_slots / p.wpc > 0 ? warp_slots / p.wpc : 1);
+    const double macs_per_block = 4.0 * (double)p.stats.kernels_surviving * (double)n * ho * wo / (double)ctas;
+    const double t_work = macs_per_block / 72e3, t_fixed = 10.0;      // 72 GMAC/s per SM, 10 us
+    auto estimate = [&](int64_t k) {
+        const int cps_k = (int)((p.n_chunks + k - 1) / k);
+        const int64_t parts = (p.n_chunks + cps_k - 1) / cps_k;
+        const double waves = std::ceil((double)(ctas * parts) / blocks_per_wave);
+        double t = waves * (t_fixed + t_work / (double)parts);
+        if (parts > 1) t += 3.0 + ((double)parts * 2.0 + 1.0) * (double)out_bytes / 4e6;   // 4 TB/s
+        return t;
+    };
+    int64_t splits = 1;
+    double best_t = estimate(1);
+    for (int64_t k = 2; k <= p.n_chunks; ++k) {
+        const double t = estimate(k);
+        if (t < 0.9 * best_t || (splits > 1 && t < best_t)) { best_t = t; splits = k; }
+    }
     if (const char *e = getenv("XGEN_PATCONV_SPLIT")) { int v = atoi(e); if (v >= 1) splits = v < p.n_chunks ? v : p.n_chunks; }
     if (splits < 1) splits = 1;
     const int cps = (int)((p.n_chunks + splits - 1) / splits);
