@@ -174,6 +174,9 @@ def run_gpu(args):
     binding.lib()                                   # fail loudly if the CUDA library is missing
 
     specs = workload(args.workload)
+    if args.only:
+        keep = set(args.only.split(","))
+        specs = [s for s in specs if s.name in keep]
     layers = []
     tdt = {"f32": torch.float32, "f16": torch.float16, "i8": torch.int32}
     for s in specs:
@@ -302,6 +305,7 @@ def main():
     ap.add_argument("--workload", default="vgg16", choices=list(wl.CONFIGS))
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
+    ap.add_argument("--only", default="", help="comma-separated layer names: restrict the stack (profiling aid)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
