@@ -55,6 +55,7 @@ struct KParams {
     int vec_in;                          // c_in is a multiple of the channels per staged word
     int vec_out;                         // widest aligned store of an 8-channel piece: 8 or 4 words, 0 = scalar
     int tab_off_words;                   // offset of the per-pixel staging table in shared memory
+    int seg_off_words;                   // offset of the block's copy of the segment offsets
     int ptab_off_words;                  // offset of the output-pixel table (32 lanes x pixels per thread)
     int fold;                            // i8: keep int32 totals in a second row and fold periodically
     int chunks_per_split;                // grid.z splits the channel chunks; 0 = no split
@@ -165,7 +166,8 @@ patconv_kernel(const KParams P) {
     const int rp = tid & (RP - 1);
     const int pix_step = nthreads / RP;
     const int npix = (P.tin_w * P.tin_h) << P.ln_log;
-    const int32_t *seg = P.seg_off + (size_t)b * P.n_chunks * (P.wpc + 1);
+    const int32_t *seg_g = P.seg_off + (size_t)b * P.n_chunks * (P.wpc + 1);
+    int *seg = reinterpret_cast<int *>(smem + P.seg_off_words);   // this block's slice, copied once
     const uint32_t smem_base = smem_u32(smem);
 
     // Per-pixel staging table, built once: {element index of channel 0 of the input
@@ -192,6 +194,10 @@ patconv_kernel(const KParams P) {
 
     const int c_begin = P.chunks_per_split ? (int)blockIdx.z * P.chunks_per_split : 0;
     const int c_end = P.chunks_per_split ? min(P.n_chunks, c_begin + P.chunks_per_split) : P.n_chunks;
+
+    // Segment offsets of this block's chunks: read once, not on every chunk's critical path.
+    for (int i = tid; i < (c_end - c_begin) * (P.wpc + 1); i += nthreads) seg[i] = seg_g[c_begin * (P.wpc + 1) + i];
+    __syncthreads();
 
     const int q0 = tid / RP;
     auto stage_load = [&](int c) {
@@ -233,7 +239,7 @@ patconv_kernel(const KParams P) {
                 }
             }
             // this block's commands for the chunk: one contiguous segment
-            const int s0 = seg[c * (P.wpc + 1)], s1 = seg[c * (P.wpc + 1) + P.wpc];
+            const int s0 = seg[(c - c_begin) * (P.wpc + 1)], s1 = seg[(c - c_begin) * (P.wpc + 1) + P.wpc];
             const uint32_t cmd = act + (uint32_t)P.act_stage_words * 4u;
             const uint4 *gsrc = reinterpret_cast<const uint4 *>(P.slots + (size_t)s0 * kSlotWords);
             const int n16 = (s1 - s0 + 2) * 2;          // two look-ahead slots beyond the segment
@@ -324,7 +330,7 @@ patconv_kernel(const KParams P) {
             __syncthreads();
             tile_base = smem_base + (uint32_t)P.exp_off_words * 4u;
         }
-        const int s0 = seg[c * (P.wpc + 1)], sg = seg[c * (P.wpc + 1) + warp];
+        const int s0 = seg[(c - c_begin) * (P.wpc + 1)], sg = seg[(c - c_begin) * (P.wpc + 1) + warp];
         uint32_t sp = act + (uint32_t)P.act_stage_words * 4u + (uint32_t)(sg - s0) * 32u;
         run_commands<STRIDE, NP>(sp, tile_base + thr_off, plane_bytes, pitch_bytes, tmem_warp);
         if (DT == XGEN_I8_I32 && P.fold && ((c - c_begin + 1) % P.flush_chunks == 0)) fold_partial_sums();
@@ -795,9 +801,10 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     const int npix_tile = (g.tin_w * g.tin_h) << g.ln_log;
     const int max_ctas = 512 / kp.tmem_cols;          // blocks per SM that tensor memory has columns for
     // Pick the stage count: three stages unless two let more blocks share an SM.
+    const size_t seg_words = ((size_t)p.n_chunks * (p.wpc + 1) + 1) & ~(size_t)1;
     auto smem_words = [&](int stages) {
         size_t w = (size_t)stages * kp.stage_words + exp_words;
-        return ((w + 1) & ~(size_t)1) + 2 * (size_t)npix_tile + 32 * (size_t)T;
+        return ((w + 1) & ~(size_t)1) + 2 * (size_t)npix_tile + 32 * (size_t)T + seg_words;
     };
     auto occupancy = [&](size_t words) {
         int o = (int)((size_t)kSmemPerSM / (words * 4 + 2112));     // + static and per-block reserved shared memory
@@ -808,7 +815,8 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     kp.n_stages = n_stages;
     kp.exp_off_words = n_stages * kp.stage_words;
     size_t words = smem_words(n_stages);
-    kp.ptab_off_words = (int)(words - 32 * T);
+    kp.seg_off_words = (int)(words - seg_words);
+    kp.ptab_off_words = kp.seg_off_words - 32 * T;
     kp.tab_off_words = kp.ptab_off_words - 2 * npix_tile;
     size_t smem = words * 4;
     const bool split = forced ? forced->splits > 1
