@@ -38,7 +38,7 @@ typedef enum {
     XGEN_ERR_UNSUPPORTED = 4,  /* stride, padding or data type outside what is built            */
     XGEN_ERR_ALLOC = 5,        /* host or device allocation failed                               */
     XGEN_ERR_CUDA = 6,         /* a CUDA runtime call failed, or the handle has no device copy   */
-    XGEN_ERR_TIMEOUT = 7       /* reserved for device-side bounded waits                         */
+    XGEN_ERR_TIMEOUT = 7       /* a device-side bounded wait ran out (see xgen_patconv_last_status) */
 } xgen_status;
 
 /* Numeric variants.  F32: x, W, y fp32.  F16_F32ACC: x, W, y IEEE fp16, bias
@@ -216,7 +216,9 @@ xgen_status xgen_patconv_query(const xgen_patconv_packed *packed, xgen_patconv_s
 xgen_status xgen_patconv_view(const xgen_patconv_packed *packed, xgen_patconv_host_view *view);
 
 /* Synchronise the stream and report the first CUDA error seen on it, as a
- * status (XGEN_OK, XGEN_ERR_CUDA).  The kernels contain no unbounded waits. */
+ * status (XGEN_OK, XGEN_ERR_CUDA).  The kernels contain no unbounded waits: a wait
+ * for a tile copy that runs out of its bound marks the handle, the kernel still
+ * ends, and this call then returns XGEN_ERR_TIMEOUT once (results are invalid). */
 xgen_status xgen_patconv_last_status(const xgen_patconv_packed *packed, void *cuda_stream);
 
 /* Release the handle and its device memory.  NULL is allowed. */

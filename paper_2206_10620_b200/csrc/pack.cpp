@@ -63,6 +63,8 @@ static float half_bits_to_float(uint16_t h) {
 PackConfig choose_pack_config(int c_in, int c_out, xgen_dtype dtype, int stride) {
     PackConfig c;
     c.channels_per_chunk = c_in <= 4 ? 4 : 8;
+    // uint8 tiles need 16 channels per chunk to be copied in 16-byte pieces
+    if (dtype == XGEN_I8_I32 && c_in % 16 == 0 && c_in >= 128 && stride == 1) c.channels_per_chunk = 16;
     // A warp's running sums take J x (pixels per thread) tensor-memory columns, and an SM
     // has 4 x 512 of them: 128 columns per warp lets 16 warps share an SM.  Long integer
     // layers keep a second row per filter (int32 totals), so they group half as many.

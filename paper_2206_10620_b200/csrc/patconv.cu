@@ -15,6 +15,7 @@
 // stores straight from tensor memory: a group is a run of consecutive output
 // channels, so a thread writes 32 contiguous bytes per pixel (operator fusion,
 // Sec. 2.2).
+#include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
@@ -56,6 +57,10 @@ struct KParams {
     int vec_out;                         // widest aligned store of an 8-channel piece: 8 or 4 words, 0 = scalar
     int tab_off_words;                   // offset of the per-pixel staging table in shared memory
     int seg_off_words;                   // offset of the block's copy of the segment offsets
+    int use_tma;                         // stage tiles with the tensor-memory-access unit (aligned channel counts)
+    int mbar_off_words;                  // one 8-byte mbarrier per stage
+    int box_bytes;                       // bytes one tensor copy delivers (the whole box, padding included)
+    int *status;                         // device word: set to 1 if a bounded wait ran out
     int ptab_off_words;                  // offset of the output-pixel table (32 lanes x pixels per thread)
     int fold;                            // i8: keep int32 totals in a second row and fold periodically
     int chunks_per_split;                // grid.z splits the channel chunks; 0 = no split
@@ -107,6 +112,22 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 #define PATCONV_S1(np) PATCONV_CORE_S1_NP##np##_F1
 #endif
 
+// Wait for an mbarrier phase with a bound: on expiry the block-wide abort flag and the
+// device status word are set and every later wait returns at once, so the kernel still
+// runs to its end (releasing tensor memory) with garbage results the host can detect.
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, volatile int *abort_flag, int *status) {
+    for (int it = 0; it < 400000; ++it) {
+        uint32_t ok;
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+                     : "=r"(ok) : "r"(mbar), "r"(parity), "r"(2000u) : "memory");
+        if (ok) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1;
+    if (status) atomicExch(status, 1);
+    return false;
+}
+
 template <int STRIDE, int NP>
 __device__ __forceinline__ void run_commands(uint32_t sp, uint32_t tbase, uint32_t plane_bytes,
                                              uint32_t pitch_bytes, uint32_t tmem_base) {
@@ -132,9 +153,10 @@ template <> struct DTraits<XGEN_I8_I32> { static constexpr int E = 4, xbytes = 1
 // ---- the kernel -----------------------------------------------------------------
 template <int DT, int STRIDE, int NP>
 __global__ void __launch_bounds__(kMaxWarps * 32)
-patconv_kernel(const KParams P) {
-    extern __shared__ __align__(16) uint32_t smem[];
+patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
+    extern __shared__ __align__(128) uint32_t smem[];
     __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
     __shared__ int soc_s[kMaxWarps * 16];           // original output channel of every filter slot of this block
     constexpr int E = DTraits<DT>::E;
     constexpr int XB = DTraits<DT>::xbytes;
@@ -169,6 +191,15 @@ patconv_kernel(const KParams P) {
     const int32_t *seg_g = P.seg_off + (size_t)b * P.n_chunks * (P.wpc + 1);
     int *seg = reinterpret_cast<int *>(smem + P.seg_off_words);   // this block's slice, copied once
     const uint32_t smem_base = smem_u32(smem);
+    const uint32_t mbar0 = smem_base + (uint32_t)P.mbar_off_words * 4u;
+    if (tid == 0) {
+        abort_s = 0;
+        if (P.use_tma) {
+            for (int st = 0; st < P.n_stages; ++st)
+                asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(mbar0 + 8u * st) : "memory");
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+    }
 
     // Per-pixel staging table, built once: {element index of channel 0 of the input
     // pixel, or -1 outside the image; word offset of the pixel inside a plane}.
@@ -201,6 +232,24 @@ patconv_kernel(const KParams P) {
 
     const int q0 = tid / RP;
     auto stage_load = [&](int c) {
+        if (P.use_tma) {
+            // one thread hands the tile (a 4-D box of the NHWC tensor, zero-filled outside the
+            // image) and the command segment to the copy engine; an mbarrier counts the bytes
+            if (c < c_end && tid == 0) {
+                const int stage = (c - c_begin) % P.n_stages;
+                const uint32_t raw = smem_base + (uint32_t)(stage * P.stage_words) * 4u;
+                const uint32_t cmd = raw + (uint32_t)P.act_stage_words * 4u;
+                const uint32_t mbar = mbar0 + 8u * stage;
+                const int s0 = seg[(c - c_begin) * (P.wpc + 1)], s1 = seg[(c - c_begin) * (P.wpc + 1) + P.wpc];
+                const uint32_t cmd_bytes = (uint32_t)(s1 - s0 + 2) * (kSlotWords * 4u);
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"((uint32_t)P.box_bytes + cmd_bytes) : "memory");
+                asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                             ::"r"(raw), "l"(&tmap), "r"(c * P.cc), "r"(gx0), "r"(gy0), "r"(n0), "r"(mbar) : "memory");
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(cmd), "l"(P.slots + (size_t)s0 * kSlotWords), "r"(cmd_bytes), "r"(mbar) : "memory");
+            }
+            return;
+        }
         if (c < c_end) {
             const int stage = (c - c_begin) % P.n_stages;
             const uint32_t act = smem_base + (uint32_t)(stage * P.stage_words) * 4u;
@@ -295,12 +344,45 @@ patconv_kernel(const KParams P) {
     // --- main loop over channel chunks --------------------------------------------
     for (int c = c_begin; c < c_end; ++c) {
         const int stage = (c - c_begin) % P.n_stages;
-        if (P.n_stages == 2) cp_async_wait<0>(); else cp_async_wait<1>();
+        if (P.use_tma) {
+            if (!abort_s) mbar_wait(mbar0 + 8u * stage, (uint32_t)(((c - c_begin) / P.n_stages) & 1), &abort_s, P.status);
+        } else {
+            if (P.n_stages == 2) cp_async_wait<0>(); else cp_async_wait<1>();
+        }
         __syncthreads();                       // chunk c has landed; everyone is done with chunk c-1
         stage_load(c + P.n_stages - 1);
         const uint32_t act = smem_base + (uint32_t)(stage * P.stage_words) * 4u;
         uint32_t tile_base = act;
-        if (DT != XGEN_F32) {
+        if (P.use_tma) {
+            // the copy engine delivered [pixel][channel]; spread it into fp32 channel planes
+            float *ex = reinterpret_cast<float *>(smem + P.exp_off_words);
+            const uint4 *raw = reinterpret_cast<const uint4 *>(smem + stage * P.stage_words);
+            const int vec_per_pix = (P.cc * XB) >> 4;                  // 16-byte pieces per pixel: 1 or 2
+            constexpr int EPV = 16 / XB;                               // elements per piece
+            for (int i = tid; i < npix; i += nthreads) {
+                float *dst = ex + tab[i].y;
+                for (int h2 = 0; h2 < vec_per_pix; ++h2) {
+                    const uint4 wd = raw[i * vec_per_pix + h2];
+                    const uint32_t w4[4] = {wd.x, wd.y, wd.z, wd.w};
+                    float *d2 = dst + (size_t)(h2 * EPV) * P.plane_stride;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        if (DT == XGEN_F32) {
+                            d2[k * P.plane_stride] = __uint_as_float(w4[k]);
+                        } else if (DT == XGEN_F16_F32ACC) {
+                            const __half2 h2v = *reinterpret_cast<const __half2 *>(&w4[k]);
+                            d2[(2 * k) * P.plane_stride] = __low2float(h2v);
+                            d2[(2 * k + 1) * P.plane_stride] = __high2float(h2v);
+                        } else {
+#pragma unroll
+                            for (int bq = 0; bq < 4; ++bq) d2[(4 * k + bq) * P.plane_stride] = (float)((w4[k] >> (8 * bq)) & 0xFFu);
+                        }
+                    }
+                }
+            }
+            __syncthreads();
+            tile_base = smem_base + (uint32_t)P.exp_off_words * 4u;
+        } else if (DT != XGEN_F32) {
             // widen the staged words to fp32 planes (exact for fp16 and for uint8)
             float *ex = reinterpret_cast<float *>(smem + P.exp_off_words);
             const int quads = P.plane_stride >> 2;             // plane_stride is a multiple of 4
@@ -544,13 +626,15 @@ struct xgen_patconv_packed {
     int plan_n = 0, plan_h = 0, plan_w = 0, plan_splits = 1, plan_cps = 0;
     uint32_t *d_partial = nullptr;
     size_t partial_bytes = 0;
+    int *d_status = nullptr;            // set by a kernel whose bounded wait ran out
 };
 
 static void free_device_layout(xgen_patconv_packed *h) {
     if (h->d_slots) cudaFree(h->d_slots);
     if (h->d_seg_off) cudaFree(h->d_seg_off);
     if (h->d_slot_oc) cudaFree(h->d_slot_oc);
-    h->d_slots = nullptr; h->d_seg_off = nullptr; h->d_slot_oc = nullptr;
+    if (h->d_status) cudaFree(h->d_status);
+    h->d_slots = nullptr; h->d_seg_off = nullptr; h->d_slot_oc = nullptr; h->d_status = nullptr;
 }
 
 // Upload the host layout; the device must be current.
@@ -562,6 +646,8 @@ static xgen_status upload_layout(xgen_patconv_packed *h) {
     cudaError_t e = cudaMalloc(&h->d_slots, sb);
     if (e == cudaSuccess) e = cudaMalloc(&h->d_seg_off, gb);
     if (e == cudaSuccess) e = cudaMalloc(&h->d_slot_oc, ob);
+    if (e == cudaSuccess) e = cudaMalloc(&h->d_status, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(h->d_slots, 0, sb);
     if (e == cudaSuccess) e = cudaMemcpy(h->d_slots, p.slots.data(), p.slots.size() * 4, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(h->d_seg_off, p.seg_off.data(), gb, cudaMemcpyHostToDevice);
@@ -582,12 +668,34 @@ static cudaError_t log_cuda(cudaError_t e, const char *what) {
     return e;
 }
 
+// cuTensorMapEncodeTiled, fetched through the runtime so the library does not link libcuda.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    static std::mutex m;
+    std::lock_guard<std::mutex> lock(m);
+    if (!tried) {
+        tried = true;
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
 template <int DT, int STRIDE>
-static cudaError_t launch_np(int np, dim3 grid, dim3 block, size_t smem, cudaStream_t st, const KParams &kp) {
+static cudaError_t launch_np(int np, dim3 grid, dim3 block, size_t smem, cudaStream_t st, const KParams &kp, const CUtensorMap &tm) {
     auto go = [&](auto kern) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMaxDynamic);
         if (e != cudaSuccess) return log_cuda(e, "cudaFuncSetAttribute");
-        kern<<<grid, block, smem, st>>>(kp);
+        kern<<<grid, block, smem, st>>>(kp, tm);
         return log_cuda(cudaGetLastError(), "kernel launch");
     };
     switch (np) {
@@ -746,7 +854,17 @@ xgen_status xgen_patconv_last_status(const xgen_patconv_packed *h, void *stream)
     if (!h) return XGEN_ERR_INVALID_ARG;
     cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) return XGEN_ERR_CUDA;
-    return cudaGetLastError() == cudaSuccess ? XGEN_OK : XGEN_ERR_CUDA;
+    if (cudaGetLastError() != cudaSuccess) return XGEN_ERR_CUDA;
+    if (h->d_status) {
+        // a kernel whose bounded wait for a tile copy ran out leaves a mark here
+        int flag = 0;
+        if (cudaMemcpy(&flag, h->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return XGEN_ERR_CUDA;
+        if (flag) {
+            cudaMemset(h->d_status, 0, sizeof(int));
+            return XGEN_ERR_TIMEOUT;
+        }
+    }
+    return XGEN_OK;
 }
 
 }  // extern "C"
@@ -783,9 +901,32 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     kp.pitch = g.pitch; kp.img_stride = g.img_stride; kp.plane_stride = g.plane_stride;
     const int E = p.dtype == XGEN_F32 ? 1 : (p.dtype == XGEN_F16_F32ACC ? 2 : 4);
     kp.raw_planes = p.cc / E;
-    kp.act_stage_words = (kp.raw_planes * g.plane_stride + 3) & ~3;
-    kp.cmd_stage_words = (p.max_seg_slots + 2) * kSlotWords;
-    kp.stage_words = kp.act_stage_words + kp.cmd_stage_words;
+    const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
+    const int npix_box = (g.tin_w * g.tin_h) << g.ln_log;
+    // The copy engine needs 16-byte multiples: the channel run of a chunk and every global stride.
+    EncodeTiledFn encode = nullptr;
+    kp.use_tma = ((p.cc * xb) % 16 == 0) && (((size_t)p.c_in * xb) % 16 == 0) && g.tin_w <= 256 && g.tin_h <= 256 &&
+                 !getenv("XGEN_PATCONV_NO_TMA") && (encode = encode_tiled_fn()) != nullptr;
+    CUtensorMap tm;
+    memset(&tm, 0, sizeof(tm));
+    if (kp.use_tma) {
+        const cuuint64_t gdim[4] = {(cuuint64_t)p.c_in, (cuuint64_t)ww, (cuuint64_t)hh, (cuuint64_t)n};
+        const cuuint64_t gstr[3] = {(cuuint64_t)p.c_in * xb, (cuuint64_t)ww * p.c_in * xb, (cuuint64_t)hh * ww * p.c_in * xb};
+        const cuuint32_t box[4] = {(cuuint32_t)p.cc, (cuuint32_t)g.tin_w, (cuuint32_t)g.tin_h, (cuuint32_t)(1 << g.ln_log)};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        const CUtensorMapDataType dt = p.dtype == XGEN_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                     : (p.dtype == XGEN_F16_F32ACC ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
+        const CUresult cr = encode(&tm, dt, 4, const_cast<void *>(x), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                   CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (cr != CUDA_SUCCESS) {          // fall back to thread-issued copies
+            if (getenv("XGEN_PATCONV_LOG")) fprintf(stderr, "libpatconv: cuTensorMapEncodeTiled failed (%d)\n", (int)cr);
+            kp.use_tma = 0;
+            memset(&tm, 0, sizeof(tm));
+        }
+    }
+    kp.box_bytes = npix_box * p.cc * xb;
+    kp.cmd_stage_words = ((p.max_seg_slots + 2) * kSlotWords + 31) & ~31;
+    kp.status = h->d_status;
     kp.vec_in = (p.c_in % E) == 0;
     // widest aligned store per 8-channel piece: 8 words (32-byte aligned rows), 4, or scalar
     kp.vec_out = ((p.c_out % 8) == 0 && ((uintptr_t)y & 31) == 0) ? 8 : ((p.c_out % 4) == 0 ? 4 : 0);
@@ -797,25 +938,36 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     kp.cols_per_warp = p.J * T * (kp.fold ? 2 : 1);
     kp.tmem_cols = next_pow2(((p.wpc + 3) / 4) * kp.cols_per_warp);
     if (kp.tmem_cols > 512) return XGEN_ERR_UNSUPPORTED;
-    const int exp_words = p.dtype == XGEN_F32 ? 0 : p.cc * g.plane_stride;
+    int exp_words = 0;
+    auto set_stage_layout = [&]() {
+        kp.act_stage_words = kp.use_tma ? ((kp.box_bytes / 4 + 31) & ~31) : ((kp.raw_planes * g.plane_stride + 31) & ~31);
+        kp.stage_words = kp.act_stage_words + kp.cmd_stage_words;
+        exp_words = (p.dtype == XGEN_F32 && !kp.use_tma) ? 0 : ((p.cc * g.plane_stride + 31) & ~31);
+    };
+    set_stage_layout();
     const int npix_tile = (g.tin_w * g.tin_h) << g.ln_log;
     const int max_ctas = 512 / kp.tmem_cols;          // blocks per SM that tensor memory has columns for
     // Pick the stage count: three stages unless two let more blocks share an SM.
     const size_t seg_words = ((size_t)p.n_chunks * (p.wpc + 1) + 1) & ~(size_t)1;
     auto smem_words = [&](int stages) {
         size_t w = (size_t)stages * kp.stage_words + exp_words;
-        return ((w + 1) & ~(size_t)1) + 2 * (size_t)npix_tile + 32 * (size_t)T + seg_words;
+        return ((w + 1) & ~(size_t)1) + 2 * (size_t)npix_tile + 32 * (size_t)T + seg_words + 8;   // + mbarriers
     };
     auto occupancy = [&](size_t words) {
         int o = (int)((size_t)kSmemPerSM / (words * 4 + 2112));     // + static and per-block reserved shared memory
         return o < max_ctas ? o : max_ctas;
     };
+    if (kp.use_tma && smem_words(2) * 4 > (size_t)kSmemMaxDynamic) {
+        kp.use_tma = 0;                   // the copy engine's layout needs one more tile buffer: does not fit
+        set_stage_layout();
+    }
     int n_stages = 3;
     if (smem_words(3) * 4 > (size_t)kSmemMaxDynamic || occupancy(smem_words(2)) > occupancy(smem_words(3))) n_stages = 2;
     kp.n_stages = n_stages;
     kp.exp_off_words = n_stages * kp.stage_words;
     size_t words = smem_words(n_stages);
-    kp.seg_off_words = (int)(words - seg_words);
+    kp.mbar_off_words = (int)(words - 8);
+    kp.seg_off_words = kp.mbar_off_words - (int)seg_words;
     kp.ptab_off_words = kp.seg_off_words - 32 * T;
     kp.tab_off_words = kp.ptab_off_words - 2 * npix_tile;
     size_t smem = words * 4;
@@ -838,11 +990,11 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e;
     if (p.dtype == XGEN_F32)
-        e = p.stride == 1 ? launch_np<XGEN_F32, 1>(p.np, grid, block, smem, st, kp) : launch_np<XGEN_F32, 2>(p.np, grid, block, smem, st, kp);
+        e = p.stride == 1 ? launch_np<XGEN_F32, 1>(p.np, grid, block, smem, st, kp, tm) : launch_np<XGEN_F32, 2>(p.np, grid, block, smem, st, kp, tm);
     else if (p.dtype == XGEN_F16_F32ACC)
-        e = p.stride == 1 ? launch_np<XGEN_F16_F32ACC, 1>(p.np, grid, block, smem, st, kp) : launch_np<XGEN_F16_F32ACC, 2>(p.np, grid, block, smem, st, kp);
+        e = p.stride == 1 ? launch_np<XGEN_F16_F32ACC, 1>(p.np, grid, block, smem, st, kp, tm) : launch_np<XGEN_F16_F32ACC, 2>(p.np, grid, block, smem, st, kp, tm);
     else
-        e = p.stride == 1 ? launch_np<XGEN_I8_I32, 1>(p.np, grid, block, smem, st, kp) : launch_np<XGEN_I8_I32, 2>(p.np, grid, block, smem, st, kp);
+        e = p.stride == 1 ? launch_np<XGEN_I8_I32, 1>(p.np, grid, block, smem, st, kp, tm) : launch_np<XGEN_I8_I32, 2>(p.np, grid, block, smem, st, kp, tm);
     if (e == cudaSuccess && split) {
         const int vec = kp.vec_out >= 4 ? 1 : 0;
         const size_t items = vec ? kp.out_elems / 4 : kp.out_elems;
