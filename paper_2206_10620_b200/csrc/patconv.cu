@@ -25,6 +25,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <utility>
 #include <new>
 #include <vector>
 
@@ -507,10 +508,14 @@ __global__ void __launch_bounds__(256)
 patconv_reduce_kernel(const uint32_t *__restrict__ partial, int splits, size_t out_elems, int c_out,
                       const void *__restrict__ bias, int relu, void *__restrict__ y, int vec) {
     const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * (vec ? 4 : 1);
+    // Launched with programmatic stream serialisation: everything above overlaps the tail
+    // of the convolution kernel; the partial sums are read only after it has completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (i >= out_elems) return;
     const int oc = (int)(i % (size_t)c_out);
     if (DT == XGEN_I8_I32) {
         int r[4] = {0, 0, 0, 0};
+#pragma unroll 4
         for (int z = 0; z < splits; ++z) {
             const uint32_t *src = partial + (size_t)z * out_elems + i;
             if (vec) { const int4 v = *reinterpret_cast<const int4 *>(src); r[0] += v.x; r[1] += v.y; r[2] += v.z; r[3] += v.w; }
@@ -523,6 +528,7 @@ patconv_reduce_kernel(const uint32_t *__restrict__ partial, int splits, size_t o
         }
     } else {
         float r[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
         for (int z = 0; z < splits; ++z) {
             const uint32_t *src = partial + (size_t)z * out_elems + i;
             if (vec) { const float4 v = *reinterpret_cast<const float4 *>(src); r[0] += v.x; r[1] += v.y; r[2] += v.z; r[3] += v.w; }
@@ -693,8 +699,22 @@ static EncodeTiledFn encode_tiled_fn() {
 template <int DT, int STRIDE>
 static cudaError_t launch_np(int np, dim3 grid, dim3 block, size_t smem, cudaStream_t st, const KParams &kp, const CUtensorMap &tm) {
     auto go = [&](auto kern) -> cudaError_t {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMaxDynamic);
-        if (e != cudaSuccess) return log_cuda(e, "cudaFuncSetAttribute");
+        // the opt-in to large dynamic shared memory is per function and per device: do it once
+        static std::mutex mu;
+        static std::vector<std::pair<const void *, int>> done;
+        {
+            std::lock_guard<std::mutex> lock(mu);
+            int dev = 0;
+            cudaGetDevice(&dev);
+            const std::pair<const void *, int> key((const void *)kern, dev);
+            bool found = false;
+            for (const auto &k : done) found = found || k == key;
+            if (!found) {
+                cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMaxDynamic);
+                if (e != cudaSuccess) return log_cuda(e, "cudaFuncSetAttribute");
+                done.push_back(key);
+            }
+        }
         kern<<<grid, block, smem, st>>>(kp, tm);
         return log_cuda(cudaGetLastError(), "kernel launch");
     };
@@ -999,13 +1019,24 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
         const int vec = kp.vec_out >= 4 ? 1 : 0;
         const size_t items = vec ? kp.out_elems / 4 : kp.out_elems;
         const unsigned blocks = (unsigned)((items + 255) / 256);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(blocks, 1, 1); cfg.blockDim = dim3(256, 1, 1); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        const uint32_t *part_c = partial;
+        const size_t oe = kp.out_elems;
+        const int co = p.c_out, rl = kp.relu;
+        const void *bias_c = bias;
         if (p.dtype == XGEN_F32)
-            patconv_reduce_kernel<XGEN_F32><<<blocks, 256, 0, st>>>(partial, n_splits, kp.out_elems, p.c_out, bias, kp.relu, y, vec);
+            e = cudaLaunchKernelEx(&cfg, patconv_reduce_kernel<XGEN_F32>, part_c, n_splits, oe, co, bias_c, rl, y, vec);
         else if (p.dtype == XGEN_F16_F32ACC)
-            patconv_reduce_kernel<XGEN_F16_F32ACC><<<blocks, 256, 0, st>>>(partial, n_splits, kp.out_elems, p.c_out, bias, kp.relu, y, vec);
+            e = cudaLaunchKernelEx(&cfg, patconv_reduce_kernel<XGEN_F16_F32ACC>, part_c, n_splits, oe, co, bias_c, rl, y, vec);
         else
-            patconv_reduce_kernel<XGEN_I8_I32><<<blocks, 256, 0, st>>>(partial, n_splits, kp.out_elems, p.c_out, bias, kp.relu, y, vec);
-        e = log_cuda(cudaGetLastError(), "reduce launch");
+            e = cudaLaunchKernelEx(&cfg, patconv_reduce_kernel<XGEN_I8_I32>, part_c, n_splits, oe, co, bias_c, rl, y, vec);
+        if (e == cudaSuccess) e = cudaGetLastError();
+        e = log_cuda(e, "reduce launch");
         if (e == cudaSuccess) g_launches.fetch_add(1);
     }
     if (prev != h->device) cudaSetDevice(prev);
