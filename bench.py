@@ -257,17 +257,28 @@ def run_gpu(args):
                 "frac_of_binding_roofline": None}
     roofline["frac_of_binding_roofline"] = roofline["binding_roofline_ms"] / layer_ms
 
-    # --- end to end through the host-buffer entry point (copies inside the timed region)
+    # --- end to end through the host-buffer entry point (copies inside the timed region):
+    # inputs and results live in pinned host memory; every step copies every layer's input
+    # and bias to the device and its result back.
     e2e_steps = max(1, min(args.steps, 5))
-    h2d = sum(d.x.nbytes + d.bias.nbytes for (s, d, *_r) in layers)
-    d2h = sum(y.numel() * y.element_size() for (*_r, y) in layers)
-    for (s, d, pk, x, b, y) in layers[:2]:
-        pk.run_host(d.x, d.bias, s.relu)
+    pinned = []
+    for (s, d, pk, x, b, y) in layers:
+        hx = torch.from_numpy(d.x).pin_memory()
+        hb = torch.from_numpy(d.bias).pin_memory()
+        hy = torch.empty(y.shape, dtype=y.dtype).pin_memory()
+        pinned.append((hx, hb, hy))
+    h2d = sum(hx.numel() * hx.element_size() + hb.numel() * hb.element_size() for hx, hb, hy in pinned)
+    d2h = sum(hy.numel() * hy.element_size() for hx, hb, hy in pinned)
+
+    def e2e_step():
+        for (s, d, pk, x, b, y), (hx, hb, hy) in zip(layers, pinned):
+            pk.run_host_ptr(hx.data_ptr(), s.n, s.h, s.w, hb.data_ptr(), s.relu, hy.data_ptr())
+
+    e2e_step()
     barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
-        for (s, d, pk, x, b, y) in layers:
-            pk.run_host(d.x, d.bias, s.relu)
+        e2e_step()
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
     e2e_s = max_over_ranks(e2e_s, dist, dev)

@@ -185,9 +185,11 @@ xgen_status xgen_patconv_run_static_scratch(const xgen_patconv_packed *packed, c
 
 /*
  * Convenience for callers that hold host tensors: copies x (and bias) to the
- * device, runs the layer, copies y back and waits.  Allocates and frees device
- * buffers on every call.  Same tensor layouts as xgen_patconv_run, all
- * pointers host memory.  Errors as xgen_patconv_run, plus ALLOC.
+ * device, runs the layer on the default stream, copies y back and waits.  The
+ * device staging buffers belong to the handle and are kept between calls (they
+ * only grow); calls on one handle are serialised.  Pinned (page-locked) host
+ * memory makes the copies faster but is not required.  Same tensor layouts as
+ * xgen_patconv_run, all pointers host memory.  Errors as xgen_patconv_run, plus ALLOC.
  */
 xgen_status xgen_patconv_run_host(const xgen_patconv_packed *packed, const void *x_host, int32_t n,
                                   int32_t h, int32_t w, const void *bias_host, int32_t relu,

@@ -186,6 +186,11 @@ class Packed:
                                            y.ctypes.data), "xgen_patconv_run_host")
         return y
 
+    def run_host_ptr(self, x_ptr, n, h, w, bias_ptr, relu, y_ptr):
+        """xgen_patconv_run_host on raw host addresses (e.g. pinned buffers)."""
+        _check(lib().xgen_patconv_run_host(self._h, x_ptr, n, h, w, bias_ptr or None, int(bool(relu)), y_ptr),
+               "xgen_patconv_run_host")
+
     def sync(self, stream=0):
         _check(lib().xgen_patconv_last_status(self._h, stream or None), "xgen_patconv_last_status")
 

@@ -633,6 +633,10 @@ struct xgen_patconv_packed {
     uint32_t *d_partial = nullptr;
     size_t partial_bytes = 0;
     int *d_status = nullptr;            // set by a kernel whose bounded wait ran out
+    // device staging buffers of xgen_patconv_run_host, kept between calls (grow only)
+    mutable std::mutex host_mu;
+    mutable void *d_hx = nullptr, *d_hy = nullptr, *d_hb = nullptr;
+    mutable size_t hx_bytes = 0, hy_bytes = 0;
 };
 
 static void free_device_layout(xgen_patconv_packed *h) {
@@ -783,6 +787,9 @@ void xgen_patconv_free(xgen_patconv_packed *h) {
     if (!h) return;
     free_device_layout(h);
     if (h->d_partial) cudaFree(h->d_partial);
+    if (h->d_hx) cudaFree(h->d_hx);
+    if (h->d_hy) cudaFree(h->d_hy);
+    if (h->d_hb) cudaFree(h->d_hb);
     delete h;
 }
 
@@ -1111,12 +1118,24 @@ xgen_status xgen_patconv_run_host(const xgen_patconv_packed *h, const void *x, i
     const size_t xbytes = (size_t)n * hh * ww * p.c_in * xb, ybytes = (size_t)n * ho * wo * p.c_out * yb;
     int prev = 0;
     if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
-    void *dx = nullptr, *dy = nullptr, *db = nullptr;
+    std::lock_guard<std::mutex> lock(h->host_mu);      // one host-buffer call per handle at a time
     xgen_status rs = XGEN_OK;
-    cudaError_t e = cudaMalloc(&dx, xbytes);
-    if (e == cudaSuccess) e = cudaMalloc(&dy, ybytes);
-    if (e == cudaSuccess && bias) e = cudaMalloc(&db, (size_t)p.c_out * 4);
+    cudaError_t e = cudaSuccess;
+    if (xbytes > h->hx_bytes) {
+        if (h->d_hx) cudaFree(h->d_hx);
+        h->d_hx = nullptr; h->hx_bytes = 0;
+        e = cudaMalloc(&h->d_hx, xbytes);
+        if (e == cudaSuccess) h->hx_bytes = xbytes;
+    }
+    if (e == cudaSuccess && ybytes > h->hy_bytes) {
+        if (h->d_hy) cudaFree(h->d_hy);
+        h->d_hy = nullptr; h->hy_bytes = 0;
+        e = cudaMalloc(&h->d_hy, ybytes);
+        if (e == cudaSuccess) h->hy_bytes = ybytes;
+    }
+    if (e == cudaSuccess && bias && !h->d_hb) e = cudaMalloc(&h->d_hb, (size_t)p.c_out * 4);
     if (e != cudaSuccess) { rs = XGEN_ERR_ALLOC; cudaGetLastError(); }
+    void *dx = h->d_hx, *dy = h->d_hy, *db = bias ? h->d_hb : nullptr;
     if (rs == XGEN_OK) {
         e = cudaMemcpyAsync(dx, x, xbytes, cudaMemcpyHostToDevice, 0);
         if (e == cudaSuccess && bias) e = cudaMemcpyAsync(db, bias, (size_t)p.c_out * 4, cudaMemcpyHostToDevice, 0);
@@ -1128,7 +1147,6 @@ xgen_status xgen_patconv_run_host(const xgen_patconv_packed *h, const void *x, i
         if (e == cudaSuccess) e = cudaStreamSynchronize(0);
         if (e != cudaSuccess) rs = XGEN_ERR_CUDA;
     }
-    cudaFree(dx); cudaFree(dy); cudaFree(db);
     cudaSetDevice(prev);
     return rs;
 }
