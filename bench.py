@@ -39,6 +39,12 @@ UNIT = "GFLOP/s"
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of patconv_kernel, average per launch over one
+# step of this workload, from the ncu capture summarised in profiles/bench_vgg16_launch_list.md
+# (taken with the kernels as committed; set to None when the kernel changes).
+NCU_DRAM_BYTES_PER_LAUNCH = 4.55e6
+
+
 def rank_seed(rank: int) -> int:
     """Every rank draws its own image (weak scaling: the batch is sharded by rank)."""
     return wl.BASE_SEED + rank
@@ -248,7 +254,8 @@ def run_gpu(args):
     layer_ms = sum(p["ms"] for p in per_layer)
     achieved = 2.0 * useful / (layer_ms * 1e-3) / 1e12
     roofline = {"bound": "alu", "achieved": achieved, "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s",
-                "frac": achieved / FP32_PEAK_TFLOPS, "traffic": None,
+                "frac": achieved / FP32_PEAK_TFLOPS,
+                "traffic": NCU_DRAM_BYTES_PER_LAUNCH if args.workload == "vgg16" and not args.only else None,
                 "kernel": "patconv_kernel<f32, stride 1, 8 patterns> (all 13 layers)",
                 "peak_source": "148 SMs x 128 lanes x 2 x 1.965 GHz (FP32 FMA pipe; derived, not in the measured-peaks file)",
                 "hbm_peak_gbs": hbm, "hbm_peak_source": hbm_src,
