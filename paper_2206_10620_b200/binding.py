@@ -65,7 +65,7 @@ def lib():
     """Load libpatconv.so (building it first if it is missing or stale)."""
     global _lib
     if _lib is None:
-        path = _build.LIB_PATH
+        path = os.environ.get("XGEN_PATCONV_LIB") or _build.LIB_PATH    # another build of the library, if named
         if not os.path.exists(path):
             path = _build.build()
         L = ctypes.CDLL(path)

@@ -63,8 +63,6 @@ static float half_bits_to_float(uint16_t h) {
 PackConfig choose_pack_config(int c_in, int c_out, xgen_dtype dtype, int stride) {
     PackConfig c;
     c.channels_per_chunk = c_in <= 4 ? 4 : 8;
-    // uint8 tiles need 16 channels per chunk to be copied in 16-byte pieces
-    if (dtype == XGEN_I8_I32 && c_in % 16 == 0 && c_in >= 128 && stride == 1) c.channels_per_chunk = 16;
     // A warp's running sums take J x (pixels per thread) tensor-memory columns, and an SM
     // has 4 x 512 of them: 128 columns per warp lets 16 warps share an SM.  Long integer
     // layers keep a second row per filter (int32 totals), so they group half as many.
@@ -250,7 +248,7 @@ xgen_status build_layout(PackedHost &out, const PackConfig &cfg) {
     s.weight_bytes = 4 * k_surv * wbytes;
     s.index_bytes = n_slots * 2 + (int64_t)out.seg_off.size() * 4 + (int64_t)out.slot_oc.size() * 4;
     s.csr_index_bytes = 4 * k_surv * 4 + (int64_t)(cout + 1) * 4;
-    s.stream_bytes = n_slots * kSlotWords * 4;
+    s.stream_bytes = n_slots * kDevSlotBytes;
     s.filters_per_group = J; s.groups_per_block = wpc; s.n_blocks = n_blocks;
     s.channels_per_chunk = cc; s.n_chunks = n_chunks; s.patterns_compiled = np;
     s.max_segment_slots = out.max_seg_slots;

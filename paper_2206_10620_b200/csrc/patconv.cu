@@ -1,20 +1,29 @@
 // libpatconv: CUDA kernels (sm_100a) and the C ABI.
 //
 // One thread block = one tile of output pixels x one block of contiguous output
-// channels.  Each warp owns a filter group (J filters); each lane owns a
-// 4x4 block of output pixels (2x4 at stride 2; up to LN images side by side for
-// small images).
-// Per chunk of input channels the block stages (cp.async) the input tile with
-// its halo into channel planes in shared memory -- the NHWC -> plane transpose
-// happens in that copy -- together with the block's slice of the command
-// stream.  Each warp then interprets its commands (core_gen.inc): LOAD brings
-// the thread's activation patch of one channel into registers once, and every
+// channels (x one range of input-channel chunks when the layer is split).  It has
+// up to 16 consumer warps and four producer warps.
+//
+// Each consumer warp owns a filter group (J filters); each of its lanes owns a 4x4
+// block of output pixels (2x4 at stride 2; up to LN images side by side for small
+// images).  The warp interprets its command stream (core_gen.inc): LOAD brings the
+// thread's activation patch of one channel into registers once, and every
 // surviving kernel of the group on that channel reuses it (the paper's load
 // redundancy elimination, Sec. 2.3); the running sums live in tensor memory,
-// addressed by filter slot.  The epilogue adds bias, applies ReLU, converts and
-// stores straight from tensor memory: a group is a run of consecutive output
-// channels, so a thread writes 32 contiguous bytes per pixel (operator fusion,
-// Sec. 2.2).
+// addressed by filter slot.
+//
+// The producer warps stage, per chunk of input channels, the input tile with its
+// halo: the tensor copy engine delivers the NHWC box (zero-filled outside the
+// image) and the block's slice of the command stream, and the producers spread
+// the box into per-channel planes laid out as the operand pairs the two-wide FMAs
+// read.  Channel counts the copy engine cannot address are read with plain loads.
+// Stages are handed over with mbarriers (full / empty), so warps never meet at a
+// block-wide barrier inside the main loop and a slow warp only delays the stage
+// it still reads.
+//
+// The epilogue adds bias, applies ReLU, converts and stores straight from tensor
+// memory: a group is a run of consecutive output channels, so a thread writes 32
+// contiguous bytes per pixel (operator fusion, Sec. 2.2).
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -36,7 +45,12 @@ namespace patconv {
 
 constexpr int kSmemPerSM = 233472;     // 228 KB
 constexpr int kSmemMaxDynamic = 232448 - 2048;  // 227 KB per block less static shared memory
-constexpr int kMaxWarps = 16;
+constexpr int kMaxWarps = 16;          // consumer warps
+constexpr int kProducerWarps = 4;      // staging warps on top of them
+constexpr int kDevSlotWords = 12;      // device command slot: 48 bytes (weights duplicated)
+constexpr int kMaxStages = 4;
+constexpr int kRawStages = 2;
+constexpr size_t kCmdStageBudget = 24 * 1024;   // bytes of commands per pipeline stage the packer aims for
 
 struct KParams {
     const void *x; void *y; const void *bias;
@@ -44,53 +58,47 @@ struct KParams {
     int n, h, w, ho, wo, c_in, c_out;
     int relu;
     int J, wpc, cc, n_chunks;
+    int rc;                              // channels per tile box (a multiple of cc)
     int lx_log, ly_log, ln_log;          // lanes along x, y and images: 2^.. each, product 32
     int tiles_x, tiles_y;
     int tin_w, tin_h;                    // staged tile extents, input pixels
-    int pitch, img_stride, plane_stride; // words
-    int raw_planes;                      // planes of one staged chunk (cc / channels per word)
-    int act_stage_words, cmd_stage_words, stage_words;
-    int n_stages;
-    int exp_off_words;                   // offset of the expanded tile (f16 / i8) in shared memory
+    int pitch, img_stride, half_stride, plane_stride;   // words
+    int raw_stage_words, plane_stage_words, cmd_stage_words;
+    int n_stages;                        // plane + command stages
+    int raw_off_words, plane_off_words, cmd_off_words;
+    int tab_off_words;                   // per staged pixel: its two destinations inside a plane
+    int src_off_words;                   // per staged pixel: element index in x, or -1 (plain-load staging)
+    int ptab_off_words;                  // output-pixel table (32 lanes x pixels per thread)
+    int seg_off_words;                   // the block's copy of the segment offsets
+    int mbar_off_words;                  // 8-byte mbarriers: full, commands, empty (per stage), raw (per raw stage)
     int tmem_cols, cols_per_warp;
     int flush_chunks;                    // i8: chunks between folds of the fp32 partial sums
-    int vec_in;                          // c_in is a multiple of the channels per staged word
     int vec_out;                         // widest aligned store of an 8-channel piece: 8 or 4 words, 0 = scalar
-    int tab_off_words;                   // offset of the per-pixel staging table in shared memory
-    int seg_off_words;                   // offset of the block's copy of the segment offsets
-    int use_tma;                         // stage tiles with the tensor-memory-access unit (aligned channel counts)
-    int mbar_off_words;                  // one 8-byte mbarrier per stage
+    int use_tma;                         // stage tiles with the tensor copy engine (aligned channel counts)
     int box_bytes;                       // bytes one tensor copy delivers (the whole box, padding included)
     int *status;                         // device word: set to 1 if a bounded wait ran out
-    int ptab_off_words;                  // offset of the output-pixel table (32 lanes x pixels per thread)
     int fold;                            // i8: keep int32 totals in a second row and fold periodically
     int chunks_per_split;                // grid.z splits the channel chunks; 0 = no split
-    uint32_t *partial;                   // split runs: [split][n*ho*wo*c_out] raw fp32 / int32 sums
+    uint32_t *partial;                   // split runs reduced by a second kernel: [split][n*ho*wo*c_out] raw sums
     size_t out_elems;                    // n*ho*wo*c_out
+    // Split runs reduced inside this kernel: every block writes its raw sums as rows of
+    // 32 lanes x 8 channels, [item][split][row][lane][8], item = (tile, filter block); a
+    // counter per item tells when all of its splits have arrived, and each of them then
+    // reduces a share of the rows.
+    uint32_t *ws;
+    uint32_t *counters;
+    uint32_t target;                     // counter value at which every split of an item has arrived
+    int n_splits;
 };
 
 // ---- small PTX wrappers -----------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
-__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src, int src_bytes) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
 __device__ __forceinline__ void tmem_ld8(uint32_t ta, uint32_t (&r)[8]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                  : "r"(ta) : "memory");
-}
-__device__ __forceinline__ void tmem_ld2(uint32_t ta, uint32_t (&r)[2]) {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0,%1}, [%2];"
-                 : "=r"(r[0]), "=r"(r[1]) : "r"(ta) : "memory");
 }
 __device__ __forceinline__ void tmem_ld4(uint32_t ta, uint32_t (&r)[4]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
@@ -103,19 +111,20 @@ __device__ __forceinline__ void tmem_st8(uint32_t ta, const uint32_t (&r)[8]) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// Stride-1 layers use the packed two-wide fp32 FMA unless built with -DPATCONV_F2=0.
-#ifndef PATCONV_F2
-#define PATCONV_F2 1
-#endif
-#if PATCONV_F2
-#define PATCONV_S1(np) PATCONV_CORE_S1_NP##np##_F2
-#else
-#define PATCONV_S1(np) PATCONV_CORE_S1_NP##np##_F1
-#endif
+__device__ __forceinline__ void mbar_init(uint32_t mbar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t mbar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(mbar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t mbar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");
+}
 
 // Wait for an mbarrier phase with a bound: on expiry the block-wide abort flag and the
-// device status word are set and every later wait returns at once, so the kernel still
-// runs to its end (releasing tensor memory) with garbage results the host can detect.
+// device status word are set and every later wait returns at once; the warps then leave
+// their loops, so the kernel still runs to its end (releasing tensor memory) with
+// results the host can tell are invalid.
 __device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, volatile int *abort_flag, int *status) {
     for (int it = 0; it < 400000; ++it) {
         uint32_t ok;
@@ -130,43 +139,98 @@ __device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, volati
 }
 
 template <int STRIDE, int NP>
-__device__ __forceinline__ void run_commands(uint32_t sp, uint32_t tbase, uint32_t plane_bytes,
-                                             uint32_t pitch_bytes, uint32_t tmem_base) {
+__device__ __forceinline__ void run_commands(uint32_t sp, uint32_t base_a, uint32_t plane_bytes,
+                                             uint32_t pitch_bytes, uint32_t tmem_base, uint32_t base_b) {
     if (STRIDE == 1) {
-        if (NP == 4) PATCONV_S1(4)(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
-        else if (NP == 8) PATCONV_S1(8)(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
-        else if (NP == 12) PATCONV_S1(12)(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
-        else PATCONV_S1(126)(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        if (NP == 4) PATCONV_CORE_S1_NP4(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
+        else if (NP == 8) PATCONV_CORE_S1_NP8(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
+        else if (NP == 12) PATCONV_CORE_S1_NP12(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
+        else PATCONV_CORE_S1_NP126(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
     } else {
-        if (NP == 4) PATCONV_CORE_S2_NP4_F1(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
-        else if (NP == 8) PATCONV_CORE_S2_NP8_F1(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
-        else if (NP == 12) PATCONV_CORE_S2_NP12_F1(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
-        else PATCONV_CORE_S2_NP126_F1(sp, tbase, plane_bytes, pitch_bytes, tmem_base);
+        if (NP == 4) PATCONV_CORE_S2_NP4(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
+        else if (NP == 8) PATCONV_CORE_S2_NP8(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
+        else if (NP == 12) PATCONV_CORE_S2_NP12(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
+        else PATCONV_CORE_S2_NP126(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
     }
 }
 
-// Channels carried by one staged 32-bit word, and element sizes.
+// Element sizes of the activations (in) and the results (out).
 template <int DT> struct DTraits;
-template <> struct DTraits<XGEN_F32> { static constexpr int E = 1, xbytes = 4, ybytes = 4; };
-template <> struct DTraits<XGEN_F16_F32ACC> { static constexpr int E = 2, xbytes = 2, ybytes = 2; };
-template <> struct DTraits<XGEN_I8_I32> { static constexpr int E = 4, xbytes = 1, ybytes = 4; };
+template <> struct DTraits<XGEN_F32> { static constexpr int xbytes = 4, ybytes = 4; };
+template <> struct DTraits<XGEN_F16_F32ACC> { static constexpr int xbytes = 2, ybytes = 2; };
+template <> struct DTraits<XGEN_I8_I32> { static constexpr int xbytes = 1, ybytes = 4; };
+
+// One staged activation element widened to fp32 (exact for fp16 and for uint8).
+template <int DT> __device__ __forceinline__ float load_widened(const char *p) {
+    if (DT == XGEN_F32) return __ldg(reinterpret_cast<const float *>(p));
+    if (DT == XGEN_F16_F32ACC) return __half2float(__ushort_as_half(__ldg(reinterpret_cast<const unsigned short *>(p))));
+    return (float)__ldg(reinterpret_cast<const unsigned char *>(p));
+}
+
+// One piece of the result: 8 adjacent output channels of one pixel.  r holds raw sums (fp32
+// bits, or int32 for the integer variant); bias and ReLU are applied here, then the piece is
+// converted and stored at element offset o of `out`.  raw = store the sums as they are (32-bit).
+template <int DT>
+__device__ __forceinline__ void store_piece(const KParams &P, const uint32_t (&rin)[8], const uint32_t (&bb)[8], int relu,
+                                            void *out, size_t o, int nv, bool raw) {
+    uint32_t r[8];
+    if (raw) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) r[k] = rin[k];
+    } else if (DT == XGEN_I8_I32) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { int q = (int)rin[k] + (int)bb[k]; if (relu) q = max(q, 0); r[k] = (uint32_t)q; }
+    } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { float q = __uint_as_float(rin[k]) + __uint_as_float(bb[k]); if (relu) q = fmaxf(q, 0.f); r[k] = __float_as_uint(q); }
+    }
+    if (raw || DT != XGEN_F16_F32ACC) {
+        uint32_t *dst = (uint32_t *)out + o;
+        if (nv == 8 && P.vec_out == 8) {
+            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
+        } else if (nv == 8 && P.vec_out == 4) {
+            *reinterpret_cast<uint4 *>(dst) = make_uint4(r[0], r[1], r[2], r[3]);
+            *reinterpret_cast<uint4 *>(dst + 4) = make_uint4(r[4], r[5], r[6], r[7]);
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) if (k < nv) dst[k] = r[k];
+        }
+    } else {
+        __half *dst = (__half *)out + o;
+        if (nv == 8 && P.vec_out >= 4 && (P.c_out & 7) == 0) {
+            uint4 pk;
+            __half2 h0 = __floats2half2_rn(__uint_as_float(r[0]), __uint_as_float(r[1]));
+            __half2 h1 = __floats2half2_rn(__uint_as_float(r[2]), __uint_as_float(r[3]));
+            __half2 h2 = __floats2half2_rn(__uint_as_float(r[4]), __uint_as_float(r[5]));
+            __half2 h3 = __floats2half2_rn(__uint_as_float(r[6]), __uint_as_float(r[7]));
+            pk.x = *reinterpret_cast<uint32_t *>(&h0); pk.y = *reinterpret_cast<uint32_t *>(&h1);
+            pk.z = *reinterpret_cast<uint32_t *>(&h2); pk.w = *reinterpret_cast<uint32_t *>(&h3);
+            *reinterpret_cast<uint4 *>(dst) = pk;
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) if (k < nv) dst[k] = __float2half_rn(__uint_as_float(r[k]));
+        }
+    }
+}
 
 // ---- the kernel -----------------------------------------------------------------
 template <int DT, int STRIDE, int NP>
-__global__ void __launch_bounds__(kMaxWarps * 32)
+__global__ void __launch_bounds__((kMaxWarps + kProducerWarps) * 32)
 patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     extern __shared__ __align__(128) uint32_t smem[];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     __shared__ int soc_s[kMaxWarps * 16];           // original output channel of every filter slot of this block
-    constexpr int E = DTraits<DT>::E;
     constexpr int XB = DTraits<DT>::xbytes;
     constexpr int BW = STRIDE == 1 ? 4 : 2, BH = 4;   // output pixels per thread: BW x BH
     constexpr int T = BW * BH;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nthreads = blockDim.x;
+    const bool producer = warp >= P.wpc;
+    const int pw = warp - P.wpc;                     // producer warp number
     const int b = blockIdx.y;
+    const int item = (int)(blockIdx.x + gridDim.x * blockIdx.y);   // (tile, filter block)
     int tile = blockIdx.x;
     const int tx = tile % P.tiles_x; tile /= P.tiles_x;
     const int ty = tile % P.tiles_y;
@@ -176,320 +240,358 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     const int TW = BW * LX, TH = BH * LY;
     const int n0 = tn << P.ln_log;                   // first image of the tile
     const int gy0 = ty * TH * STRIDE - 1, gx0 = tx * TW * STRIDE - 1;   // input coords of tile (0,0)
+    const int NS = P.n_stages;
+    const int npix = (P.tin_w * P.tin_h) << P.ln_log;
 
-    // --- tensor memory for the running sums --------------------------------------
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t mbar0 = smem_base + (uint32_t)P.mbar_off_words * 4u;
+    auto bar_full = [&](int s) { return mbar0 + 8u * (uint32_t)s; };            // planes of a stage written
+    auto bar_cmd = [&](int s) { return mbar0 + 8u * (uint32_t)(NS + s); };      // commands of a stage landed
+    auto bar_empty = [&](int s) { return mbar0 + 8u * (uint32_t)(2 * NS + s); };   // every consumer warp done with a stage
+    auto bar_raw = [&](int r) { return mbar0 + 8u * (uint32_t)(3 * NS + r); };  // a tile box landed
+    auto bar_rawfree = [&](int r) { return mbar0 + 8u * (uint32_t)(3 * NS + kRawStages + r); };   // every producer warp done with a box
+
+    const int c_begin = P.chunks_per_split ? (int)blockIdx.z * P.chunks_per_split : 0;
+    const int c_end = P.chunks_per_split ? min(P.n_chunks, c_begin + P.chunks_per_split) : P.n_chunks;
+
+    // --- tensor memory for the running sums; barriers -------------------------------
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)P.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-
-    // --- staging -------------------------------------------------------------------
-    const int RP = P.raw_planes;                      // power of two
-    const int rp = tid & (RP - 1);
-    const int pix_step = nthreads / RP;
-    const int npix = (P.tin_w * P.tin_h) << P.ln_log;
-    const int32_t *seg_g = P.seg_off + (size_t)b * P.n_chunks * (P.wpc + 1);
-    int *seg = reinterpret_cast<int *>(smem + P.seg_off_words);   // this block's slice, copied once
-    const uint32_t smem_base = smem_u32(smem);
-    const uint32_t mbar0 = smem_base + (uint32_t)P.mbar_off_words * 4u;
-    if (tid == 0) {
+    if (pw == 0 && lane == 0) {
         abort_s = 0;
-        if (P.use_tma) {
-            for (int st = 0; st < P.n_stages; ++st)
-                asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(mbar0 + 8u * st) : "memory");
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        }
+        for (int s = 0; s < NS; ++s) { mbar_init(bar_full(s), kProducerWarps); mbar_init(bar_cmd(s), 1); mbar_init(bar_empty(s), (uint32_t)P.wpc); }
+        for (int r = 0; r < kRawStages; ++r) { mbar_init(bar_raw(r), 1); mbar_init(bar_rawfree(r), kProducerWarps); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    __syncthreads();
 
-    // Per-pixel staging table, built once: {element index of channel 0 of the input
-    // pixel, or -1 outside the image; word offset of the pixel inside a plane}.
+    // A tile box carries rc channels, i.e. spb = rc / cc consecutive chunks; boxes q0..q_end
+    // cover this block's chunks.  Box q is handed to the copy engine by one thread.
+    const int spb = P.rc / P.cc;
+    const int q0 = c_begin / spb, q_end = (c_end - 1) / spb;
+    auto issue_box = [&](int q) {
+        const int r = (q - q0) % kRawStages;
+        const uint32_t dst = smem_base + (uint32_t)(P.raw_off_words + r * P.raw_stage_words) * 4u;
+        mbar_expect_tx(bar_raw(r), (uint32_t)P.box_bytes);
+        asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                     ::"r"(dst), "l"(&tmap), "r"(q * P.rc), "r"(gx0), "r"(gy0), "r"(n0), "r"(bar_raw(r)) : "memory");
+    };
+    if (pw == 0 && lane == 0 && P.use_tma)
+        for (int r = 0; r < kRawStages && q0 + r <= q_end; ++r) issue_box(q0 + r);
+
+    // --- tables, built once by all threads while the first boxes are in flight --------
+    // Per staged pixel: where its value goes inside a channel plane.  A plane holds, per
+    // tile row and lane column, half 0 = input columns (0,2,1,3) of that lane's patch and
+    // half 1 = (2,4,3,5) (stride 2: (2,4)): the operand pairs of the two-wide FMAs.  A
+    // pixel therefore lands in at most two places.
     int2 *tab = reinterpret_cast<int2 *>(smem + P.tab_off_words);
+    int *srct = reinterpret_cast<int *>(smem + P.src_off_words);
     for (int q = tid; q < npix; q += nthreads) {
         const int col = q % P.tin_w, t2 = q / P.tin_w;
         const int row = t2 % P.tin_h, im = t2 / P.tin_h;
-        const int gy = gy0 + row, gx = gx0 + col, gn = n0 + im;
-        const bool ok = gn < P.n && gy >= 0 && gy < P.h && gx >= 0 && gx < P.w;
-        tab[q] = make_int2(ok ? ((gn * P.h + gy) * P.w + gx) * P.c_in : -1,
-                           im * P.img_stride + row * P.pitch + col);
+        const int base = im * P.img_stride + row * P.pitch;
+        const int bx = col >> 2, cq = col & 3;
+        int d0 = -1, d1 = -1;
+        auto put = [&](int half, int word, int bxx) {
+            const int o = half * P.half_stride + base + bxx * 4 + word;
+            if (d0 < 0) d0 = o; else d1 = o;
+        };
+        if (bx < LX) {
+            if (cq == 0) put(0, 0, bx);
+            else if (cq == 1) put(0, 2, bx);
+            else if (cq == 2) { put(0, 1, bx); put(1, 0, bx); }
+            else { put(0, 3, bx); if (STRIDE == 1) put(1, 2, bx); }
+        }
+        if (bx >= 1 && bx - 1 < LX) {
+            if (cq == 0) put(1, 1, bx - 1);
+            else if (cq == 1 && STRIDE == 1) put(1, 3, bx - 1);
+        }
+        tab[q] = make_int2(d0, d1);
+        if (!P.use_tma) {
+            const int gy = gy0 + row, gx = gx0 + col, gn = n0 + im;
+            const bool ok = gn < P.n && gy >= 0 && gy < P.h && gx >= 0 && gx < P.w;
+            srct[q] = ok ? ((gn * P.h + gy) * P.w + gx) * P.c_in : -1;
+        }
     }
     for (int i = tid; i < P.wpc * P.J; i += nthreads) soc_s[i] = P.slot_oc[(size_t)blockIdx.y * P.wpc * P.J + i];
-    // Output-pixel table: linear pixel index of (pixel t of lane l), or -1 outside the output.
+    // Output-pixel table: linear pixel index of (sum t of lane l), or -1 outside the output.
+    // Stride 1 keeps a row's four pixels as the pairs (0,2) and (1,3): sum 4*py + 2*h + e is
+    // pixel (py, h + 2*e); stride 2: sum 2*py + e is pixel (py, e).
     int *ptab = reinterpret_cast<int *>(smem + P.ptab_off_words);
     for (int i = tid; i < 32 * T; i += nthreads) {
         const int t = i >> 5, l2 = i & 31;
         const int p_x = l2 & (LX - 1), p_y = (l2 >> P.lx_log) & (LY - 1), p_n = l2 >> (P.lx_log + P.ly_log);
-        const int ox = tx * TW + p_x * BW + (t % BW), oy = ty * TH + p_y * BH + (t / BW), on = n0 + p_n;
+        const int py = STRIDE == 1 ? (t >> 2) : (t >> 1);
+        const int px = STRIDE == 1 ? (((t >> 1) & 1) + 2 * (t & 1)) : (t & 1);
+        const int ox = tx * TW + p_x * BW + px, oy = ty * TH + p_y * BH + py, on = n0 + p_n;
         ptab[i] = (on < P.n && oy < P.ho && ox < P.wo) ? (on * P.ho + oy) * P.wo + ox : -1;
     }
-    __syncthreads();
-
-    const int c_begin = P.chunks_per_split ? (int)blockIdx.z * P.chunks_per_split : 0;
-    const int c_end = P.chunks_per_split ? min(P.n_chunks, c_begin + P.chunks_per_split) : P.n_chunks;
-
-    // Segment offsets of this block's chunks: read once, not on every chunk's critical path.
+    // Segment offsets of this block's chunks.
+    const int32_t *seg_g = P.seg_off + (size_t)b * P.n_chunks * (P.wpc + 1);
+    int *seg = reinterpret_cast<int *>(smem + P.seg_off_words);
     for (int i = tid; i < (c_end - c_begin) * (P.wpc + 1); i += nthreads) seg[i] = seg_g[c_begin * (P.wpc + 1) + i];
-    __syncthreads();
-
-    const int q0 = tid / RP;
-    auto stage_load = [&](int c) {
-        if (P.use_tma) {
-            // one thread hands the tile (a 4-D box of the NHWC tensor, zero-filled outside the
-            // image) and the command segment to the copy engine; an mbarrier counts the bytes
-            if (c < c_end && tid == 0) {
-                const int stage = (c - c_begin) % P.n_stages;
-                const uint32_t raw = smem_base + (uint32_t)(stage * P.stage_words) * 4u;
-                const uint32_t cmd = raw + (uint32_t)P.act_stage_words * 4u;
-                const uint32_t mbar = mbar0 + 8u * stage;
-                const int s0 = seg[(c - c_begin) * (P.wpc + 1)], s1 = seg[(c - c_begin) * (P.wpc + 1) + P.wpc];
-                const uint32_t cmd_bytes = (uint32_t)(s1 - s0 + 2) * (kSlotWords * 4u);
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"((uint32_t)P.box_bytes + cmd_bytes) : "memory");
-                asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-                             ::"r"(raw), "l"(&tmap), "r"(c * P.cc), "r"(gx0), "r"(gy0), "r"(n0), "r"(mbar) : "memory");
-                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                             ::"r"(cmd), "l"(P.slots + (size_t)s0 * kSlotWords), "r"(cmd_bytes), "r"(mbar) : "memory");
-            }
-            return;
-        }
-        if (c < c_end) {
-            const int stage = (c - c_begin) % P.n_stages;
-            const uint32_t act = smem_base + (uint32_t)(stage * P.stage_words) * 4u;
-            // activations: one 32-bit word = E consecutive channels of one pixel
-            const int ic = c * P.cc + rp * E;
-            const bool ic_ok = ic < P.c_in;
-            const uint32_t plane = act + (uint32_t)(rp * P.plane_stride) * 4u;
-            const char *xc = (const char *)P.x + (size_t)(ic_ok ? ic : 0) * XB;
-            if (E == 1 || P.vec_in) {
-                auto copy1 = [&](const int2 t) {
-                    const bool ok = ic_ok && t.x >= 0;
-                    cp_async4(plane + (uint32_t)t.y * 4u, xc + (size_t)(ok ? t.x : 0) * XB, ok ? 4 : 0);
-                };
-                int q = q0;
-                for (; q + 3 * pix_step < npix; q += 4 * pix_step) {      // four independent copies in flight
-                    const int2 t0 = tab[q], t1 = tab[q + pix_step], t2 = tab[q + 2 * pix_step], t3 = tab[q + 3 * pix_step];
-                    copy1(t0); copy1(t1); copy1(t2); copy1(t3);
-                }
-                for (; q < npix; q += pix_step) copy1(tab[q]);
-            } else {
-                // channel count not a multiple of E: assemble the word element by element
-                for (int q = q0; q < npix; q += pix_step) {
-                    const int2 t = tab[q];
-                    const bool ok = ic_ok && t.x >= 0;
-                    const char *src = xc + (size_t)(ok ? t.x : 0) * XB;
-                    uint32_t word = 0;
-                    if (ok) {
-                        for (int k = 0; k < E; ++k) {
-                            if (ic + k < P.c_in) {
-                                if (XB == 2) word |= (uint32_t)((const uint16_t *)src)[k] << (16 * k);
-                                else word |= (uint32_t)((const uint8_t *)src)[k] << (8 * k);
-                            }
-                        }
-                    }
-                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(plane + (uint32_t)t.y * 4u), "r"(word) : "memory");
-                }
-            }
-            // this block's commands for the chunk: one contiguous segment
-            const int s0 = seg[(c - c_begin) * (P.wpc + 1)], s1 = seg[(c - c_begin) * (P.wpc + 1) + P.wpc];
-            const uint32_t cmd = act + (uint32_t)P.act_stage_words * 4u;
-            const uint4 *gsrc = reinterpret_cast<const uint4 *>(P.slots + (size_t)s0 * kSlotWords);
-            const int n16 = (s1 - s0 + 2) * 2;          // two look-ahead slots beyond the segment
-            for (int i = tid; i < n16; i += nthreads) cp_async16(cmd + (uint32_t)i * 16u, gsrc + i);
-        }
-        cp_async_commit();
-    };
-
-    for (int s = 0; s < P.n_stages - 1; ++s) stage_load(c_begin + s);
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_cta = tmem_base_s;
-    const uint32_t tmem_warp = tmem_cta + (((uint32_t)(warp & 3) * 32u) << 16) + (uint32_t)((warp >> 2) * P.cols_per_warp);
-    {
-        const uint32_t z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        for (int c = 0; c < P.cols_per_warp; c += 8) tmem_st8(tmem_warp + c, z);
-        tmem_wait_st();
-    }
-    const uint32_t tmem_int = tmem_warp + (uint32_t)(P.J * T);   // i8 with folding: int32 totals
-
-    // i8: fold the exact fp32 partial sums into the int32 totals and clear them
-    auto fold_partial_sums = [&]() {
-        for (int c8 = 0; c8 < P.J * T; c8 += 8) {
-            uint32_t f[8], q[8];
-            tmem_ld8(tmem_warp + c8, f);
-            tmem_ld8(tmem_int + c8, q);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 8; ++i) { q[i] = (uint32_t)((int)q[i] + __float2int_rn(__uint_as_float(f[i]))); f[i] = 0u; }
-            tmem_st8(tmem_int + c8, q);
-            tmem_st8(tmem_warp + c8, f);
-        }
-        tmem_wait_st();
-    };
-    // i8 without folding (few channels): the fp32 sums are exact integers; convert in place
-    auto sums_to_int = [&]() {
-        for (int c8 = 0; c8 < P.J * T; c8 += 8) {
-            uint32_t f[8];
-            tmem_ld8(tmem_warp + c8, f);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 8; ++i) f[i] = (uint32_t)__float2int_rn(__uint_as_float(f[i]));
-            tmem_st8(tmem_warp + c8, f);
-        }
-        tmem_wait_st();
-    };
-
-    const uint32_t thr_off = (uint32_t)(l_n * P.img_stride + l_y * BH * STRIDE * P.pitch + l_x * BW * STRIDE) * 4u;
     const uint32_t plane_bytes = (uint32_t)P.plane_stride * 4u, pitch_bytes = (uint32_t)P.pitch * 4u;
 
-    // --- main loop over channel chunks --------------------------------------------
-    for (int c = c_begin; c < c_end; ++c) {
-        const int stage = (c - c_begin) % P.n_stages;
-        if (P.use_tma) {
-            if (!abort_s) mbar_wait(mbar0 + 8u * stage, (uint32_t)(((c - c_begin) / P.n_stages) & 1), &abort_s, P.status);
-        } else {
-            if (P.n_stages == 2) cp_async_wait<0>(); else cp_async_wait<1>();
-        }
-        __syncthreads();                       // chunk c has landed; everyone is done with chunk c-1
-        stage_load(c + P.n_stages - 1);
-        const uint32_t act = smem_base + (uint32_t)(stage * P.stage_words) * 4u;
-        uint32_t tile_base = act;
-        if (P.use_tma) {
-            // the copy engine delivered [pixel][channel]; spread it into fp32 channel planes
-            float *ex = reinterpret_cast<float *>(smem + P.exp_off_words);
-            const uint4 *raw = reinterpret_cast<const uint4 *>(smem + stage * P.stage_words);
-            const int vec_per_pix = (P.cc * XB) >> 4;                  // 16-byte pieces per pixel: 1 or 2
-            constexpr int EPV = 16 / XB;                               // elements per piece
-            for (int i = tid; i < npix; i += nthreads) {
-                float *dst = ex + tab[i].y;
-                for (int h2 = 0; h2 < vec_per_pix; ++h2) {
-                    const uint4 wd = raw[i * vec_per_pix + h2];
-                    const uint32_t w4[4] = {wd.x, wd.y, wd.z, wd.w};
-                    float *d2 = dst + (size_t)(h2 * EPV) * P.plane_stride;
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
+    if (producer) {
+        // ===== producer warps: fill stage after stage; warp 0 also drives the copy engine =====
+        const int ptid = pw * 32 + lane;
+        for (int c = c_begin; c < c_end; ++c) {
+            const int k = c - c_begin, s = k % NS;
+            if (k >= NS && !mbar_wait(bar_empty(s), (uint32_t)((k / NS - 1) & 1), &abort_s, P.status)) break;
+            if (pw == 0 && lane == 0) {
+                // this block's commands for the chunk: one contiguous segment, two look-ahead slots beyond it
+                const int s0 = seg[k * (P.wpc + 1)], s1 = seg[k * (P.wpc + 1) + P.wpc];
+                const uint32_t cmd_bytes = (uint32_t)(s1 - s0 + 2) * (kDevSlotWords * 4u);
+                const uint32_t cmd = smem_base + (uint32_t)(P.cmd_off_words + s * P.cmd_stage_words) * 4u;
+                mbar_expect_tx(bar_cmd(s), cmd_bytes);
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(cmd), "l"(P.slots + (size_t)s0 * kDevSlotWords), "r"(cmd_bytes), "r"(bar_cmd(s)) : "memory");
+            }
+            float *pl = reinterpret_cast<float *>(smem + P.plane_off_words + s * P.plane_stage_words);
+            if (P.use_tma) {
+                const int q = c / spb, sub = c - q * spb;
+                const int r = (q - q0) % kRawStages;
+                if ((k == 0 || sub == 0) &&
+                    !mbar_wait(bar_raw(r), (uint32_t)(((q - q0) / kRawStages) & 1), &abort_s, P.status)) break;
+                // the copy engine delivered [pixel][channel]; spread this chunk's channels into the
+                // fp32 operand planes
+                const int len = P.cc * XB, pix_bytes = P.rc * XB;          // bytes per pixel: chunk, box
+                const char *rawb = reinterpret_cast<const char *>(smem + P.raw_off_words + r * P.raw_stage_words) + sub * len;
+                const int ps = P.plane_stride;
+#pragma unroll 2
+                for (int i = ptid; i < npix; i += kProducerWarps * 32) {
+                    const int2 d = tab[i];
+                    float *d0 = pl + d.x, *d1 = pl + (d.y >= 0 ? d.y : d.x);
+                    const char *src = rawb + (size_t)i * pix_bytes;
+                    auto word = [&](uint32_t w, int e) {                   // one 32-bit word = 4 / XB channels from e on
                         if (DT == XGEN_F32) {
-                            d2[k * P.plane_stride] = __uint_as_float(w4[k]);
+                            const float v = __uint_as_float(w);
+                            d0[e * ps] = v; d1[e * ps] = v;
                         } else if (DT == XGEN_F16_F32ACC) {
-                            const __half2 h2v = *reinterpret_cast<const __half2 *>(&w4[k]);
-                            d2[(2 * k) * P.plane_stride] = __low2float(h2v);
-                            d2[(2 * k + 1) * P.plane_stride] = __high2float(h2v);
+                            const __half2 hv = *reinterpret_cast<const __half2 *>(&w);
+                            const float v0 = __low2float(hv), v1 = __high2float(hv);
+                            d0[e * ps] = v0; d1[e * ps] = v0;
+                            d0[(e + 1) * ps] = v1; d1[(e + 1) * ps] = v1;
                         } else {
 #pragma unroll
-                            for (int bq = 0; bq < 4; ++bq) d2[(4 * k + bq) * P.plane_stride] = (float)((w4[k] >> (8 * bq)) & 0xFFu);
+                            for (int bq = 0; bq < 4; ++bq) {
+                                const float v = (float)((w >> (8 * bq)) & 0xFFu);
+                                d0[(e + bq) * ps] = v; d1[(e + bq) * ps] = v;
+                            }
                         }
-                    }
-                }
-            }
-            __syncthreads();
-            tile_base = smem_base + (uint32_t)P.exp_off_words * 4u;
-        } else if (DT != XGEN_F32) {
-            // widen the staged words to fp32 planes (exact for fp16 and for uint8)
-            float *ex = reinterpret_cast<float *>(smem + P.exp_off_words);
-            const int quads = P.plane_stride >> 2;             // plane_stride is a multiple of 4
-            for (int r = 0; r < RP; ++r) {
-                const uint4 *raw = reinterpret_cast<const uint4 *>(smem + stage * P.stage_words + r * P.plane_stride);
-                for (int i = tid; i < quads; i += nthreads) {
-                    const uint4 wd = raw[i];
-                    const uint32_t w4[4] = {wd.x, wd.y, wd.z, wd.w};
-                    if (DT == XGEN_F16_F32ACC) {
-                        float lo[4], hi[4];
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const __half2 h2 = *reinterpret_cast<const __half2 *>(&w4[k]);
-                            lo[k] = __low2float(h2); hi[k] = __high2float(h2);
+                    };
+                    constexpr int EPW = 4 / XB;                            // channels per word
+                    if (len >= 16) {
+                        for (int h2 = 0; h2 < (len >> 4); ++h2) {
+                            const uint4 wd = *reinterpret_cast<const uint4 *>(src + 16 * h2);
+                            word(wd.x, (4 * h2) * EPW); word(wd.y, (4 * h2 + 1) * EPW);
+                            word(wd.z, (4 * h2 + 2) * EPW); word(wd.w, (4 * h2 + 3) * EPW);
                         }
-                        reinterpret_cast<float4 *>(ex + (2 * r) * P.plane_stride)[i] = make_float4(lo[0], lo[1], lo[2], lo[3]);
-                        reinterpret_cast<float4 *>(ex + (2 * r + 1) * P.plane_stride)[i] = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                    } else if (len == 8) {
+                        const uint2 wd = *reinterpret_cast<const uint2 *>(src);
+                        word(wd.x, 0); word(wd.y, EPW);
                     } else {
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            reinterpret_cast<float4 *>(ex + (4 * r + k) * P.plane_stride)[i] =
-                                make_float4((float)((w4[0] >> (8 * k)) & 0xFFu), (float)((w4[1] >> (8 * k)) & 0xFFu),
-                                            (float)((w4[2] >> (8 * k)) & 0xFFu), (float)((w4[3] >> (8 * k)) & 0xFFu));
+                        word(*reinterpret_cast<const uint32_t *>(src), 0);
                     }
                 }
-            }
-            __syncthreads();
-            tile_base = smem_base + (uint32_t)P.exp_off_words * 4u;
-        }
-        const int s0 = seg[(c - c_begin) * (P.wpc + 1)], sg = seg[(c - c_begin) * (P.wpc + 1) + warp];
-        uint32_t sp = act + (uint32_t)P.act_stage_words * 4u + (uint32_t)(sg - s0) * 32u;
-        run_commands<STRIDE, NP>(sp, tile_base + thr_off, plane_bytes, pitch_bytes, tmem_warp);
-        if (DT == XGEN_I8_I32 && P.fold && ((c - c_begin + 1) % P.flush_chunks == 0)) fold_partial_sums();
-    }
-    cp_async_wait<0>();
-    if (DT == XGEN_I8_I32) { if (P.fold) fold_partial_sums(); else sums_to_int(); }
-
-    // --- epilogue: bias + ReLU + convert, straight from tensor memory to NHWC -------
-    // A group is a run of J consecutive output channels, so for one pixel a thread holds
-    // 8 adjacent channels per 8 filter slots: 32 bytes (16 for fp16) it can store as one
-    // piece.  No shared memory, no block-wide barrier: every warp drains on its own.
-    const int *soc = soc_s + warp * P.J;
-    const uint32_t tmem_res = (DT == XGEN_I8_I32 && P.fold) ? tmem_int : tmem_warp;
-    const int oc_base = soc[0];
-    if (oc_base >= 0) {
-        const int *pt = ptab + lane;
-        uint32_t *const part = P.partial ? P.partial + (size_t)blockIdx.z * P.out_elems : nullptr;
-        for (int j0 = 0; j0 < P.J; j0 += 8) {
-            const int oc0 = oc_base + j0;
-            if (oc0 >= P.c_out) break;
-            const int nv = min(8, P.c_out - oc0);                 // valid channels of this piece
-            uint32_t bb[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) bb[k] = (P.bias && !part && k < nv) ? ((const uint32_t *)P.bias)[oc0 + k] : 0u;
-            for (int t0 = 0; t0 < T; t0 += 4) {
-                uint32_t v[8][4];
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    if (j0 + k < P.J) tmem_ld4(tmem_res + (j0 + k) * T + t0, v[k]);
-                    else { v[k][0] = v[k][1] = v[k][2] = v[k][3] = 0u; }
+                __syncwarp();
+                if ((sub == spb - 1 || c == c_end - 1) && q + kRawStages <= q_end) {
+                    // the box is refilled once every producer warp has read its share of it
+                    if (lane == 0) mbar_arrive(bar_rawfree(r));
+                    if (pw == 0) {
+                        if (!mbar_wait(bar_rawfree(r), (uint32_t)(((q - q0) / kRawStages) & 1), &abort_s, P.status)) break;
+                        if (lane == 0) {
+                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // reads of the box before its reuse
+                            issue_box(q + kRawStages);
+                        }
+                    }
                 }
+            } else {
+                // plain loads: any channel count, any alignment
+                const char *xb = (const char *)P.x;
+                const int ic0 = c * P.cc;
+                for (int i = ptid; i < npix; i += kProducerWarps * 32) {
+                    const int2 d = tab[i];
+                    const int src = srct[i];
+                    float *d0 = pl + d.x, *d1 = pl + (d.y >= 0 ? d.y : d.x);
+#pragma unroll 4
+                    for (int e = 0; e < P.cc; ++e) {
+                        const bool ok = src >= 0 && ic0 + e < P.c_in;
+                        const float v = ok ? load_widened<DT>(xb + (size_t)(src + ic0 + e) * XB) : 0.f;
+                        d0[e * P.plane_stride] = v; d1[e * P.plane_stride] = v;
+                    }
+                }
+                __syncwarp();
+            }
+            if (lane == 0) mbar_arrive(bar_full(s));
+        }
+    } else {
+        // ===== consumer warps ===========================================================
+        const uint32_t tmem_warp = tmem_cta + (((uint32_t)(warp & 3) * 32u) << 16) + (uint32_t)((warp >> 2) * P.cols_per_warp);
+        {
+            const uint32_t z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            for (int c = 0; c < P.cols_per_warp; c += 8) tmem_st8(tmem_warp + c, z);
+            tmem_wait_st();
+        }
+        const uint32_t tmem_int = tmem_warp + (uint32_t)(P.J * T);   // i8 with folding: int32 totals
+
+        // i8: fold the exact fp32 partial sums into the int32 totals and clear them
+        auto fold_partial_sums = [&]() {
+            for (int c8 = 0; c8 < P.J * T; c8 += 8) {
+                uint32_t f[8], q[8];
+                tmem_ld8(tmem_warp + c8, f);
+                tmem_ld8(tmem_int + c8, q);
                 tmem_wait_ld();
 #pragma unroll
-                for (int tt = 0; tt < 4; ++tt) {
-                    const int pidx = pt[(t0 + tt) * 32];
-                    if (pidx < 0) continue;
-                    const size_t o = (size_t)pidx * P.c_out + oc0;
-                    uint32_t r[8];
-                    if (part) {
+                for (int i = 0; i < 8; ++i) { q[i] = (uint32_t)((int)q[i] + __float2int_rn(__uint_as_float(f[i]))); f[i] = 0u; }
+                tmem_st8(tmem_int + c8, q);
+                tmem_st8(tmem_warp + c8, f);
+            }
+            tmem_wait_st();
+        };
+        // i8 without folding (few channels): the fp32 sums are exact integers; convert in place
+        auto sums_to_int = [&]() {
+            for (int c8 = 0; c8 < P.J * T; c8 += 8) {
+                uint32_t f[8];
+                tmem_ld8(tmem_warp + c8, f);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) f[i] = (uint32_t)__float2int_rn(__uint_as_float(f[i]));
+                tmem_st8(tmem_warp + c8, f);
+            }
+            tmem_wait_st();
+        };
+
+        const uint32_t thr_off = (uint32_t)(l_n * P.img_stride + l_y * BH * STRIDE * P.pitch + l_x * 4) * 4u;
+        const uint32_t half_bytes = (uint32_t)P.half_stride * 4u;
+
+        // --- main loop over channel chunks --------------------------------------------
+        for (int c = c_begin; c < c_end; ++c) {
+            const int k = c - c_begin, s = k % NS;
+            const uint32_t par = (uint32_t)((k / NS) & 1);
+            if (!mbar_wait(bar_full(s), par, &abort_s, P.status)) break;
+            if (!mbar_wait(bar_cmd(s), par, &abort_s, P.status)) break;
+            const int s0 = seg[k * (P.wpc + 1)], sg = seg[k * (P.wpc + 1) + warp];
+            const uint32_t sp = smem_base + (uint32_t)(P.cmd_off_words + s * P.cmd_stage_words) * 4u +
+                                (uint32_t)(sg - s0) * (kDevSlotWords * 4u);
+            const uint32_t base_a = smem_base + (uint32_t)(P.plane_off_words + s * P.plane_stage_words) * 4u + thr_off;
+            run_commands<STRIDE, NP>(sp, base_a, plane_bytes, pitch_bytes, tmem_warp, base_a + half_bytes);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty(s));
+            if (DT == XGEN_I8_I32 && P.fold && ((k + 1) % P.flush_chunks == 0)) fold_partial_sums();
+        }
+        if (DT == XGEN_I8_I32) { if (P.fold) fold_partial_sums(); else sums_to_int(); }
+
+        // --- epilogue: bias + ReLU + convert, straight from tensor memory to NHWC -------
+        // A group is a run of J consecutive output channels, so for one pixel a thread holds
+        // 8 adjacent channels per 8 filter slots: 32 bytes (16 for fp16) it can store as one
+        // piece.  No shared memory, no block-wide barrier: every warp drains on its own.
+        const int *soc = soc_s + warp * P.J;
+        const uint32_t tmem_res = (DT == XGEN_I8_I32 && P.fold) ? tmem_int : tmem_warp;
+        const int oc_base = soc[0];
+        if (oc_base >= 0) {
+            const int *pt = ptab + lane;
+            uint32_t *const part = P.partial ? P.partial + (size_t)blockIdx.z * P.out_elems : nullptr;
+            const int K8 = (P.J + 7) >> 3;
+            uint32_t *const wrow = P.ws ? P.ws + ((((size_t)item * P.n_splits + blockIdx.z) * (size_t)(P.wpc * K8 * T)
+                                                   + (size_t)warp * K8 * T) * 32 + lane) * 8 : nullptr;
+            for (int j0 = 0; j0 < P.J; j0 += 8) {
+                const int oc0 = oc_base + j0;
+                if (oc0 >= P.c_out) break;
+                const int nv = min(8, P.c_out - oc0);                 // valid channels of this piece
+                uint32_t bb[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) bb[k] = (P.bias && !part && !wrow && k < nv) ? ((const uint32_t *)P.bias)[oc0 + k] : 0u;
+                for (int t0 = 0; t0 < T; t0 += 4) {
+                    uint32_t v[8][4];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        if (j0 + k < P.J) tmem_ld4(tmem_res + (j0 + k) * T + t0, v[k]);
+                        else { v[k][0] = v[k][1] = v[k][2] = v[k][3] = 0u; }
+                    }
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int tt = 0; tt < 4; ++tt) {
+                        uint32_t r[8];
 #pragma unroll
                         for (int k = 0; k < 8; ++k) r[k] = v[k][tt];
-                    } else if (DT == XGEN_I8_I32) {
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) { int q = (int)v[k][tt] + (int)bb[k]; if (P.relu) q = max(q, 0); r[k] = (uint32_t)q; }
-                    } else {
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) { float q = __uint_as_float(v[k][tt]) + __uint_as_float(bb[k]); if (P.relu) q = fmaxf(q, 0.f); r[k] = __float_as_uint(q); }
-                    }
-                    if (part || DT != XGEN_F16_F32ACC) {
-                        uint32_t *dst = (part ? part : (uint32_t *)P.y) + o;
-                        if (nv == 8 && P.vec_out == 8) {
+                        if (wrow) {
+                            // raw sums, one 1 KB row per warp and store: lanes side by side
+                            uint32_t *dst = wrow + (size_t)(((j0 >> 3) * T + t0 + tt) * 32) * 8;
                             asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
-                        } else if (nv == 8 && P.vec_out == 4) {
-                            *reinterpret_cast<uint4 *>(dst) = make_uint4(r[0], r[1], r[2], r[3]);
-                            *reinterpret_cast<uint4 *>(dst + 4) = make_uint4(r[4], r[5], r[6], r[7]);
-                        } else {
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) if (k < nv) dst[k] = r[k];
+                            continue;
                         }
-                    } else {
-                        __half *dst = (__half *)P.y + o;
-                        if (nv == 8 && P.vec_out >= 4 && (P.c_out & 7) == 0) {
-                            uint4 pk;
-                            __half2 h0 = __floats2half2_rn(__uint_as_float(r[0]), __uint_as_float(r[1]));
-                            __half2 h1 = __floats2half2_rn(__uint_as_float(r[2]), __uint_as_float(r[3]));
-                            __half2 h2 = __floats2half2_rn(__uint_as_float(r[4]), __uint_as_float(r[5]));
-                            __half2 h3 = __floats2half2_rn(__uint_as_float(r[6]), __uint_as_float(r[7]));
-                            pk.x = *reinterpret_cast<uint32_t *>(&h0); pk.y = *reinterpret_cast<uint32_t *>(&h1);
-                            pk.z = *reinterpret_cast<uint32_t *>(&h2); pk.w = *reinterpret_cast<uint32_t *>(&h3);
-                            *reinterpret_cast<uint4 *>(dst) = pk;
-                        } else {
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) if (k < nv) dst[k] = __float2half_rn(__uint_as_float(r[k]));
-                        }
+                        const int pidx = pt[(t0 + tt) * 32];
+                        if (pidx < 0) continue;
+                        if (part) store_piece<XGEN_F32>(P, r, bb, false, part, (size_t)pidx * P.c_out + oc0, nv, true);
+                        else store_piece<DT>(P, r, bb, P.relu, P.y, (size_t)pidx * P.c_out + oc0, nv, false);
                     }
                 }
+            }
+        }
+    }
+
+    if (P.ws) {
+        // ===== split run: wait for the other splits of this item, then reduce a share =====
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t *cnt = P.counters + item;
+            asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(cnt) : "memory");
+            bool ok = false;
+            for (int it = 0; it < 2000000 && !abort_s; ++it) {
+                uint32_t v;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(cnt) : "memory");
+                if ((int)(v - P.target) >= 0) { ok = true; break; }
+                __nanosleep(100);
+            }
+            if (!ok) { abort_s = 1; if (P.status) atomicExch(P.status, 1); }
+        }
+        __syncthreads();
+        if (!abort_s) {
+            const int K8 = (P.J + 7) >> 3;
+            const int R = P.wpc * K8 * T, S = P.n_splits, nwarps = nthreads >> 5;
+            const uint32_t *base = P.ws + (size_t)item * S * R * 256;
+            for (int row = (int)blockIdx.z + S * warp; row < R; row += S * nwarps) {
+                const int t = row % T, k8 = (row / T) % K8, w = row / (T * K8);
+                const int ocb = soc_s[w * P.J];
+                const int oc0 = ocb + k8 * 8;
+                const int pidx = ptab[t * 32 + lane];
+                if (ocb < 0 || oc0 >= P.c_out || pidx < 0) continue;
+                const int nv = min(8, P.c_out - oc0);
+                uint32_t acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                auto add8 = [&](const uint4 &lo, const uint4 &hi) {
+                    const uint32_t q[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        if (DT == XGEN_I8_I32) acc[k] = (uint32_t)((int)acc[k] + (int)q[k]);
+                        else acc[k] = __float_as_uint(__uint_as_float(acc[k]) + __uint_as_float(q[k]));
+                    }
+                };
+                const size_t zstride = (size_t)R * 64;                // uint4 per split
+                const uint4 *src = reinterpret_cast<const uint4 *>(base + ((size_t)row * 32 + lane) * 8);
+                int z = 0;
+                for (; z + 4 <= S; z += 4) {                          // four splits in flight; summed in order 0, 1, ...
+                    uint4 lo[4], hi[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) { lo[u] = __ldcg(src + (z + u) * zstride); hi[u] = __ldcg(src + (z + u) * zstride + 1); }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) add8(lo[u], hi[u]);
+                }
+                for (; z < S; ++z) add8(__ldcg(src + z * zstride), __ldcg(src + z * zstride + 1));
+                uint32_t bb[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) bb[k] = (P.bias && k < nv) ? ((const uint32_t *)P.bias)[oc0 + k] : 0u;
+                store_piece<DT>(P, acc, bb, P.relu, P.y, (size_t)pidx * P.c_out + oc0, nv, false);
             }
         }
     }
@@ -561,16 +663,16 @@ static inline int pixels_per_thread(int stride) { return 4 * pixels_per_thread_x
 
 struct Geometry {
     int lx_log, ly_log, ln_log, tiles_x, tiles_y, tiles_n;
-    int tin_w, tin_h, pitch, img_stride, plane_stride;
+    int tin_w, tin_h, pitch, img_stride, half_stride, plane_stride;
 };
 
-// Worst bank multiplicity of the 128-bit patch-row load for a candidate pitch.
+// Worst bank multiplicity of a thread's 128-bit patch-row load for a candidate layout:
+// a lane reads 4 words at (image, its first tile row, its lane column x 4).
 static int row_load_conflicts(int stride, int lx_log, int ly_log, int pitch, int img_stride) {
     const int LX = 1 << lx_log, LY = 1 << ly_log;
-    const int bw = pixels_per_thread_x(stride);
     auto addr = [&](int lane) {
         int x = lane & (LX - 1), y = (lane >> lx_log) & (LY - 1), n = lane >> (lx_log + ly_log);
-        return n * img_stride + y * 4 * stride * pitch + x * bw * stride;   // words
+        return n * img_stride + y * 4 * stride * pitch + x * 4;   // words
     };
     int worst = 0;
     for (int ph = 0; ph < 4; ++ph) {                      // 128-bit accesses: 8 lanes per wavefront
@@ -604,17 +706,20 @@ static Geometry choose_geometry(int n, int ho, int wo, int stride) {
     best.tiles_x = (wo + TW - 1) / TW; best.tiles_y = (ho + TH - 1) / TH; best.tiles_n = (n + LN - 1) / LN;
     best.tin_w = stride == 1 ? TW + 2 : 2 * TW + 1;
     best.tin_h = stride == 1 ? TH + 2 : 2 * TH + 1;
-    const int align = 4;                                  // 16-byte aligned patch rows
-    int p0 = (best.tin_w + align - 1) / align * align, best_p = p0, best_c = 1 << 30;
-    for (int p = p0; p <= p0 + 8; p += align) {
-        int c = row_load_conflicts(stride, best.lx_log, best.ly_log, p, best.tin_h * p);
-        if (c < best_c) { best_c = c; best_p = p; }
-    }
+    // One half of a plane row holds 4 words per lane column; pad the row and the image so
+    // that the 128-bit loads of a quarter warp fall into distinct banks.
+    const int p0 = 4 << best.lx_log;
+    int best_p = p0, best_i = best.tin_h * p0, best_c = 1 << 30;
+    for (int p = p0; p <= p0 + 12; p += 4)
+        for (int ipad = 0; ipad <= (LN > 1 ? 28 : 0); ipad += 4) {
+            const int istr = best.tin_h * p + ipad;
+            const int c = row_load_conflicts(stride, best.lx_log, best.ly_log, p, istr);
+            if (c < best_c) { best_c = c; best_p = p; best_i = istr; }
+        }
     best.pitch = best_p;
-    best.img_stride = best.tin_h * best.pitch;
-    int ps = LN * best.img_stride;
-    while ((ps & 31) != 4) ++ps;                          // planes 4 banks apart: conflict-free staging writes
-    best.plane_stride = ps;
+    best.img_stride = best_i;
+    best.half_stride = LN * best.img_stride;
+    best.plane_stride = 2 * best.half_stride;
     return best;
 }
 
@@ -630,8 +735,11 @@ struct xgen_patconv_packed {
     int32_t *d_slot_oc = nullptr;
     // set by xgen_patconv_plan: split the channel chunks of this shape across blocks
     int plan_n = 0, plan_h = 0, plan_w = 0, plan_splits = 1, plan_cps = 0;
-    uint32_t *d_partial = nullptr;
+    uint32_t *d_partial = nullptr;      // partial sums of the planned split, reduced inside the kernel
     size_t partial_bytes = 0;
+    uint32_t *d_counters = nullptr;     // one arrival counter per (tile, filter block) of the planned shape
+    size_t counter_bytes = 0;
+    mutable std::atomic<uint32_t> split_seq{0};   // planned split launches so far (counters only grow)
     int *d_status = nullptr;            // set by a kernel whose bounded wait ran out
     // device staging buffers of xgen_patconv_run_host, kept between calls (grow only)
     mutable std::mutex host_mu;
@@ -647,19 +755,27 @@ static void free_device_layout(xgen_patconv_packed *h) {
     h->d_slots = nullptr; h->d_seg_off = nullptr; h->d_slot_oc = nullptr; h->d_status = nullptr;
 }
 
-// Upload the host layout; the device must be current.
+// Upload the host layout; the device must be current.  On the device a command slot is
+// 48 bytes: {opcode, operand, -, -, w0, w0, w1, w1, w2, w2, w3, w3}; every weight twice, so
+// that a 64-bit load yields the operand pair of a two-wide FMA.
 static xgen_status upload_layout(xgen_patconv_packed *h) {
     const PackedHost &p = h->host;
     free_device_layout(h);
-    // two spare slots: harmless over-read room for 16-byte copies
-    size_t sb = (p.slots.size() + 2 * kSlotWords) * 4, gb = p.seg_off.size() * 4, ob = p.slot_oc.size() * 4;
+    const size_t n_slots = p.slots.size() / kSlotWords;
+    std::vector<uint32_t> dev((n_slots + 2) * kDevSlotWords, 0u);    // two spare slots: look-ahead room
+    for (size_t i = 0; i < n_slots; ++i) {
+        const uint32_t *src = &p.slots[i * kSlotWords];
+        uint32_t *dst = &dev[i * kDevSlotWords];
+        dst[0] = src[0]; dst[1] = src[1];
+        for (int k = 0; k < 4; ++k) dst[4 + 2 * k] = dst[5 + 2 * k] = src[4 + k];
+    }
+    const size_t sb = dev.size() * 4, gb = p.seg_off.size() * 4, ob = p.slot_oc.size() * 4;
     cudaError_t e = cudaMalloc(&h->d_slots, sb);
     if (e == cudaSuccess) e = cudaMalloc(&h->d_seg_off, gb);
     if (e == cudaSuccess) e = cudaMalloc(&h->d_slot_oc, ob);
     if (e == cudaSuccess) e = cudaMalloc(&h->d_status, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(int));
-    if (e == cudaSuccess) e = cudaMemset(h->d_slots, 0, sb);
-    if (e == cudaSuccess) e = cudaMemcpy(h->d_slots, p.slots.data(), p.slots.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(h->d_slots, dev.data(), sb, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(h->d_seg_off, p.seg_off.data(), gb, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(h->d_slot_oc, p.slot_oc.data(), ob, cudaMemcpyHostToDevice);
     if (e != cudaSuccess) {
@@ -701,33 +817,35 @@ static EncodeTiledFn encode_tiled_fn() {
 }
 
 template <int DT, int STRIDE>
-static cudaError_t launch_np(int np, dim3 grid, dim3 block, size_t smem, cudaStream_t st, const KParams &kp, const CUtensorMap &tm) {
-    auto go = [&](auto kern) -> cudaError_t {
-        // the opt-in to large dynamic shared memory is per function and per device: do it once
-        static std::mutex mu;
-        static std::vector<std::pair<const void *, int>> done;
-        {
-            std::lock_guard<std::mutex> lock(mu);
-            int dev = 0;
-            cudaGetDevice(&dev);
-            const std::pair<const void *, int> key((const void *)kern, dev);
-            bool found = false;
-            for (const auto &k : done) found = found || k == key;
-            if (!found) {
-                cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMaxDynamic);
-                if (e != cudaSuccess) return log_cuda(e, "cudaFuncSetAttribute");
-                done.push_back(key);
-            }
-        }
-        kern<<<grid, block, smem, st>>>(kp, tm);
-        return log_cuda(cudaGetLastError(), "kernel launch");
-    };
+static const void *kernel_np(int np) {
     switch (np) {
-        case 4: return go(patconv_kernel<DT, STRIDE, 4>);
-        case 8: return go(patconv_kernel<DT, STRIDE, 8>);
-        case 12: return go(patconv_kernel<DT, STRIDE, 12>);
-        default: return go(patconv_kernel<DT, STRIDE, 126>);
+        case 4: return (const void *)patconv_kernel<DT, STRIDE, 4>;
+        case 8: return (const void *)patconv_kernel<DT, STRIDE, 8>;
+        case 12: return (const void *)patconv_kernel<DT, STRIDE, 12>;
+        default: return (const void *)patconv_kernel<DT, STRIDE, 126>;
     }
+}
+
+// The kernel instance of a packed layer.
+static const void *kernel_for(const PackedHost &p) {
+    if (p.dtype == XGEN_F32) return p.stride == 1 ? kernel_np<XGEN_F32, 1>(p.np) : kernel_np<XGEN_F32, 2>(p.np);
+    if (p.dtype == XGEN_F16_F32ACC) return p.stride == 1 ? kernel_np<XGEN_F16_F32ACC, 1>(p.np) : kernel_np<XGEN_F16_F32ACC, 2>(p.np);
+    return p.stride == 1 ? kernel_np<XGEN_I8_I32, 1>(p.np) : kernel_np<XGEN_I8_I32, 2>(p.np);
+}
+
+// The opt-in to large dynamic shared memory is per function and per device: do it once.
+static cudaError_t allow_large_smem(const void *kern) {
+    static std::mutex mu;
+    static std::vector<std::pair<const void *, int>> done;
+    std::lock_guard<std::mutex> lock(mu);
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const std::pair<const void *, int> key(kern, dev);
+    for (const auto &k : done) if (k == key) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMaxDynamic);
+    if (e != cudaSuccess) return log_cuda(e, "cudaFuncSetAttribute");
+    done.push_back(key);
+    return cudaSuccess;
 }
 
 static int next_pow2(int v) { int p = 32; while (p < v) p <<= 1; return p; }
@@ -767,6 +885,13 @@ xgen_status xgen_patconv_pack(const xgen_patconv_desc *desc, const void *dense_w
         if (const char *e = getenv("XGEN_PATCONV_CC")) { int v = atoi(e); if (v == 2 || v == 4 || v == 8 || v == 16) cfg.channels_per_chunk = v; }
         if (desc->dtype == XGEN_I8_I32 && cfg.channels_per_chunk < 4) cfg.channels_per_chunk = 4;
         st = pack_host(*desc, dense_w_host, pattern_id_host, cfg, h->host);
+        // A stage of the kernel's pipeline holds the commands of one chunk for the whole
+        // block: halve the chunk until the longest segment fits the command buffer.
+        while (st == XGEN_OK && !getenv("XGEN_PATCONV_CC") && cfg.channels_per_chunk > 4 &&
+               (size_t)h->host.max_seg_slots * kDevSlotBytes > kCmdStageBudget) {
+            cfg.channels_per_chunk /= 2;
+            st = build_layout(h->host, cfg);
+        }
     } catch (const std::bad_alloc &) {
         st = XGEN_ERR_ALLOC;
     }
@@ -787,6 +912,7 @@ void xgen_patconv_free(xgen_patconv_packed *h) {
     if (!h) return;
     free_device_layout(h);
     if (h->d_partial) cudaFree(h->d_partial);
+    if (h->d_counters) cudaFree(h->d_counters);
     if (h->d_hx) cudaFree(h->d_hx);
     if (h->d_hy) cudaFree(h->d_hy);
     if (h->d_hb) cudaFree(h->d_hb);
@@ -817,66 +943,6 @@ xgen_status xgen_patconv_view(const xgen_patconv_packed *h, xgen_patconv_host_vi
     return XGEN_OK;
 }
 
-xgen_status xgen_patconv_plan(xgen_patconv_packed *h, int32_t n, int32_t hh, int32_t ww) {
-    if (!h) return XGEN_ERR_INVALID_ARG;
-    if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
-    if (h->device < 0) return XGEN_ERR_CUDA;
-    const PackedHost &p = h->host;
-    const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
-    if ((int64_t)n * ho * wo * p.c_out > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
-    const Geometry g = choose_geometry(n, ho, wo, p.stride);
-    const int64_t ctas = (int64_t)g.tiles_x * g.tiles_y * g.tiles_n * p.n_blocks;
-    const int flush_chunks_plan = 16777216 / (p.cc * 4 * 32640);
-    const int cols_per_warp = p.J * pixels_per_thread(p.stride) * ((p.dtype == XGEN_I8_I32 && p.n_chunks > flush_chunks_plan) ? 2 : 1);
-    const int warp_slots = 4 * (512 / cols_per_warp);                 // per SM, set by tensor memory
-    int sms = 148;
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
-    const size_t out_bytes = (size_t)n * ho * wo * p.c_out * 4;
-    // Pick the split count with a small cost model (microseconds): blocks run in waves of
-    // (SMs x blocks per SM); a block costs a fixed prologue + epilogue plus its share of the
-    // multiply-adds at the rate one busy SM sustains; a split adds one write and one read of
-    // the fp32 output per part, plus a second launch.
-    const double blocks_per_wave = (double)sms * (warp_slots / p.wpc > 0 ? warp_slots / p.wpc : 1);
-    const double macs_per_block = 4.0 * (double)p.stats.kernels_surviving * (double)n * ho * wo / (double)ctas;
-    const double t_work = macs_per_block / 72e3, t_fixed = 10.0;      // 72 GMAC/s per SM, 10 us
-    auto estimate = [&](int64_t k) {
-        const int cps_k = (int)((p.n_chunks + k - 1) / k);
-        const int64_t parts = (p.n_chunks + cps_k - 1) / cps_k;
-        const double waves = std::ceil((double)(ctas * parts) / blocks_per_wave);
-        double t = waves * (t_fixed + t_work / (double)parts);
-        if (parts > 1) t += 3.0 + ((double)parts * 2.0 + 1.0) * (double)out_bytes / 4e6;   // 4 TB/s
-        return t;
-    };
-    int64_t splits = 1;
-    double best_t = estimate(1);
-    for (int64_t k = 2; k <= p.n_chunks; ++k) {
-        const double t = estimate(k);
-        if (t < 0.9 * best_t || (splits > 1 && t < best_t)) { best_t = t; splits = k; }
-    }
-    if (const char *e = getenv("XGEN_PATCONV_SPLIT")) { int v = atoi(e); if (v >= 1) splits = v < p.n_chunks ? v : p.n_chunks; }
-    if (splits < 1) splits = 1;
-    const int cps = (int)((p.n_chunks + splits - 1) / splits);
-    splits = (p.n_chunks + cps - 1) / cps;
-    int prev = 0;
-    if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
-    xgen_status rs = XGEN_OK;
-    if (cudaDeviceSynchronize() != cudaSuccess) rs = XGEN_ERR_CUDA;
-    if (rs == XGEN_OK && splits > 1) {
-        const size_t need = out_bytes * (size_t)splits;
-        if (need > h->partial_bytes) {
-            if (h->d_partial) cudaFree(h->d_partial);
-            h->d_partial = nullptr; h->partial_bytes = 0;
-            if (cudaMalloc(&h->d_partial, need) != cudaSuccess) { cudaGetLastError(); rs = XGEN_ERR_ALLOC; }
-            else h->partial_bytes = need;
-        }
-    }
-    cudaSetDevice(prev);
-    if (rs != XGEN_OK) { h->plan_splits = 1; h->plan_n = 0; return rs; }
-    h->plan_n = n; h->plan_h = hh; h->plan_w = ww;
-    h->plan_splits = (int)splits; h->plan_cps = cps;
-    return XGEN_OK;
-}
-
 xgen_status xgen_patconv_last_status(const xgen_patconv_packed *h, void *stream) {
     if (!h) return XGEN_ERR_INVALID_ARG;
     cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
@@ -888,6 +954,9 @@ xgen_status xgen_patconv_last_status(const xgen_patconv_packed *h, void *stream)
         if (cudaMemcpy(&flag, h->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return XGEN_ERR_CUDA;
         if (flag) {
             cudaMemset(h->d_status, 0, sizeof(int));
+            // a run that gave up may have left the arrival counters of a split half way
+            if (h->d_counters) cudaMemset(h->d_counters, 0, h->counter_bytes);
+            h->split_seq.store(0);
             return XGEN_ERR_TIMEOUT;
         }
     }
@@ -895,6 +964,94 @@ xgen_status xgen_patconv_last_status(const xgen_patconv_packed *h, void *stream)
 }
 
 }  // extern "C"
+
+// Everything about a launch that depends only on the layer and the input shape: tile
+// geometry, shared-memory layout, tensor-memory columns.
+struct Layout {
+    Geometry g;
+    KParams kp;          // pointers, split and tensor-map fields left empty
+    size_t smem;
+    int items;           // (tile, filter block) pairs = blocks of an unsplit launch
+};
+
+static xgen_status make_layout(const PackedHost &p, int n, int hh, int ww, bool y_aligned32, bool tma_ok, Layout &L) {
+    const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
+    const Geometry g = choose_geometry(n, ho, wo, p.stride);
+    L.g = g;
+    KParams kp{};
+    kp.n = n; kp.h = hh; kp.w = ww; kp.ho = ho; kp.wo = wo; kp.c_in = p.c_in; kp.c_out = p.c_out;
+    kp.J = p.J; kp.wpc = p.wpc; kp.cc = p.cc; kp.n_chunks = p.n_chunks;
+    kp.lx_log = g.lx_log; kp.ly_log = g.ly_log; kp.ln_log = g.ln_log;
+    kp.tiles_x = g.tiles_x; kp.tiles_y = g.tiles_y;
+    kp.tin_w = g.tin_w; kp.tin_h = g.tin_h;
+    kp.pitch = g.pitch; kp.img_stride = g.img_stride; kp.plane_stride = g.plane_stride;
+    kp.half_stride = g.half_stride;
+    const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
+    const int npix_box = (g.tin_w * g.tin_h) << g.ln_log;
+    // A box carries at least 16 bytes of channels per pixel; a chunk may be a part of it.
+    // The copy engine needs 16-byte multiples in every global stride.
+    kp.rc = p.cc * xb >= 16 ? p.cc : 16 / xb;
+    kp.use_tma = tma_ok && ((p.cc * xb) % 4 == 0) && (((size_t)p.c_in * xb) % 16 == 0) && g.tin_w <= 256 && g.tin_h <= 256 &&
+                 !getenv("XGEN_PATCONV_NO_TMA");
+    kp.box_bytes = npix_box * kp.rc * xb;
+    // widest aligned store per 8-channel piece: 8 words (32-byte aligned rows), 4, or scalar
+    kp.vec_out = ((p.c_out % 8) == 0 && y_aligned32) ? 8 : ((p.c_out % 4) == 0 ? 4 : 0);
+    const bool is_i8 = p.dtype == XGEN_I8_I32;
+    const int T = pixels_per_thread(p.stride);
+    kp.flush_chunks = 16777216 / (p.cc * 4 * 32640);
+    if (kp.flush_chunks < 1) return XGEN_ERR_UNSUPPORTED;
+    kp.fold = (is_i8 && p.n_chunks > kp.flush_chunks) ? 1 : 0;
+    kp.cols_per_warp = p.J * T * (kp.fold ? 2 : 1);
+    kp.tmem_cols = next_pow2(((p.wpc + 3) / 4) * kp.cols_per_warp);
+    if (kp.tmem_cols > 512) return XGEN_ERR_UNSUPPORTED;
+    // Shared-memory layout (words): raw boxes | plane stages | command stages | tables | barriers.
+    kp.cmd_stage_words = ((p.max_seg_slots + 2) * kDevSlotWords + 31) & ~31;
+    kp.plane_stage_words = (p.cc * g.plane_stride + 31) & ~31;
+    const int max_ctas = 512 / kp.tmem_cols;          // blocks per SM that tensor memory has columns for
+    const size_t seg_words = ((size_t)p.n_chunks * (p.wpc + 1) + 1) & ~(size_t)1;
+    auto smem_words = [&](int stages, int tma) {
+        size_t w = (size_t)(tma ? kRawStages * ((kp.box_bytes / 4 + 31) & ~31) : 0);
+        w += (size_t)stages * (kp.plane_stage_words + kp.cmd_stage_words);
+        w += 2 * (size_t)npix_box + (tma ? 0 : ((size_t)npix_box + 1) & ~(size_t)1) + 32 * (size_t)T + seg_words;
+        return w + 2 * (3 * kMaxStages + 2 * kRawStages + 2);     // + mbarriers
+    };
+    auto occupancy = [&](size_t words) {
+        int o = (int)((size_t)kSmemPerSM / (words * 4 + 2112));     // + static and per-block reserved shared memory
+        return o < max_ctas ? o : max_ctas;
+    };
+    if (kp.use_tma && smem_words(2, 1) * 4 > (size_t)kSmemMaxDynamic) kp.use_tma = 0;   // the raw boxes do not fit
+    // Stage count: as many as fit (up to 4) without lowering the number of blocks per SM.
+    int n_stages = 2;
+    for (int st = 3; st <= kMaxStages; ++st)
+        if (smem_words(st, kp.use_tma) * 4 <= (size_t)kSmemMaxDynamic &&
+            occupancy(smem_words(st, kp.use_tma)) >= occupancy(smem_words(2, kp.use_tma))) n_stages = st;
+    if (const char *e = getenv("XGEN_PATCONV_STAGES")) { int v = atoi(e); if (v >= 2 && v <= kMaxStages && smem_words(v, kp.use_tma) * 4 <= (size_t)kSmemMaxDynamic) n_stages = v; }
+    kp.n_stages = n_stages;
+    kp.raw_stage_words = kp.use_tma ? ((kp.box_bytes / 4 + 31) & ~31) : 0;
+    kp.raw_off_words = 0;
+    kp.plane_off_words = kp.use_tma ? kRawStages * kp.raw_stage_words : 0;
+    kp.cmd_off_words = kp.plane_off_words + n_stages * kp.plane_stage_words;
+    kp.tab_off_words = kp.cmd_off_words + n_stages * kp.cmd_stage_words;
+    kp.src_off_words = kp.tab_off_words + 2 * npix_box;
+    kp.ptab_off_words = kp.src_off_words + (kp.use_tma ? 0 : ((npix_box + 1) & ~1));
+    kp.seg_off_words = kp.ptab_off_words + 32 * T;
+    kp.mbar_off_words = kp.seg_off_words + (int)seg_words;
+    size_t smem = smem_words(n_stages, kp.use_tma) * 4;
+    // Never let more blocks share an SM than tensor memory has columns for.
+    const size_t floor_bytes = (size_t)kSmemPerSM / (max_ctas + 1);
+    if (smem < floor_bytes) smem = floor_bytes;
+    if (smem > (size_t)kSmemMaxDynamic) return XGEN_ERR_UNSUPPORTED;
+    kp.out_elems = (size_t)n * ho * wo * p.c_out;
+    L.kp = kp;
+    L.smem = smem;
+    L.items = g.tiles_x * g.tiles_y * g.tiles_n * p.n_blocks;
+    return XGEN_OK;
+}
+
+// 1 KB rows of partial sums one (item, split) writes in a split run reduced inside the kernel.
+static size_t rows_per_item(const PackedHost &p) {
+    return (size_t)p.wpc * ((p.J + 7) / 8) * pixels_per_thread(p.stride);
+}
 
 // Where a run keeps the partial sums of a split, when the caller (not the plan) decides.
 struct SplitChoice { int splits, chunks_per_split; uint32_t *partial; };
@@ -908,121 +1065,84 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     if (h->device < 0) return XGEN_ERR_CUDA;
     const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
     if ((int64_t)n * hh * ww * p.c_in > 0x7FFFFFFFLL || (int64_t)n * ho * wo * p.c_out > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
+    const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
     {
         const char *xa = (const char *)x, *ya = (const char *)y;
-        const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
         const int yb = p.dtype == XGEN_F16_F32ACC ? 2 : 4;
         const char *xe = xa + (size_t)n * hh * ww * p.c_in * xb, *ye = ya + (size_t)n * ho * wo * p.c_out * yb;
         if (xa < ye && ya < xe) return XGEN_ERR_INVALID_ARG;   // overlap
     }
-    Geometry g = choose_geometry(n, ho, wo, p.stride);
-    KParams kp{};
-    kp.x = x; kp.y = y; kp.bias = bias;
-    kp.slots = h->d_slots; kp.seg_off = h->d_seg_off; kp.slot_oc = h->d_slot_oc;
-    kp.n = n; kp.h = hh; kp.w = ww; kp.ho = ho; kp.wo = wo; kp.c_in = p.c_in; kp.c_out = p.c_out;
-    kp.relu = relu ? 1 : 0;
-    kp.J = p.J; kp.wpc = p.wpc; kp.cc = p.cc; kp.n_chunks = p.n_chunks;
-    kp.lx_log = g.lx_log; kp.ly_log = g.ly_log; kp.ln_log = g.ln_log;
-    kp.tiles_x = g.tiles_x; kp.tiles_y = g.tiles_y;
-    kp.tin_w = g.tin_w; kp.tin_h = g.tin_h;
-    kp.pitch = g.pitch; kp.img_stride = g.img_stride; kp.plane_stride = g.plane_stride;
-    const int E = p.dtype == XGEN_F32 ? 1 : (p.dtype == XGEN_F16_F32ACC ? 2 : 4);
-    kp.raw_planes = p.cc / E;
-    const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
-    const int npix_box = (g.tin_w * g.tin_h) << g.ln_log;
-    // The copy engine needs 16-byte multiples: the channel run of a chunk and every global stride.
-    EncodeTiledFn encode = nullptr;
-    kp.use_tma = ((p.cc * xb) % 16 == 0) && (((size_t)p.c_in * xb) % 16 == 0) && g.tin_w <= 256 && g.tin_h <= 256 &&
-                 !getenv("XGEN_PATCONV_NO_TMA") && (encode = encode_tiled_fn()) != nullptr;
+    EncodeTiledFn encode = encode_tiled_fn();
+    Layout L;
+    xgen_status ls = make_layout(p, n, hh, ww, ((uintptr_t)y & 31) == 0, encode != nullptr, L);
+    if (ls != XGEN_OK) return ls;
     CUtensorMap tm;
     memset(&tm, 0, sizeof(tm));
-    if (kp.use_tma) {
+    if (L.kp.use_tma) {
+        const Geometry &g = L.g;
         const cuuint64_t gdim[4] = {(cuuint64_t)p.c_in, (cuuint64_t)ww, (cuuint64_t)hh, (cuuint64_t)n};
         const cuuint64_t gstr[3] = {(cuuint64_t)p.c_in * xb, (cuuint64_t)ww * p.c_in * xb, (cuuint64_t)hh * ww * p.c_in * xb};
-        const cuuint32_t box[4] = {(cuuint32_t)p.cc, (cuuint32_t)g.tin_w, (cuuint32_t)g.tin_h, (cuuint32_t)(1 << g.ln_log)};
+        const cuuint32_t box[4] = {(cuuint32_t)L.kp.rc, (cuuint32_t)g.tin_w, (cuuint32_t)g.tin_h, (cuuint32_t)(1 << g.ln_log)};
         const cuuint32_t estr[4] = {1, 1, 1, 1};
         const CUtensorMapDataType dt = p.dtype == XGEN_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
                                      : (p.dtype == XGEN_F16_F32ACC ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
         const CUresult cr = encode(&tm, dt, 4, const_cast<void *>(x), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                    CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (cr != CUDA_SUCCESS) {          // fall back to thread-issued copies
+        if (cr != CUDA_SUCCESS) {          // fall back to plain loads
             if (getenv("XGEN_PATCONV_LOG")) fprintf(stderr, "libpatconv: cuTensorMapEncodeTiled failed (%d)\n", (int)cr);
-            kp.use_tma = 0;
             memset(&tm, 0, sizeof(tm));
+            ls = make_layout(p, n, hh, ww, ((uintptr_t)y & 31) == 0, false, L);
+            if (ls != XGEN_OK) return ls;
         }
     }
-    kp.box_bytes = npix_box * p.cc * xb;
-    kp.cmd_stage_words = ((p.max_seg_slots + 2) * kSlotWords + 31) & ~31;
+    KParams kp = L.kp;
+    const size_t smem = L.smem;
+    kp.x = x; kp.y = y; kp.bias = bias;
+    kp.slots = h->d_slots; kp.seg_off = h->d_seg_off; kp.slot_oc = h->d_slot_oc;
+    kp.relu = relu ? 1 : 0;
     kp.status = h->d_status;
-    kp.vec_in = (p.c_in % E) == 0;
-    // widest aligned store per 8-channel piece: 8 words (32-byte aligned rows), 4, or scalar
-    kp.vec_out = ((p.c_out % 8) == 0 && ((uintptr_t)y & 31) == 0) ? 8 : ((p.c_out % 4) == 0 ? 4 : 0);
-    const bool is_i8 = p.dtype == XGEN_I8_I32;
-    const int T = pixels_per_thread(p.stride);
-    kp.flush_chunks = 16777216 / (p.cc * 4 * 32640);
-    if (kp.flush_chunks < 1) return XGEN_ERR_UNSUPPORTED;
-    kp.fold = (is_i8 && p.n_chunks > kp.flush_chunks) ? 1 : 0;
-    kp.cols_per_warp = p.J * T * (kp.fold ? 2 : 1);
-    kp.tmem_cols = next_pow2(((p.wpc + 3) / 4) * kp.cols_per_warp);
-    if (kp.tmem_cols > 512) return XGEN_ERR_UNSUPPORTED;
-    int exp_words = 0;
-    auto set_stage_layout = [&]() {
-        kp.act_stage_words = kp.use_tma ? ((kp.box_bytes / 4 + 31) & ~31) : ((kp.raw_planes * g.plane_stride + 31) & ~31);
-        kp.stage_words = kp.act_stage_words + kp.cmd_stage_words;
-        exp_words = (p.dtype == XGEN_F32 && !kp.use_tma) ? 0 : ((p.cc * g.plane_stride + 31) & ~31);
-    };
-    set_stage_layout();
-    const int npix_tile = (g.tin_w * g.tin_h) << g.ln_log;
-    const int max_ctas = 512 / kp.tmem_cols;          // blocks per SM that tensor memory has columns for
-    // Pick the stage count: three stages unless two let more blocks share an SM.
-    const size_t seg_words = ((size_t)p.n_chunks * (p.wpc + 1) + 1) & ~(size_t)1;
-    auto smem_words = [&](int stages) {
-        size_t w = (size_t)stages * kp.stage_words + exp_words;
-        return ((w + 1) & ~(size_t)1) + 2 * (size_t)npix_tile + 32 * (size_t)T + seg_words + 8;   // + mbarriers
-    };
-    auto occupancy = [&](size_t words) {
-        int o = (int)((size_t)kSmemPerSM / (words * 4 + 2112));     // + static and per-block reserved shared memory
-        return o < max_ctas ? o : max_ctas;
-    };
-    if (kp.use_tma && smem_words(2) * 4 > (size_t)kSmemMaxDynamic) {
-        kp.use_tma = 0;                   // the copy engine's layout needs one more tile buffer: does not fit
-        set_stage_layout();
-    }
-    int n_stages = 3;
-    if (smem_words(3) * 4 > (size_t)kSmemMaxDynamic || occupancy(smem_words(2)) > occupancy(smem_words(3))) n_stages = 2;
-    kp.n_stages = n_stages;
-    kp.exp_off_words = n_stages * kp.stage_words;
-    size_t words = smem_words(n_stages);
-    kp.mbar_off_words = (int)(words - 8);
-    kp.seg_off_words = kp.mbar_off_words - (int)seg_words;
-    kp.ptab_off_words = kp.seg_off_words - 32 * T;
-    kp.tab_off_words = kp.ptab_off_words - 2 * npix_tile;
-    size_t smem = words * 4;
-    const bool split = forced ? forced->splits > 1
-                              : (h->plan_splits > 1 && h->plan_n == n && h->plan_h == hh && h->plan_w == ww && h->d_partial);
+    // Split runs: a caller-chosen split keeps [split][output] sums for a second kernel; the
+    // planned split is reduced inside the kernel (rows of partial sums plus arrival counters).
+    const bool planned = !forced && h->plan_splits > 1 && h->plan_n == n && h->plan_h == hh && h->plan_w == ww &&
+                         h->d_partial && h->d_counters;
+    const bool split = forced ? forced->splits > 1 : planned;
     const int n_splits = forced ? forced->splits : h->plan_splits;
-    uint32_t *const partial = forced ? forced->partial : h->d_partial;
-    kp.out_elems = (size_t)n * ho * wo * p.c_out;
     kp.chunks_per_split = split ? (forced ? forced->chunks_per_split : h->plan_cps) : 0;
-    kp.partial = split ? partial : nullptr;
-    // Never let more blocks share an SM than tensor memory has columns for.
-    const size_t floor_bytes = (size_t)kSmemPerSM / (max_ctas + 1);
-    if (smem < floor_bytes) smem = floor_bytes;
-    if (smem > (size_t)kSmemMaxDynamic) return XGEN_ERR_UNSUPPORTED;
+    kp.partial = (split && forced) ? forced->partial : nullptr;
+    kp.n_splits = split ? n_splits : 1;
+    if (planned) {
+        kp.ws = h->d_partial;
+        kp.counters = h->d_counters;
+        kp.target = (h->split_seq.fetch_add(1) + 1u) * (uint32_t)n_splits;
+    }
 
     int prev = 0;
     if (cudaGetDevice(&prev) != cudaSuccess) return XGEN_ERR_CUDA;
     if (prev != h->device && cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
-    dim3 grid((unsigned)(g.tiles_x * g.tiles_y * g.tiles_n), (unsigned)p.n_blocks, (unsigned)(split ? n_splits : 1)), block((unsigned)(p.wpc * 32), 1, 1);
+    dim3 grid((unsigned)(L.g.tiles_x * L.g.tiles_y * L.g.tiles_n), (unsigned)p.n_blocks, (unsigned)(split ? n_splits : 1)), block((unsigned)((p.wpc + kProducerWarps) * 32), 1, 1);
     cudaStream_t st = (cudaStream_t)stream;
-    cudaError_t e;
-    if (p.dtype == XGEN_F32)
-        e = p.stride == 1 ? launch_np<XGEN_F32, 1>(p.np, grid, block, smem, st, kp, tm) : launch_np<XGEN_F32, 2>(p.np, grid, block, smem, st, kp, tm);
-    else if (p.dtype == XGEN_F16_F32ACC)
-        e = p.stride == 1 ? launch_np<XGEN_F16_F32ACC, 1>(p.np, grid, block, smem, st, kp, tm) : launch_np<XGEN_F16_F32ACC, 2>(p.np, grid, block, smem, st, kp, tm);
-    else
-        e = p.stride == 1 ? launch_np<XGEN_I8_I32, 1>(p.np, grid, block, smem, st, kp, tm) : launch_np<XGEN_I8_I32, 2>(p.np, grid, block, smem, st, kp, tm);
-    if (e == cudaSuccess && split) {
+    if (getenv("XGEN_PATCONV_LOG"))
+        fprintf(stderr, "libpatconv: grid %u x %u x %u, %u threads, %zu bytes shared, %d stages, lanes %dx%dx%d, tile in %dx%d, tma %d, cc %d, fused split %d\n",
+                grid.x, grid.y, grid.z, block.x, smem, kp.n_stages, 1 << L.g.lx_log, 1 << L.g.ly_log, 1 << L.g.ln_log,
+                L.g.tin_w, L.g.tin_h, kp.use_tma, p.cc, planned ? 1 : 0);
+    const void *kern = kernel_for(p);
+    cudaError_t e = allow_large_smem(kern);
+    if (e == cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        if (planned) {
+            // the splits of an item wait for each other: all blocks must be resident together
+            attr[0].id = cudaLaunchAttributeCooperative;
+            attr[0].val.cooperative = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+        }
+        void *args[2] = {(void *)&kp, (void *)&tm};
+        e = cudaLaunchKernelExC(&cfg, kern, args);
+        if (e == cudaSuccess) e = cudaGetLastError();
+        e = log_cuda(e, "kernel launch");
+    }
+    if (e == cudaSuccess && split && forced) {
         const int vec = kp.vec_out >= 4 ? 1 : 0;
         const size_t items = vec ? kp.out_elems / 4 : kp.out_elems;
         const unsigned blocks = (unsigned)((items + 255) / 256);
@@ -1032,7 +1152,7 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr; cfg.numAttrs = 1;
-        const uint32_t *part_c = partial;
+        const uint32_t *part_c = forced->partial;
         const size_t oe = kp.out_elems;
         const int co = p.c_out, rl = kp.relu;
         const void *bias_c = bias;
@@ -1060,6 +1180,83 @@ static uint32_t *g_static_scratch_addr[64];        // device address per device 
 static std::mutex g_static_scratch_mutex;
 
 extern "C" {
+
+xgen_status xgen_patconv_plan(xgen_patconv_packed *h, int32_t n, int32_t hh, int32_t ww) {
+    if (!h) return XGEN_ERR_INVALID_ARG;
+    if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
+    if (h->device < 0) return XGEN_ERR_CUDA;
+    const PackedHost &p = h->host;
+    const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
+    if ((int64_t)n * ho * wo * p.c_out > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
+    Layout L;
+    xgen_status ls = make_layout(p, n, hh, ww, true, encode_tiled_fn() != nullptr, L);
+    if (ls != XGEN_OK) return ls;
+    int prev = 0;
+    if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
+    xgen_status rs = XGEN_OK;
+    int sms = 148, bps = 0;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
+    const void *kern = kernel_for(p);
+    if (allow_large_smem(kern) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, kern, (p.wpc + kProducerWarps) * 32, L.smem) != cudaSuccess) {
+        cudaGetLastError();
+        rs = XGEN_ERR_CUDA;
+    }
+    bps = std::min(bps, 512 / L.kp.tmem_cols);
+    // The splits of an item wait for each other inside the kernel, so every block of the
+    // launch must be resident at once: items x splits <= SMs x blocks per SM.  Within that,
+    // pick the split count with a small cost model (cycles): a block costs a fixed prologue
+    // and epilogue plus its multiply-adds at the rate an SM sustains with the warps it then
+    // hosts; a split run adds the exchange of the partial sums.
+    const int64_t capacity = (int64_t)sms * bps;
+    const int64_t max_splits = std::min<int64_t>(p.n_chunks, L.items > 0 ? capacity / L.items : 1);
+    const double slot_macs_item = 4.0 * (double)p.stats.kernels_surviving / (double)p.n_blocks * 32.0 * pixels_per_thread(p.stride);
+    auto sm_rate = [&](int warps) { return 50.0 * std::pow((double)std::min(warps, 16) / 16.0, 0.65); };   // multiply-adds per cycle
+    auto estimate = [&](int64_t k) {
+        const int cps_k = (int)((p.n_chunks + k - 1) / k);
+        const int64_t parts = (p.n_chunks + cps_k - 1) / cps_k;
+        const int64_t blocks = L.items * parts;
+        const int per_sm = (int)((blocks + sms - 1) / sms);
+        const double work = slot_macs_item * (double)cps_k / (double)p.n_chunks;
+        double t = 9000.0 + work * per_sm / sm_rate(per_sm * p.wpc);
+        if (parts > 1) t += 5000.0 + 150.0 * (double)parts;
+        return t;
+    };
+    int64_t splits = 1;
+    double best_t = estimate(1);
+    for (int64_t k = 2; k <= max_splits; ++k) {
+        const double t = estimate(k);
+        if (t < 0.97 * best_t) { best_t = t; splits = k; }
+    }
+    if (const char *e = getenv("XGEN_PATCONV_SPLIT")) { int v = atoi(e); if (v >= 1) splits = std::min<int64_t>(v, std::max<int64_t>(1, max_splits)); }
+    if (splits < 1) splits = 1;
+    const int cps = (int)((p.n_chunks + splits - 1) / splits);
+    splits = (p.n_chunks + cps - 1) / cps;
+    if (rs == XGEN_OK && cudaDeviceSynchronize() != cudaSuccess) rs = XGEN_ERR_CUDA;
+    if (rs == XGEN_OK && splits > 1) {
+        const size_t need = (size_t)L.items * (size_t)splits * rows_per_item(p) * 1024;
+        const size_t need_c = (size_t)L.items * sizeof(uint32_t);
+        if (need > h->partial_bytes) {
+            if (h->d_partial) cudaFree(h->d_partial);
+            h->d_partial = nullptr; h->partial_bytes = 0;
+            if (cudaMalloc(&h->d_partial, need) != cudaSuccess) { cudaGetLastError(); rs = XGEN_ERR_ALLOC; }
+            else h->partial_bytes = need;
+        }
+        if (rs == XGEN_OK && need_c > h->counter_bytes) {
+            if (h->d_counters) cudaFree(h->d_counters);
+            h->d_counters = nullptr; h->counter_bytes = 0;
+            if (cudaMalloc(&h->d_counters, need_c) != cudaSuccess) { cudaGetLastError(); rs = XGEN_ERR_ALLOC; }
+            else h->counter_bytes = need_c;
+        }
+        if (rs == XGEN_OK && cudaMemset(h->d_counters, 0, h->counter_bytes) != cudaSuccess) rs = XGEN_ERR_CUDA;
+        h->split_seq.store(0);
+    }
+    cudaSetDevice(prev);
+    if (rs != XGEN_OK) { h->plan_splits = 1; h->plan_n = 0; return rs; }
+    h->plan_n = n; h->plan_h = hh; h->plan_w = ww;
+    h->plan_splits = (int)splits; h->plan_cps = cps;
+    return XGEN_OK;
+}
 
 xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
                              const void *bias, int32_t relu, void *y, void *stream) {

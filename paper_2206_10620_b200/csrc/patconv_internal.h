@@ -7,7 +7,8 @@
 
 namespace patconv {
 
-constexpr int kSlotWords = 8;   // one command slot = 32 bytes
+constexpr int kSlotWords = 8;   // one command slot of the host image = 32 bytes
+constexpr int kDevSlotBytes = 48;   // on the device every weight is stored twice (operand pairs)
 // A thread owns a 4x4 block of output pixels at stride 1 and a 2x4 block at stride 2;
 // a filter's running sums take that many tensor-memory columns.
 constexpr int pix_per_thread(int stride) { return stride == 1 ? 16 : 8; }
