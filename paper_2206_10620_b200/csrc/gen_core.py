@@ -35,15 +35,16 @@ columns (0,2,1,3) and half 1 holds (2,4,3,5) (stride 2: (2,4)).  The two halves
 are separate arrays (operands %1 and %5) so that the loads of a quarter warp
 fall into distinct banks.
 
-Command decoding is software-pipelined over two register sets (A and B), with
-every block emitted once per set: while command i runs from set A, command i+1
-is already decoded in set B, command i+2 is read from shared memory into set A
-once command i's weights are consumed, and the block ends with an indirect
-branch on set B's opcode (brx.idx).  Between two LOADs every kernel command
+Every block starts by asking tensor memory for its row and shared memory for
+its weights and for the opcode and operand of the following command, waits for
+the row, runs its FMAs and ends with an indirect branch on that next opcode
+(brx.idx): the loads overlap the row fetch, the next opcode is long there when
+the branch needs it, and one copy of each block keeps the code small enough to
+stay in the instruction cache.  Between two LOADs every kernel command
 addresses a different filter; a LOAD and the block's exit wait for all
 tensor-memory writes (tcgen05.wait::st), which covers a filter that ends one
-channel and starts the next.  The stream segment is staged with two valid
-spare slots so the look-ahead never reads undefined data.
+channel and starts the next.  The stream segment is staged with valid spare
+slots behind it so the look-ahead never reads undefined data.
 
 Operands of every block, in order:
   %0 "+r" shared-memory address of the warp's first command slot
@@ -74,73 +75,70 @@ def gen_block(np_, stride):
     rows = (bh - 1) * stride + 3
     ppr = 4 if stride == 1 else 3            # operand pairs per patch row
     L = ["{"]
-    L.append(" .reg .b32 opA, payA, opB, payB, ta, adA, adB;")
+    L.append(" .reg .b32 op, pay, ta, adA, adB;")
     L.append(" .reg .b32 a<%d>;" % T)
-    L.append(" .reg .b64 q<%d>, acc<%d>, wdA<4>, wdB<4>;" % (rows * ppr, T // 2))
+    L.append(" .reg .b64 q<%d>, acc<%d>, wd<4>;" % (rows * ppr, T // 2))
     # Registers written on one path and read on another must be defined on every
-    # path into the branch tables, or register allocation degrades badly.
+    # path into the branch table, or register allocation degrades badly.
     for i in range(rows * ppr):
         L.append(" mov.b64 q%d, 0;" % i)
-    for S in "AB":
-        L.append(" ts%s: .branchtargets %s;" % (
-            S, ",".join("K%s%d" % (S, i) for i in range(len(masks))) + ",LOAD%s,END%s" % (S, S)))
-
-    def fetch(S, off):
-        return [" ld.shared.v2.b32 {op%s, pay%s}, [%%0+%d];" % (S, S, off),
-                " ld.shared.v2.b64 {wd%s0, wd%s1}, [%%0+%d];" % (S, S, off + 16),
-                " ld.shared.v2.b64 {wd%s2, wd%s3}, [%%0+%d];" % (S, S, off + 32)]
+    L.append(" ts: .branchtargets %s;" % (",".join("K%d" % i for i in range(len(masks))) + ",LOAD,END"))
 
     accs = "{" + ",".join("a%d" % i for i in range(T)) + "}"
 
-    # prologue: commands 0 and 1 decoded
-    L += fetch("A", 0) + fetch("B", SLOT_BYTES)
-    L.append(" add.u32 %%0, %%0, %d;" % (2 * SLOT_BYTES))
-    L.append(" brx.idx.uni opA, tsA;")
+    def next_header():
+        # opcode and operand of the following command; %0 moves on to it
+        return [" ld.shared.v2.b32 {op, pay}, [%%0+%d];" % SLOT_BYTES,
+                " add.u32 %%0, %%0, %d;" % SLOT_BYTES]
 
-    for S, O in (("A", "B"), ("B", "A")):
-        def refill_and_go():
-            return fetch(S, 0) + [" add.u32 %%0, %%0, %d;" % SLOT_BYTES, " brx.idx.uni op%s, ts%s;" % (O, O)]
+    # prologue: command 0 decoded
+    L.append(" ld.shared.v2.b32 {op, pay}, [%0];")
+    L.append(" brx.idx.uni op, ts;")
 
-        for pi, m in enumerate(masks):
-            L.append(" K%s%d:" % (S, pi))
-            L.append(" add.u32 ta, %%4, pay%s;" % S)
-            L.append(" tcgen05.ld.sync.aligned.32x32b.x%d.b32 %s, [ta];" % (T, accs))
-            taps = [t for t in range(9) if (m >> t) & 1]
-            L.append(" tcgen05.wait::ld.sync.aligned;")
-            for n in range(T // 2):
-                L.append(" mov.b64 acc%d, {a%d, a%d};" % (n, 2 * n, 2 * n + 1))
-            for k, t in enumerate(taps):
-                dy, dx = divmod(t, 3)
-                for py in range(bh):
-                    if stride == 1:
-                        for h in range(2):
-                            L.append(" fma.rn.f32x2 acc%d, wd%s%d, q%d, acc%d;" % (
-                                py * 2 + h, S, k, (py + dy) * ppr + dx + h, py * 2 + h))
-                    else:
-                        L.append(" fma.rn.f32x2 acc%d, wd%s%d, q%d, acc%d;" % (
-                            py, S, k, (2 * py + dy) * ppr + dx, py))
-            for n in range(T // 2):
-                L.append(" mov.b64 {a%d, a%d}, acc%d;" % (2 * n, 2 * n + 1, n))
-            L.append(" tcgen05.st.sync.aligned.32x32b.x%d.b32 [ta], %s;" % (T, accs))
-            L += refill_and_go()
+    for pi, m in enumerate(masks):
+        L.append(" K%d:" % pi)
+        L.append(" add.u32 ta, %4, pay;")
+        L.append(" tcgen05.ld.sync.aligned.32x32b.x%d.b32 %s, [ta];" % (T, accs))
+        L.append(" ld.shared.v2.b64 {wd0, wd1}, [%0+16];")
+        L.append(" ld.shared.v2.b64 {wd2, wd3}, [%0+32];")
+        L += next_header()
+        taps = [t for t in range(9) if (m >> t) & 1]
+        L.append(" tcgen05.wait::ld.sync.aligned;")
+        for n in range(T // 2):
+            L.append(" mov.b64 acc%d, {a%d, a%d};" % (n, 2 * n, 2 * n + 1))
+        for k, t in enumerate(taps):
+            dy, dx = divmod(t, 3)
+            for py in range(bh):
+                if stride == 1:
+                    for h in range(2):
+                        L.append(" fma.rn.f32x2 acc%d, wd%d, q%d, acc%d;" % (
+                            py * 2 + h, k, (py + dy) * ppr + dx + h, py * 2 + h))
+                else:
+                    L.append(" fma.rn.f32x2 acc%d, wd%d, q%d, acc%d;" % (
+                        py, k, (2 * py + dy) * ppr + dx, py))
+        for n in range(T // 2):
+            L.append(" mov.b64 {a%d, a%d}, acc%d;" % (2 * n, 2 * n + 1, n))
+        L.append(" tcgen05.st.sync.aligned.32x32b.x%d.b32 [ta], %s;" % (T, accs))
+        L.append(" brx.idx.uni op, ts;")
 
-        L.append(" LOAD%s:" % S)
-        L.append(" tcgen05.wait::st.sync.aligned;")          # no write to any row is in flight
-        L.append(" mad.lo.u32 adA, pay%s, %%2, %%1;" % S)
-        L.append(" mad.lo.u32 adB, pay%s, %%2, %%5;" % S)
-        for r in range(rows):
-            L.append(" ld.shared.v2.b64 {q%d,q%d}, [adA];" % (r * ppr, r * ppr + 1))
-            if stride == 1:
-                L.append(" ld.shared.v2.b64 {q%d,q%d}, [adB];" % (r * ppr + 2, r * ppr + 3))
-            else:
-                L.append(" ld.shared.b64 q%d, [adB];" % (r * ppr + 2))
-            if r < rows - 1:
-                L.append(" add.u32 adA, adA, %3;")
-                L.append(" add.u32 adB, adB, %3;")
-        L += refill_and_go()
+    L.append(" LOAD:")
+    L.append(" tcgen05.wait::st.sync.aligned;")          # no write to any row is in flight
+    L.append(" mad.lo.u32 adA, pay, %2, %1;")
+    L.append(" mad.lo.u32 adB, pay, %2, %5;")
+    L += next_header()
+    for r in range(rows):
+        L.append(" ld.shared.v2.b64 {q%d,q%d}, [adA];" % (r * ppr, r * ppr + 1))
+        if stride == 1:
+            L.append(" ld.shared.v2.b64 {q%d,q%d}, [adB];" % (r * ppr + 2, r * ppr + 3))
+        else:
+            L.append(" ld.shared.b64 q%d, [adB];" % (r * ppr + 2))
+        if r < rows - 1:
+            L.append(" add.u32 adA, adA, %3;")
+            L.append(" add.u32 adB, adB, %3;")
+    L.append(" brx.idx.uni op, ts;")
 
-        L.append(" END%s:" % S)
-        L.append(" bra.uni DONE;")
+    L.append(" END:")
+    L.append(" bra.uni DONE;")
     L.append(" DONE:")
     L.append(" tcgen05.wait::st.sync.aligned;")
     L.append("}")
