@@ -42,7 +42,7 @@ FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 # dram__bytes_read.sum + dram__bytes_write.sum of patconv_kernel, average per launch over one
 # step of this workload, from the ncu capture summarised in profiles/bench_vgg16_launch_list.md
 # (taken with the kernels as committed; set to None when the kernel changes).
-NCU_DRAM_BYTES_PER_LAUNCH = 4.55e6
+NCU_DRAM_BYTES_PER_LAUNCH = 5.6e6
 
 
 def rank_seed(rank: int) -> int:

@@ -267,6 +267,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
 
     // A tile box carries rc channels, i.e. spb = rc / cc consecutive chunks; boxes q0..q_end
@@ -282,6 +283,25 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     };
     if (pw == 0 && lane == 0 && P.use_tma)
         for (int r = 0; r < kRawStages && q0 + r <= q_end; ++r) issue_box(q0 + r);
+    // The block's commands of chunk c (one contiguous segment [s0, s1) plus two look-ahead
+    // slots), handed to the copy engine (one thread) for stage s.
+    auto issue_commands = [&](int s, int s0, int s1) {
+        const uint32_t cmd_bytes = (uint32_t)(s1 - s0 + 2) * (kDevSlotWords * 4u);
+        const uint32_t cmd = smem_base + (uint32_t)(P.cmd_off_words + s * P.cmd_stage_words) * 4u;
+        mbar_expect_tx(bar_cmd(s), cmd_bytes);
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(cmd), "l"(P.slots + (size_t)s0 * kDevSlotWords), "r"(cmd_bytes), "r"(bar_cmd(s)) : "memory");
+    };
+    const int32_t *seg_g = P.seg_off + ((size_t)b * P.n_chunks + c_begin) * (P.wpc + 1);
+    // The first stages are free: their commands start now, with offsets read straight from
+    // global memory, instead of after the tables below are built.
+    if (pw == 0 && lane == 0)
+        for (int k = 0; k < NS && c_begin + k < c_end; ++k)
+            issue_commands(k, __ldg(seg_g + k * (P.wpc + 1)), __ldg(seg_g + k * (P.wpc + 1) + P.wpc));
+    // Global reads of the tables below, started before the index arithmetic they do not need.
+    const int soc_v = tid < P.wpc * P.J ? __ldg(P.slot_oc + (size_t)blockIdx.y * P.wpc * P.J + tid) : -1;
+    const int n_seg = (c_end - c_begin) * (P.wpc + 1);
+    const int seg_v = tid < n_seg ? __ldg(seg_g + tid) : 0;
 
     // --- tables, built once by all threads while the first boxes are in flight --------
     // Per staged pixel: where its value goes inside a channel plane.  A plane holds, per
@@ -317,7 +337,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
             srct[q] = ok ? ((gn * P.h + gy) * P.w + gx) * P.c_in : -1;
         }
     }
-    for (int i = tid; i < P.wpc * P.J; i += nthreads) soc_s[i] = P.slot_oc[(size_t)blockIdx.y * P.wpc * P.J + i];
+    if (tid < P.wpc * P.J) soc_s[tid] = soc_v;                       // wpc * J <= 256 < threads of a block
     // Output-pixel table: linear pixel index of (sum t of lane l), or -1 outside the output.
     // Stride 1 keeps a row's four pixels as the pairs (0,2) and (1,3): sum 4*py + 2*h + e is
     // pixel (py, h + 2*e); stride 2: sum 2*py + e is pixel (py, e).
@@ -331,9 +351,17 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         ptab[i] = (on < P.n && oy < P.ho && ox < P.wo) ? (on * P.ho + oy) * P.wo + ox : -1;
     }
     // Segment offsets of this block's chunks.
-    const int32_t *seg_g = P.seg_off + (size_t)b * P.n_chunks * (P.wpc + 1);
     int *seg = reinterpret_cast<int *>(smem + P.seg_off_words);
-    for (int i = tid; i < (c_end - c_begin) * (P.wpc + 1); i += nthreads) seg[i] = seg_g[c_begin * (P.wpc + 1) + i];
+    if (tid < n_seg) seg[tid] = seg_v;
+    for (int i = tid + nthreads; i < n_seg; i += nthreads) seg[i] = seg_g[i];
+    // The consumer warps clear their running sums while the staging warps finish the tables.
+    if (!producer) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t tw = tmem_base_s + (((uint32_t)(warp & 3) * 32u) << 16) + (uint32_t)((warp >> 2) * P.cols_per_warp);
+        const uint32_t z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        for (int c = 0; c < P.cols_per_warp; c += 8) tmem_st8(tw + c, z);
+        tmem_wait_st();
+    }
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -347,15 +375,8 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         for (int c = c_begin; c < c_end; ++c) {
             const int k = c - c_begin, s = k % NS;
             if (k >= NS && !mbar_wait(bar_empty(s), (uint32_t)((k / NS - 1) & 1), &abort_s, P.status)) break;
-            if (pw == 0 && lane == 0) {
-                // this block's commands for the chunk: one contiguous segment, two look-ahead slots beyond it
-                const int s0 = seg[k * (P.wpc + 1)], s1 = seg[k * (P.wpc + 1) + P.wpc];
-                const uint32_t cmd_bytes = (uint32_t)(s1 - s0 + 2) * (kDevSlotWords * 4u);
-                const uint32_t cmd = smem_base + (uint32_t)(P.cmd_off_words + s * P.cmd_stage_words) * 4u;
-                mbar_expect_tx(bar_cmd(s), cmd_bytes);
-                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                             ::"r"(cmd), "l"(P.slots + (size_t)s0 * kDevSlotWords), "r"(cmd_bytes), "r"(bar_cmd(s)) : "memory");
-            }
+            if (pw == 0 && lane == 0 && k >= NS)      // the first NS chunks' commands are on their way already
+                issue_commands(s, seg[k * (P.wpc + 1)], seg[k * (P.wpc + 1) + P.wpc]);
             float *pl = reinterpret_cast<float *>(smem + P.plane_off_words + s * P.plane_stage_words);
             if (P.use_tma) {
                 const int q = c / spb, sub = c - q * spb;
@@ -437,11 +458,6 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     } else {
         // ===== consumer warps ===========================================================
         const uint32_t tmem_warp = tmem_cta + (((uint32_t)(warp & 3) * 32u) << 16) + (uint32_t)((warp >> 2) * P.cols_per_warp);
-        {
-            const uint32_t z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-            for (int c = 0; c < P.cols_per_warp; c += 8) tmem_st8(tmem_warp + c, z);
-            tmem_wait_st();
-        }
         const uint32_t tmem_int = tmem_warp + (uint32_t)(P.J * T);   // i8 with folding: int32 totals
 
         // i8: fold the exact fp32 partial sums into the int32 totals and clear them
