@@ -68,7 +68,8 @@ typedef struct {
                                      operand byte per command, plus the offset and slot tables */
     int64_t csr_index_bytes;      /* index bytes CSR would need for the same non-zeros
                                      (one 4-byte column per weight + one row pointer per filter) */
-    int64_t stream_bytes;         /* bytes of the command stream as stored on the device      */
+    int64_t stream_bytes;         /* bytes of the command stream as stored on the device
+                                     (48-byte slots: every kept weight is stored twice there) */
     int32_t filters_per_group;    /* J: filters one warp accumulates together                 */
     int32_t groups_per_block;     /* filter groups (warps) per thread block                   */
     int32_t n_blocks;             /* blocks of contiguous output channels                     */
@@ -79,7 +80,7 @@ typedef struct {
     int64_t load_commands;        /* activation-patch loads in the stream (one per group and
                                      input channel that group is connected to)                */
     double  group_imbalance;      /* worst thread block: max / mean of surviving kernels over
-                                     the block's groups (its warps wait for each other)       */
+                                     the block's groups (its warps share the staged tiles)    */
 } xgen_patconv_stats;
 
 /* Read-only view of the packed layout on the host, for inspection and tests.
@@ -99,7 +100,9 @@ typedef struct {
  * entry g = G is one past the segment.  Inside a group's run every LOAD is
  * followed by the kernel commands of that channel, and the run ends with END.
  * slot_oc[(b * G + g) * J + j] is the original output channel of filter slot j,
- * or -1 for an empty slot. */
+ * or -1 for an empty slot.
+ * The device copy holds the same commands as 48-byte slots
+ * {opcode, operand, -, -, w0, w0, w1, w1, w2, w2, w3, w3}. */
 typedef struct {
     const uint32_t *slots;          int64_t n_slots;
     const int32_t  *seg_off;        /* [n_blocks * n_chunks * (G + 1)]                         */
@@ -199,10 +202,16 @@ xgen_status xgen_patconv_run_host(const xgen_patconv_packed *packed, const void 
  * Optional: prepare the handle for one input shape.  Layers with few output
  * pixels do not fill the GPU with (pixel tile x filter block) work items; for
  * such a shape this call lets later xgen_patconv_run calls split the input
- * channels across thread blocks and reduce the partial sums (the paper does
- * not discuss this; it is the cross-channel reduction of this implementation).
- * It allocates a workspace owned by the handle, so it synchronises and must not
- * be called while the handle is in use.  Without it every shape runs unsplit.
+ * channels across thread blocks (the paper does not discuss this; it is the
+ * cross-channel reduction of this implementation).  The blocks of a split write
+ * their partial sums to a workspace, count themselves in, wait (with a bound)
+ * for the others and each reduce a share, all inside the one kernel, which is
+ * therefore launched cooperatively: the split count is chosen so that every
+ * block is resident at once.  The call allocates the workspace and the
+ * counters, owned by the handle, so it synchronises and must not be called
+ * while the handle is in use; planned runs of one handle share them and must
+ * not overlap on the GPU (use one stream, or order them with events).  Without
+ * this call every shape runs unsplit.
  * Errors: INVALID_ARG, SHAPE, ALLOC, CUDA.
  */
 xgen_status xgen_patconv_plan(xgen_patconv_packed *packed, int32_t n, int32_t h, int32_t w);
@@ -219,8 +228,9 @@ xgen_status xgen_patconv_view(const xgen_patconv_packed *packed, xgen_patconv_ho
 
 /* Synchronise the stream and report the first CUDA error seen on it, as a
  * status (XGEN_OK, XGEN_ERR_CUDA).  The kernels contain no unbounded waits: a wait
- * for a tile copy that runs out of its bound marks the handle, the kernel still
- * ends, and this call then returns XGEN_ERR_TIMEOUT once (results are invalid). */
+ * (for a staged tile, a free stage, or the other blocks of a split) that runs out
+ * of its bound marks the handle, the kernel still ends, and this call then returns
+ * XGEN_ERR_TIMEOUT once (results are invalid; the split counters are reset). */
 xgen_status xgen_patconv_last_status(const xgen_patconv_packed *packed, void *cuda_stream);
 
 /* Release the handle and its device memory.  NULL is allowed. */
