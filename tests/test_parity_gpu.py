@@ -131,7 +131,7 @@ def test_argument_errors():
 @pytest.mark.parametrize("stride", [1, 2])
 def test_planned_shape_splits_input_channels(dtype, stride):
     # few output pixels, many input channels: plan() splits the channel chunks across
-    # blocks and a second kernel reduces the partial sums
+    # blocks, which exchange their partial sums and reduce them inside the one kernel
     d = _layer(dtype, 1, 256, 72, 14, 14, stride, prune=0.6, lib=8, seed=11)
     pk = pack(d)
     pk.plan(1, 14, 14)
@@ -154,4 +154,40 @@ def test_planned_odd_channel_count():
     d = _layer("f32", 2, 130, 37, 7, 7, 1, prune=0.3, lib=12, seed=4)
     pk = pack(d)
     pk.plan(2, 7, 7)
+    compare(d, run_gpu(pk, d.x, d.bias, True))
+
+
+def test_planned_runs_back_to_back_and_replanned():
+    """The arrival counters of a planned split only grow: many launches in a row on one
+    stream, without a host synchronisation in between, must all reduce correctly; planning
+    the handle for another shape starts over."""
+    import torch
+    d = _layer("f32", 1, 192, 64, 12, 12, 1, prune=0.5, lib=8, seed=31)
+    pk = pack(d)
+    pk.plan(1, 12, 12)
+    x = torch.from_numpy(d.x).cuda()
+    b = torch.from_numpy(d.bias).cuda()
+    ys = [torch.full((1, 12, 12, 64), 777.0, device="cuda") for _ in range(25)]
+    st = torch.cuda.current_stream().cuda_stream
+    for y in ys:
+        pk.run(x.data_ptr(), 1, 12, 12, b.data_ptr(), True, y.data_ptr(), st)
+    pk.sync(st)
+    first = ys[0].cpu().numpy()
+    compare(d, first)
+    for y in ys[1:]:
+        assert np.array_equal(y.cpu().numpy(), first)
+    d2 = _layer("f32", 2, 192, 64, 7, 7, 1, prune=0.5, lib=8, seed=31)
+    pk.plan(2, 7, 7)
+    y2 = run_gpu(pk, d2.x, d.bias, True)
+    d2.w, d2.pid, d2.masks = d.w, d.pid, d.masks
+    compare(d2, y2, bias=d.bias)
+    compare(d, run_gpu(pk, d.x, d.bias, True))          # the first shape now runs unsplit
+
+
+def test_planned_long_integer_layer():
+    # more than 128 input channels: the integer variant folds its exact fp32 partial sums into
+    # int32 totals on the way, and the split exchanges those totals
+    d = _layer("i8", 1, 320, 48, 10, 10, 1, prune=0.4, lib=8, seed=17)
+    pk = pack(d)
+    pk.plan(1, 10, 10)
     compare(d, run_gpu(pk, d.x, d.bias, True))
