@@ -205,9 +205,10 @@ xgen_status xgen_patconv_run_host(const xgen_patconv_packed *packed, const void 
  * channels across thread blocks (the paper does not discuss this; it is the
  * cross-channel reduction of this implementation).  The blocks of a split write
  * their partial sums to a workspace, count themselves in, wait (with a bound)
- * for the others and each reduce a share, all inside the one kernel, which is
- * therefore launched cooperatively: the split count is chosen so that every
- * block is resident at once.  The call allocates the workspace and the
+ * for the others and each reduce a share, all inside the one kernel: the split
+ * count is chosen so that every block of the launch is resident at once on an
+ * otherwise idle GPU (other work on the GPU at the same time can only delay the
+ * blocks; a wait that runs out is reported by xgen_patconv_last_status).  The call allocates the workspace and the
  * counters, owned by the handle, so it synchronises and must not be called
  * while the handle is in use; planned runs of one handle share them and must
  * not overlap on the GPU (use one stream, or order them with events).  Without

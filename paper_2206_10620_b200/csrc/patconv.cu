@@ -254,6 +254,11 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     const int c_begin = P.chunks_per_split ? (int)blockIdx.z * P.chunks_per_split : 0;
     const int c_end = P.chunks_per_split ? min(P.n_chunks, c_begin + P.chunks_per_split) : P.n_chunks;
 
+    // Launched with programmatic stream serialisation: the next kernel of the stream may be
+    // scheduled as soon as SMs free up (its launch latency then overlaps this kernel's tail);
+    // every kernel waits for its predecessors below, before it touches global memory.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     // --- tensor memory for the running sums; barriers -------------------------------
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -269,6 +274,8 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // everything launched before this kernel is complete
 
     // A tile box carries rc channels, i.e. spb = rc / cc consecutive chunks; boxes q0..q_end
     // cover this block's chunks.  Box q is handed to the copy engine by one thread.
@@ -1146,13 +1153,15 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     if (e == cudaSuccess) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        // Programmatic stream serialisation: this kernel may be scheduled while its predecessor
+        // in the stream drains (it waits for it, griddepcontrol.wait, before touching memory), and
+        // it lets its successor do the same.  A dependent grid starts only after every block of
+        // this one has started, so the blocks of a split, which wait for each other and which the
+        // planner keeps within what the GPU holds at once, are never kept out by a successor.
         cudaLaunchAttribute attr[1];
-        if (planned) {
-            // the splits of an item wait for each other: all blocks must be resident together
-            attr[0].id = cudaLaunchAttributeCooperative;
-            attr[0].val.cooperative = 1;
-            cfg.attrs = attr; cfg.numAttrs = 1;
-        }
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = getenv("XGEN_PATCONV_NO_PDL") ? 0 : 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
         void *args[2] = {(void *)&kp, (void *)&tm};
         e = cudaLaunchKernelExC(&cfg, kern, args);
         if (e == cudaSuccess) e = cudaGetLastError();
