@@ -275,7 +275,11 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
 
-    asm volatile("griddepcontrol.wait;" ::: "memory");     // everything launched before this kernel is complete
+    // From here on only the packed layer (commands, tables: written at pack time, before any
+    // launch) is read without more ado.  Whatever an earlier kernel of the stream may have
+    // produced or may still read -- x, y, the split's workspace and counters -- is touched only
+    // after griddepcontrol.wait, by each thread that touches it: the table building below can
+    // overlap the tail of the previous kernel.
 
     // A tile box carries rc channels, i.e. spb = rc / cc consecutive chunks; boxes q0..q_end
     // cover this block's chunks.  Box q is handed to the copy engine by one thread.
@@ -288,8 +292,10 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
                      ::"r"(dst), "l"(&tmap), "r"(q * P.rc), "r"(gx0), "r"(gy0), "r"(n0), "r"(bar_raw(r)) : "memory");
     };
-    if (pw == 0 && lane == 0 && P.use_tma)
+    if (pw == 0 && lane == 0 && P.use_tma) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");       // x is complete
         for (int r = 0; r < kRawStages && q0 + r <= q_end; ++r) issue_box(q0 + r);
+    }
     // The block's commands of chunk c (one contiguous segment [s0, s1) plus two look-ahead
     // slots), handed to the copy engine (one thread) for stage s.
     auto issue_commands = [&](int s, int s0, int s1) {
@@ -378,6 +384,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
 
     if (producer) {
         // ===== producer warps: fill stage after stage; warp 0 also drives the copy engine =====
+        if (!P.use_tma) asm volatile("griddepcontrol.wait;" ::: "memory");   // they read x themselves
         const int ptid = pw * 32 + lane;
         for (int c = c_begin; c < c_end; ++c) {
             const int k = c - c_begin, s = k % NS;
@@ -518,6 +525,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         // A group is a run of J consecutive output channels, so for one pixel a thread holds
         // 8 adjacent channels per 8 filter slots: 32 bytes (16 for fp16) it can store as one
         // piece.  No shared memory, no block-wide barrier: every warp drains on its own.
+        asm volatile("griddepcontrol.wait;" ::: "memory");       // before the first store to y or the workspace
         const int *soc = soc_s + warp * P.J;
         const uint32_t tmem_res = (DT == XGEN_I8_I32 && P.fold) ? tmem_int : tmem_warp;
         const int oc_base = soc[0];
@@ -565,6 +573,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
 
     if (P.ws) {
         // ===== split run: wait for the other splits of this item, then reduce a share =====
+        asm volatile("griddepcontrol.wait;" ::: "memory");       // the producer warps join in here
         __threadfence();
         __syncthreads();
         if (tid == 0) {
