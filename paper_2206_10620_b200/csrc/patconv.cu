@@ -62,6 +62,8 @@ struct KParams {
     int lx_log, ly_log, ln_log;          // lanes along x, y and images: 2^.. each, product 32
     int tiles_x, tiles_y;
     int tin_w, tin_h;                    // staged tile extents, input pixels
+    uint32_t mg_tiles_x, mg_tiles_y, mg_tin_w, mg_tin_h, mg_spb;   // division by these as a multiplication (div_by)
+    int spb;                             // chunks per tile box, rc / cc
     int pitch, img_stride, half_stride, plane_stride;   // words
     int raw_stage_words, plane_stage_words, cmd_stage_words;
     int n_stages;                        // plane + command stages
@@ -213,6 +215,10 @@ __device__ __forceinline__ void store_piece(const KParams &P, const uint32_t (&r
     }
 }
 
+// n / d for the small divisors of the launch geometry: m = 2^32 / d + 1 (0 stands for d = 1),
+// exact while n * d < 2^32.
+__device__ __forceinline__ int div_by(int n, uint32_t m) { return m ? (int)__umulhi((uint32_t)n, m) : n; }
+
 // ---- the kernel -----------------------------------------------------------------
 template <int DT, int STRIDE, int NP>
 __global__ void __launch_bounds__((kMaxWarps + kProducerWarps) * 32)
@@ -231,10 +237,11 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     const int pw = warp - P.wpc;                     // producer warp number
     const int b = blockIdx.y;
     const int item = (int)(blockIdx.x + gridDim.x * blockIdx.y);   // (tile, filter block)
-    int tile = blockIdx.x;
-    const int tx = tile % P.tiles_x; tile /= P.tiles_x;
-    const int ty = tile % P.tiles_y;
-    const int tn = tile / P.tiles_y;
+    const int tile = blockIdx.x;
+    const int tile_r = div_by(tile, P.mg_tiles_x);
+    const int tx = tile - tile_r * P.tiles_x;
+    const int tn = div_by(tile_r, P.mg_tiles_y);
+    const int ty = tile_r - tn * P.tiles_y;
     const int LX = 1 << P.lx_log, LY = 1 << P.ly_log;
     const int l_x = lane & (LX - 1), l_y = (lane >> P.lx_log) & (LY - 1), l_n = lane >> (P.lx_log + P.ly_log);
     const int TW = BW * LX, TH = BH * LY;
@@ -283,8 +290,8 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
 
     // A tile box carries rc channels, i.e. spb = rc / cc consecutive chunks; boxes q0..q_end
     // cover this block's chunks.  Box q is handed to the copy engine by one thread.
-    const int spb = P.rc / P.cc;
-    const int q0 = c_begin / spb, q_end = (c_end - 1) / spb;
+    const int spb = P.spb;
+    const int q0 = div_by(c_begin, P.mg_spb), q_end = div_by(c_end - 1, P.mg_spb);
     auto issue_box = [&](int q) {
         const int r = (q - q0) % kRawStages;
         const uint32_t dst = smem_base + (uint32_t)(P.raw_off_words + r * P.raw_stage_words) * 4u;
@@ -324,8 +331,8 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     int2 *tab = reinterpret_cast<int2 *>(smem + P.tab_off_words);
     int *srct = reinterpret_cast<int *>(smem + P.src_off_words);
     for (int q = tid; q < npix; q += nthreads) {
-        const int col = q % P.tin_w, t2 = q / P.tin_w;
-        const int row = t2 % P.tin_h, im = t2 / P.tin_h;
+        const int t2 = div_by(q, P.mg_tin_w), col = q - t2 * P.tin_w;
+        const int im = div_by(t2, P.mg_tin_h), row = t2 - im * P.tin_h;
         const int base = im * P.img_stride + row * P.pitch;
         const int bx = col >> 2, cq = col & 3;
         int d0 = -1, d1 = -1;
@@ -386,14 +393,15 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         // ===== producer warps: fill stage after stage; warp 0 also drives the copy engine =====
         if (!P.use_tma) asm volatile("griddepcontrol.wait;" ::: "memory");   // they read x themselves
         const int ptid = pw * 32 + lane;
-        for (int c = c_begin; c < c_end; ++c) {
-            const int k = c - c_begin, s = k % NS;
-            if (k >= NS && !mbar_wait(bar_empty(s), (uint32_t)((k / NS - 1) & 1), &abort_s, P.status)) break;
+        // chunk k uses stage s = k mod NS in its round ph = (k / NS) mod 2
+        for (int c = c_begin, s = 0, ph = 0; c < c_end; ++c, s = (s + 1 == NS ? 0 : s + 1), ph ^= (s == 0)) {
+            const int k = c - c_begin;
+            if (k >= NS && !mbar_wait(bar_empty(s), (uint32_t)(ph ^ 1), &abort_s, P.status)) break;
             if (pw == 0 && lane == 0 && k >= NS)      // the first NS chunks' commands are on their way already
                 issue_commands(s, seg[k * (P.wpc + 1)], seg[k * (P.wpc + 1) + P.wpc]);
             float *pl = reinterpret_cast<float *>(smem + P.plane_off_words + s * P.plane_stage_words);
             if (P.use_tma) {
-                const int q = c / spb, sub = c - q * spb;
+                const int q = div_by(c, P.mg_spb), sub = c - q * spb;
                 const int r = (q - q0) % kRawStages;
                 if ((k == 0 || sub == 0) &&
                     !mbar_wait(bar_raw(r), (uint32_t)(((q - q0) / kRawStages) & 1), &abort_s, P.status)) break;
@@ -505,9 +513,9 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         const uint32_t half_bytes = (uint32_t)P.half_stride * 4u;
 
         // --- main loop over channel chunks --------------------------------------------
-        for (int c = c_begin; c < c_end; ++c) {
-            const int k = c - c_begin, s = k % NS;
-            const uint32_t par = (uint32_t)((k / NS) & 1);
+        for (int c = c_begin, s = 0, ph = 0; c < c_end; ++c, s = (s + 1 == NS ? 0 : s + 1), ph ^= (s == 0)) {
+            const int k = c - c_begin;
+            const uint32_t par = (uint32_t)ph;
             if (!mbar_wait(bar_full(s), par, &abort_s, P.status)) break;
             if (!mbar_wait(bar_cmd(s), par, &abort_s, P.status)) break;
             const int s0 = seg[k * (P.wpc + 1)], sg = seg[k * (P.wpc + 1) + warp];
@@ -1023,6 +1031,10 @@ static xgen_status make_layout(const PackedHost &p, int n, int hh, int ww, bool 
     // A box carries at least 16 bytes of channels per pixel; a chunk may be a part of it.
     // The copy engine needs 16-byte multiples in every global stride.
     kp.rc = p.cc * xb >= 16 ? p.cc : 16 / xb;
+    kp.spb = kp.rc / p.cc;
+    auto magic = [](int d) { return d <= 1 ? 0u : (uint32_t)((1ull << 32) / (uint64_t)d + 1ull); };
+    kp.mg_tiles_x = magic(g.tiles_x); kp.mg_tiles_y = magic(g.tiles_y);
+    kp.mg_tin_w = magic(g.tin_w); kp.mg_tin_h = magic(g.tin_h); kp.mg_spb = magic(kp.spb);
     kp.use_tma = tma_ok && ((p.cc * xb) % 4 == 0) && (((size_t)p.c_in * xb) % 16 == 0) && g.tin_w <= 256 && g.tin_h <= 256 &&
                  !getenv("XGEN_PATCONV_NO_TMA");
     kp.box_bytes = npix_box * kp.rc * xb;
