@@ -357,12 +357,18 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
             srct[q] = ok ? ((gn * P.h + gy) * P.w + gx) * P.c_in : -1;
         }
     }
-    if (tid < P.wpc * P.J) soc_s[tid] = soc_v;                       // wpc * J <= 256 < threads of a block
+    // The staging warps need the table above and nothing of what follows: they wait for it
+    // here (named barrier 1, every thread of the block counted once) and start on the first
+    // tile, while the consumer warps only announce their entries and go on with their own tables.
+    if (producer) asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+    else { __threadfence_block(); asm volatile("bar.arrive 1, %0;" ::"r"(nthreads) : "memory"); }
+    const int cthreads = P.wpc * 32;
+    if (tid < P.wpc * P.J) soc_s[tid] = soc_v;                       // wpc * J <= consumer threads
     // Output-pixel table: linear pixel index of (sum t of lane l), or -1 outside the output.
     // Stride 1 keeps a row's four pixels as the pairs (0,2) and (1,3): sum 4*py + 2*h + e is
     // pixel (py, h + 2*e); stride 2: sum 2*py + e is pixel (py, e).
     int *ptab = reinterpret_cast<int *>(smem + P.ptab_off_words);
-    for (int i = tid; i < 32 * T; i += nthreads) {
+    for (int i = tid; !producer && i < 32 * T; i += cthreads) {
         const int t = i >> 5, l2 = i & 31;
         const int p_x = l2 & (LX - 1), p_y = (l2 >> P.lx_log) & (LY - 1), p_n = l2 >> (P.lx_log + P.ly_log);
         const int py = STRIDE == 1 ? (t >> 2) : (t >> 1);
@@ -372,20 +378,17 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     }
     // Segment offsets of this block's chunks.
     int *seg = reinterpret_cast<int *>(smem + P.seg_off_words);
-    if (tid < n_seg) seg[tid] = seg_v;
-    for (int i = tid + nthreads; i < n_seg; i += nthreads) seg[i] = seg_g[i];
-    // The consumer warps clear their running sums while the staging warps finish the tables.
     if (!producer) {
+        if (tid < n_seg) seg[tid] = seg_v;
+        for (int i = tid + cthreads; i < n_seg; i += cthreads) seg[i] = seg_g[i];
+        // and clear their running sums
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t tw = tmem_base_s + (((uint32_t)(warp & 3) * 32u) << 16) + (uint32_t)((warp >> 2) * P.cols_per_warp);
         const uint32_t z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         for (int c = 0; c < P.cols_per_warp; c += 8) tmem_st8(tw + c, z);
         tmem_wait_st();
+        asm volatile("bar.sync 2, %0;" ::"r"(cthreads) : "memory");   // the consumer warps' tables are complete
     }
-
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_cta = tmem_base_s;
     const uint32_t plane_bytes = (uint32_t)P.plane_stride * 4u, pitch_bytes = (uint32_t)P.pitch * 4u;
 
@@ -393,12 +396,19 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         // ===== producer warps: fill stage after stage; warp 0 also drives the copy engine =====
         if (!P.use_tma) asm volatile("griddepcontrol.wait;" ::: "memory");   // they read x themselves
         const int ptid = pw * 32 + lane;
+        // Offsets of the next chunk's commands (the consumer warps' copy in shared memory may not
+        // be written yet), fetched one chunk ahead by the thread that hands them to the copy engine.
+        const bool cmd_thread = pw == 0 && lane == 0;
+        int cmd_s0 = 0, cmd_s1 = 0;
+        if (cmd_thread && c_begin + NS < c_end) { cmd_s0 = __ldg(seg_g + NS * (P.wpc + 1)); cmd_s1 = __ldg(seg_g + NS * (P.wpc + 1) + P.wpc); }
         // chunk k uses stage s = k mod NS in its round ph = (k / NS) mod 2
         for (int c = c_begin, s = 0, ph = 0; c < c_end; ++c, s = (s + 1 == NS ? 0 : s + 1), ph ^= (s == 0)) {
             const int k = c - c_begin;
             if (k >= NS && !mbar_wait(bar_empty(s), (uint32_t)(ph ^ 1), &abort_s, P.status)) break;
-            if (pw == 0 && lane == 0 && k >= NS)      // the first NS chunks' commands are on their way already
-                issue_commands(s, seg[k * (P.wpc + 1)], seg[k * (P.wpc + 1) + P.wpc]);
+            if (cmd_thread && k >= NS) {              // the first NS chunks' commands are on their way already
+                issue_commands(s, cmd_s0, cmd_s1);
+                if (c + 1 < c_end) { cmd_s0 = __ldg(seg_g + (k + 1) * (P.wpc + 1)); cmd_s1 = __ldg(seg_g + (k + 1) * (P.wpc + 1) + P.wpc); }
+            }
             float *pl = reinterpret_cast<float *>(smem + P.plane_off_words + s * P.plane_stage_words);
             if (P.use_tma) {
                 const int q = div_by(c, P.mg_spb), sub = c - q * spb;
