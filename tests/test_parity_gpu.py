@@ -184,6 +184,36 @@ def test_planned_runs_back_to_back_and_replanned():
     compare(d, run_gpu(pk, d.x, d.bias, True))          # the first shape now runs unsplit
 
 
+@pytest.mark.parametrize("c_out", [64, 160])
+def test_unsplit_runs_back_to_back_overlap(c_out):
+    """Launches follow each other on one stream without a host synchronisation: a kernel may be
+    scheduled while its predecessor drains (programmatic stream serialisation), so its blocks start
+    at different times and its prologue overlaps foreign work.  64 output channels give 8 consumer
+    warps per block, 160 give 16; several images make more blocks than the GPU holds at once.
+    The second layer of each pair reads what the first one wrote."""
+    import torch
+    d1 = _layer("f32", 6, 24, c_out, 40, 40, 1, prune=0.5, lib=8, seed=41)
+    d2 = _layer("f32", 6, c_out, 32, 40, 40, 1, prune=0.5, lib=8, seed=42)
+    p1, p2 = pack(d1), pack(d2)
+    x = torch.from_numpy(d1.x).cuda()
+    b1 = torch.from_numpy(d1.bias).cuda()
+    b2 = torch.from_numpy(d2.bias).cuda()
+    st = torch.cuda.current_stream().cuda_stream
+    mids = [torch.full((6, 40, 40, c_out), 777.0, device="cuda") for _ in range(6)]
+    outs = [torch.full((6, 40, 40, 32), 777.0, device="cuda") for _ in range(6)]
+    for m, o in zip(mids, outs):
+        p1.run(x.data_ptr(), 6, 40, 40, b1.data_ptr(), True, m.data_ptr(), st)
+        p2.run(m.data_ptr(), 6, 40, 40, b2.data_ptr(), True, o.data_ptr(), st)
+    p2.sync(st)
+    mid = mids[0].cpu().numpy()
+    compare(d1, mid)
+    out = outs[0].cpu().numpy()
+    compare(d2, out, x=mid)
+    for m, o in zip(mids[1:], outs[1:]):
+        assert np.array_equal(m.cpu().numpy(), mid)
+        assert np.array_equal(o.cpu().numpy(), out)
+
+
 def test_planned_long_integer_layer():
     # more than 128 input channels: the integer variant folds its exact fp32 partial sums into
     # int32 totals on the way, and the split exchanges those totals
