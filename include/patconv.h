@@ -188,7 +188,8 @@ xgen_status xgen_patconv_run_static_scratch(const xgen_patconv_packed *packed, c
 
 /*
  * Convenience for callers that hold host tensors: copies x (and bias) to the
- * device, runs the layer on the default stream, copies y back and waits.  The
+ * device, runs the layer on the default stream, copies y back and waits
+ * (xgen_patconv_enqueue_host followed by the wait).  The
  * device staging buffers belong to the handle and are kept between calls (they
  * only grow); calls on one handle are serialised.  Pinned (page-locked) host
  * memory makes the copies faster but is not required.  Same tensor layouts as
@@ -197,6 +198,27 @@ xgen_status xgen_patconv_run_static_scratch(const xgen_patconv_packed *packed, c
 xgen_status xgen_patconv_run_host(const xgen_patconv_packed *packed, const void *x_host, int32_t n,
                                   int32_t h, int32_t w, const void *bias_host, int32_t relu,
                                   void *y_host);
+
+/*
+ * The same three steps, only enqueued, without waiting: x (and bias) are copied to the
+ * handle's device staging buffers on a stream of the handle's own, the layer (Sec. 2.1,
+ * Sec. 2.2, as xgen_patconv_run) runs on cuda_stream (NULL = the default stream) once they
+ * are there, and y is copied back on a second stream of the handle's own.  The caller's
+ * stream thus carries kernels only: with page-locked host memory the call returns at once
+ * and a sequence of such calls on different handles overlaps the copies in, the kernels
+ * and the copies out with each other, in one caller stream.  With pageable memory the
+ * copies may block the caller.  x_host and bias_host must stay unchanged, and y_host is
+ * undefined, until xgen_patconv_last_status(packed, cuda_stream) has returned: it waits
+ * for the stream and for the handle's copies and reports a kernel whose bounded wait ran
+ * out.  Work enqueued on cuda_stream after this call is NOT ordered after the copy of y.
+ * A further host-buffer call on the same handle waits, on the device, until this one
+ * has released the staging buffers.  A staging buffer that has to grow is reallocated,
+ * which synchronises the device; streams and events are created at the first call.  Not
+ * for use inside a stream capture.  Errors as xgen_patconv_run, plus ALLOC.
+ */
+xgen_status xgen_patconv_enqueue_host(const xgen_patconv_packed *packed, const void *x_host, int32_t n,
+                                      int32_t h, int32_t w, const void *bias_host, int32_t relu,
+                                      void *y_host, void *cuda_stream);
 
 /*
  * Optional: prepare the handle for one input shape.  Layers with few output

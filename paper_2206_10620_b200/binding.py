@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_PATTERN", 3: "SHAPE", 4: "UNS
                 5: "ALLOC", 6: "CUDA", 7: "TIMEOUT"}
 
 EXPORTS = ["xgen_patconv_pack", "xgen_patconv_run", "xgen_patconv_run_static_scratch",
-           "xgen_patconv_run_host", "xgen_patconv_plan",
+           "xgen_patconv_run_host", "xgen_patconv_enqueue_host", "xgen_patconv_plan",
            "xgen_patconv_out_shape", "xgen_patconv_query", "xgen_patconv_view",
            "xgen_patconv_last_status", "xgen_patconv_free", "xgen_strerror",
            "xgen_patconv_launch_count"]
@@ -74,6 +74,7 @@ def lib():
         L.xgen_patconv_run.argtypes = [P, P, I, I, I, P, I, P, P]
         L.xgen_patconv_run_static_scratch.argtypes = [P, P, I, I, I, P, I, P, I, P]
         L.xgen_patconv_run_host.argtypes = [P, P, I, I, I, P, I, P]
+        L.xgen_patconv_enqueue_host.argtypes = [P, P, I, I, I, P, I, P, P]
         L.xgen_patconv_plan.argtypes = [P, I, I, I]
         L.xgen_patconv_out_shape.argtypes = [P, I, I, ctypes.POINTER(I), ctypes.POINTER(I)]
         L.xgen_patconv_query.argtypes = [P, ctypes.POINTER(Stats)]
@@ -185,6 +186,12 @@ class Packed:
                                            None if b is None else b.ctypes.data, int(bool(relu)),
                                            y.ctypes.data), "xgen_patconv_run_host")
         return y
+
+    def enqueue_host_ptr(self, x_ptr, n, h, w, bias_ptr, relu, y_ptr, stream=0):
+        """xgen_patconv_enqueue_host on raw host addresses (pinned buffers) and a raw
+        cudaStream_t; returns without waiting, sync(stream) waits."""
+        _check(lib().xgen_patconv_enqueue_host(self._h, x_ptr, n, h, w, bias_ptr or None, int(bool(relu)), y_ptr,
+                                               stream or None), "xgen_patconv_enqueue_host")
 
     def run_host_ptr(self, x_ptr, n, h, w, bias_ptr, relu, y_ptr):
         """xgen_patconv_run_host on raw host addresses (e.g. pinned buffers)."""

@@ -795,6 +795,10 @@ struct xgen_patconv_packed {
     mutable std::mutex host_mu;
     mutable void *d_hx = nullptr, *d_hy = nullptr, *d_hb = nullptr;
     mutable size_t hx_bytes = 0, hy_bytes = 0;
+    // their copies run on two streams of the handle's own, tied to the caller's stream by events
+    mutable cudaStream_t s_in = nullptr, s_out = nullptr;
+    mutable cudaEvent_t ev_in = nullptr, ev_run = nullptr, ev_out = nullptr;
+    mutable bool host_call_before = false;
 };
 
 static void free_device_layout(xgen_patconv_packed *h) {
@@ -966,6 +970,11 @@ void xgen_patconv_free(xgen_patconv_packed *h) {
     if (h->d_hx) cudaFree(h->d_hx);
     if (h->d_hy) cudaFree(h->d_hy);
     if (h->d_hb) cudaFree(h->d_hb);
+    if (h->s_in) cudaStreamDestroy(h->s_in);
+    if (h->s_out) cudaStreamDestroy(h->s_out);
+    if (h->ev_in) cudaEventDestroy(h->ev_in);
+    if (h->ev_run) cudaEventDestroy(h->ev_run);
+    if (h->ev_out) cudaEventDestroy(h->ev_out);
     delete h;
 }
 
@@ -997,6 +1006,7 @@ xgen_status xgen_patconv_last_status(const xgen_patconv_packed *h, void *stream)
     if (!h) return XGEN_ERR_INVALID_ARG;
     cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) return XGEN_ERR_CUDA;
+    if (h->s_out && cudaStreamSynchronize(h->s_out) != cudaSuccess) return XGEN_ERR_CUDA;   // copies out of host-buffer calls
     if (cudaGetLastError() != cudaSuccess) return XGEN_ERR_CUDA;
     if (h->d_status) {
         // a kernel whose bounded wait for a tile copy ran out leaves a mark here
@@ -1359,8 +1369,8 @@ xgen_status xgen_patconv_run_static_scratch(const xgen_patconv_packed *h, const 
     return run_layer(h, x, n, hh, ww, bias, relu, y, stream, &choice);
 }
 
-xgen_status xgen_patconv_run_host(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
-                                  const void *bias, int32_t relu, void *y) {
+xgen_status xgen_patconv_enqueue_host(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
+                                      const void *bias, int32_t relu, void *y, void *stream) {
     if (!h || !x || !y) return XGEN_ERR_INVALID_ARG;
     if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
     if (h->device < 0) return XGEN_ERR_CUDA;
@@ -1371,7 +1381,8 @@ xgen_status xgen_patconv_run_host(const xgen_patconv_packed *h, const void *x, i
     const size_t xbytes = (size_t)n * hh * ww * p.c_in * xb, ybytes = (size_t)n * ho * wo * p.c_out * yb;
     int prev = 0;
     if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
-    std::lock_guard<std::mutex> lock(h->host_mu);      // one host-buffer call per handle at a time
+    std::lock_guard<std::mutex> lock(h->host_mu);      // one host-buffer call per handle is enqueued at a time
+    cudaStream_t st = (cudaStream_t)stream;
     xgen_status rs = XGEN_OK;
     cudaError_t e = cudaSuccess;
     if (xbytes > h->hx_bytes) {
@@ -1387,19 +1398,48 @@ xgen_status xgen_patconv_run_host(const xgen_patconv_packed *h, const void *x, i
         if (e == cudaSuccess) h->hy_bytes = ybytes;
     }
     if (e == cudaSuccess && bias && !h->d_hb) e = cudaMalloc(&h->d_hb, (size_t)p.c_out * 4);
+    if (e == cudaSuccess && !h->s_in) e = cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking);
+    if (e == cudaSuccess && !h->s_out) e = cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking);
+    if (e == cudaSuccess && !h->ev_in) e = cudaEventCreateWithFlags(&h->ev_in, cudaEventDisableTiming);
+    if (e == cudaSuccess && !h->ev_run) e = cudaEventCreateWithFlags(&h->ev_run, cudaEventDisableTiming);
+    if (e == cudaSuccess && !h->ev_out) e = cudaEventCreateWithFlags(&h->ev_out, cudaEventDisableTiming);
     if (e != cudaSuccess) { rs = XGEN_ERR_ALLOC; cudaGetLastError(); }
     void *dx = h->d_hx, *dy = h->d_hy, *db = bias ? h->d_hb : nullptr;
+    // Copy in on the handle's first stream, the layer on the caller's, copy out on the handle's
+    // second stream: the caller's stream carries kernels only, so the copies of one handle
+    // overlap the kernels and the copies (in the other direction) of other handles.
     if (rs == XGEN_OK) {
-        e = cudaMemcpyAsync(dx, x, xbytes, cudaMemcpyHostToDevice, 0);
-        if (e == cudaSuccess && bias) e = cudaMemcpyAsync(db, bias, (size_t)p.c_out * 4, cudaMemcpyHostToDevice, 0);
+        if (h->host_call_before) {
+            e = cudaStreamWaitEvent(h->s_in, h->ev_run, 0);           // the earlier call's kernel has read x and bias
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(st, h->ev_out, 0);   // and its copy out has read y
+        }
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dx, x, xbytes, cudaMemcpyHostToDevice, h->s_in);
+        if (e == cudaSuccess && bias) e = cudaMemcpyAsync(db, bias, (size_t)p.c_out * 4, cudaMemcpyHostToDevice, h->s_in);
+        if (e == cudaSuccess) e = cudaEventRecord(h->ev_in, h->s_in);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, h->ev_in, 0);
         if (e != cudaSuccess) rs = XGEN_ERR_CUDA;
     }
-    if (rs == XGEN_OK) rs = xgen_patconv_run(h, dx, n, hh, ww, db, relu, dy, nullptr);
+    if (rs == XGEN_OK) rs = xgen_patconv_run(h, dx, n, hh, ww, db, relu, dy, stream);
     if (rs == XGEN_OK) {
-        e = cudaMemcpyAsync(y, dy, ybytes, cudaMemcpyDeviceToHost, 0);
-        if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+        e = cudaEventRecord(h->ev_run, st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(h->s_out, h->ev_run, 0);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(y, dy, ybytes, cudaMemcpyDeviceToHost, h->s_out);
+        if (e == cudaSuccess) e = cudaEventRecord(h->ev_out, h->s_out);
         if (e != cudaSuccess) rs = XGEN_ERR_CUDA;
+        h->host_call_before = true;
     }
+    cudaSetDevice(prev);
+    return rs;
+}
+
+xgen_status xgen_patconv_run_host(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
+                                  const void *bias, int32_t relu, void *y) {
+    xgen_status rs = xgen_patconv_enqueue_host(h, x, n, hh, ww, bias, relu, y, nullptr);
+    if (rs != XGEN_OK) return rs;
+    int prev = 0;
+    if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
+    if (cudaStreamSynchronize(0) != cudaSuccess) rs = XGEN_ERR_CUDA;
+    if (h->s_out && cudaStreamSynchronize(h->s_out) != cudaSuccess) rs = XGEN_ERR_CUDA;
     cudaSetDevice(prev);
     return rs;
 }

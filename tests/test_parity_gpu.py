@@ -104,6 +104,31 @@ def test_int8_extremes_and_long_reduction():
     compare(d, run_gpu(pack(d), d.x, d.bias, True))
 
 
+def test_enqueue_host_overlapping_calls():
+    """Host-buffer calls that only enqueue: two handles in turn on one stream, each several
+    times (a later call on a handle has to wait for the staging buffers of the earlier one),
+    results read after xgen_patconv_last_status."""
+    import torch
+    da = _layer("f32", 3, 40, 48, 30, 30, 1, prune=0.5, lib=8, seed=51)
+    db = _layer("f16", 2, 64, 24, 21, 21, 2, prune=0.4, lib=8, seed=52)
+    pa, pb = pack(da), pack(db)
+    st = torch.cuda.current_stream().cuda_stream
+    bufs = []
+    for rep in range(3):
+        for d, pk in ((da, pa), (db, pb)):
+            hx = torch.from_numpy(d.x * (rep + 1) if d.spec.dtype == "f32" else d.x).pin_memory()
+            hb = torch.from_numpy(d.bias).pin_memory()
+            ho, wo = pk.out_shape(d.spec.h, d.spec.w)
+            hy = torch.full((d.spec.n, ho, wo, d.spec.c_out), 777.0,
+                            dtype=torch.float32 if d.spec.dtype == "f32" else torch.float16).pin_memory()
+            pk.enqueue_host_ptr(hx.data_ptr(), d.spec.n, d.spec.h, d.spec.w, hb.data_ptr(), True, hy.data_ptr(), st)
+            bufs.append((d, hx, hy))
+    pa.sync(st)
+    pb.sync(st)
+    for d, hx, hy in bufs:
+        compare(d, hy.numpy(), x=hx.numpy())
+
+
 def test_run_host_entry_point():
     d = _layer("f16", 2, 32, 48, 20, 20)
     pk = pack(d)
