@@ -249,8 +249,8 @@ xgen_status xgen_patconv_query(const xgen_patconv_packed *packed, xgen_patconv_s
 /* Fill *view with pointers into the handle's host copy of the packed layout. */
 xgen_status xgen_patconv_view(const xgen_patconv_packed *packed, xgen_patconv_host_view *view);
 
-/* Synchronise the stream and report the first CUDA error seen on it, as a
- * status (XGEN_OK, XGEN_ERR_CUDA).  The kernels contain no unbounded waits: a wait
+/* Synchronise the stream (and the handle's own copy streams, if xgen_patconv_enqueue_host was
+ * used on it) and report the first CUDA error seen, as a status (XGEN_OK, XGEN_ERR_CUDA).  The kernels contain no unbounded waits: a wait
  * (for a staged tile, a free stage, or the other blocks of a split) that runs out
  * of its bound marks the handle, the kernel still ends, and this call then returns
  * XGEN_ERR_TIMEOUT once (results are invalid; the split counters are reset). */
