@@ -931,7 +931,8 @@ xgen_status xgen_patconv_pack(const xgen_patconv_desc *desc, const void *dense_w
     xgen_status st;
     try {
         PackConfig cfg = choose_pack_config(desc->c_in, desc->c_out, desc->dtype, desc->stride);
-        if (const char *e = getenv("XGEN_PATCONV_J")) { int v = atoi(e); if (v == 4 || v == 8 || v == 16 || v == 32) {
+        // a group is stored in pieces of 8 adjacent channels (32-byte stores): whole pieces only
+        if (const char *e = getenv("XGEN_PATCONV_J")) { int v = atoi(e); if (v == 8 || v == 16) {
             cfg.filters_per_group = v;
             int groups = (desc->c_out + v - 1) / v; cfg.groups_per_block = groups < kMaxWarps ? groups : kMaxWarps; } }
         if (const char *e = getenv("XGEN_PATCONV_WPC")) { int v = atoi(e); if (v >= 1 && v <= kMaxWarps) {
