@@ -63,9 +63,13 @@ typedef struct {
     int64_t kernels_surviving;    /* kernels with a pattern (not removed)                     */
     int64_t macs_per_pixel;       /* 4 * kernels_surviving: useful multiply-adds per output pixel */
     int64_t weight_bytes;         /* bytes of kept weights at the layer's storage precision   */
-    int64_t index_bytes;          /* bytes a compact encoding of this layout spends on
-                                     everything that is not a weight: one opcode byte and one
-                                     operand byte per command, plus the offset and slot tables */
+    int64_t index_bytes;          /* bytes the device copy stores beyond weight_bytes: the
+                                     command stream (48-byte slots: 16 bytes of opcode and
+                                     operand, every kept weight widened to fp32 and stored
+                                     twice) plus the offset and slot tables, less weight_bytes */
+    int64_t compact_index_bytes;  /* the information in those bytes: one opcode byte and one
+                                     operand byte per command, plus the offset and slot tables
+                                     (what a byte-packed encoding of this layout would take)   */
     int64_t csr_index_bytes;      /* index bytes CSR would need for the same non-zeros
                                      (one 4-byte column per weight + one row pointer per filter) */
     int64_t stream_bytes;         /* bytes of the command stream as stored on the device
@@ -135,18 +139,21 @@ xgen_status xgen_patconv_pack(const xgen_patconv_desc *desc, const void *dense_w
  * Run the layer (paper Sec. 2.3, "Load Redundancy Elimination": tiled input,
  * per-pattern code with static tap offsets; Sec. 2.2: bias and ReLU fused).
  *   x_dev    [n][h][w][c_in]  NHWC, dtype's activation type, 16-byte aligned
- *   bias_dev [c_out] fp32 (int32 for XGEN_I8_I32) or NULL for no bias
+ *   bias_dev [c_out] fp32 (int32 for XGEN_I8_I32), 4-byte aligned, or NULL for no bias
  *   relu     non-zero applies max(.,0)
  *   y_dev    [n][ho][wo][c_out] NHWC, 16-byte aligned, must not overlap x_dev;
  *            ho, wo as xgen_patconv_out_shape reports
  *   cuda_stream  a cudaStream_t passed as void* (NULL = default stream)
- * Only enqueues work on the stream: no synchronisation, no allocation.  The
- * caller keeps x, bias and y alive until the stream reaches that work.  The
- * handle is not modified, so concurrent calls on different streams are allowed
- * (for a shape prepared with xgen_patconv_plan, which uses a workspace owned by
- * the handle, concurrent calls must be on one stream).
- * Errors: INVALID_ARG, SHAPE (n,h,w < 1 or a tensor beyond 2^31-1 elements),
- * CUDA (launch failure or host-only handle).
+ * Only enqueues work on the stream: no synchronisation, no device allocation.
+ * The caller keeps x, bias and y alive until the stream reaches that work.
+ * Concurrent calls on different streams are allowed for unplanned shapes (the
+ * handle only remembers, under a lock, the launch geometry and tensor map of the
+ * last few (shape, x address) pairs, so repeated calls skip that work).  For a
+ * shape prepared with xgen_patconv_plan see the rules there.
+ * Errors: INVALID_ARG (null or misaligned pointer, y overlapping x), SHAPE
+ * (n,h,w < 1 or a tensor beyond 2^31-1 elements), UNSUPPORTED (a tile of this
+ * shape does not fit shared or tensor memory), CUDA (launch failure or
+ * host-only handle).
  */
 xgen_status xgen_patconv_run(const xgen_patconv_packed *packed, const void *x_dev, int32_t n,
                              int32_t h, int32_t w, const void *bias_dev, int32_t relu,
@@ -167,8 +174,10 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *packed, const void *x_de
  *            output pixels, and cost splits x 4 bytes of scratch per output element
  *   others   exactly as xgen_patconv_run; the caller still owns x, bias and y
  *
- * Limit: splits x n*ho*wo*c_out x 4 bytes must not exceed
- * XGEN_PATCONV_STATIC_SCRATCH_BYTES; beyond that the call returns XGEN_ERR_SHAPE and
+ * Limit: s x n*ho*wo*c_out x 4 bytes must not exceed
+ * XGEN_PATCONV_STATIC_SCRATCH_BYTES, where s is the number of splits that actually get
+ * channel chunks (splits after clamping, rounded so that every split has the same
+ * number of chunks; s = 1 needs no scratch); beyond that the call returns XGEN_ERR_SHAPE and
  * launches nothing (with XGEN_PATCONV_LOG set, the reason goes to stderr).  The array is
  * part of the loaded library: every GPU that uses the library holds those bytes until
  * the process exits.
@@ -226,18 +235,85 @@ xgen_status xgen_patconv_enqueue_host(const xgen_patconv_packed *packed, const v
  * such a shape this call lets later xgen_patconv_run calls split the input
  * channels across thread blocks (the paper does not discuss this; it is the
  * cross-channel reduction of this implementation).  The blocks of a split write
- * their partial sums to a workspace, count themselves in, wait (with a bound)
- * for the others and each reduce a share, all inside the one kernel: the split
- * count is chosen so that every block of the launch is resident at once on an
- * otherwise idle GPU (other work on the GPU at the same time can only delay the
- * blocks; a wait that runs out is reported by xgen_patconv_last_status).  The call allocates the workspace and the
- * counters, owned by the handle, so it synchronises and must not be called
- * while the handle is in use; planned runs of one handle share them and must
- * not overlap on the GPU (use one stream, or order them with events).  Without
- * this call every shape runs unsplit.
- * Errors: INVALID_ARG, SHAPE, ALLOC, CUDA.
+ * their partial sums to a workspace, count themselves in, wait (with a bound in
+ * time) for the others and each reduce a share, all inside the one kernel.
+ * Because they wait for each other, the split count is chosen so that every
+ * block of the launch is resident at once on an otherwise idle GPU.  Hence the
+ * rule: a planned split launch must not share the GPU with another planned
+ * split launch -- of this handle (they also share the workspace) or of any
+ * other handle -- nor with any other kernel that may keep its blocks from
+ * becoming resident; put such launches on one stream or order them with
+ * events.  If the rule is broken the blocks may hold each other's places; the
+ * waits then run out (default 2 s), the kernel ends, its results are invalid,
+ * and xgen_patconv_last_status returns XGEN_ERR_TIMEOUT (xgen_patconv_run has
+ * returned XGEN_OK long before: it only enqueues).  Work that merely delays the
+ * blocks (a kernel running before them on the same stream) is harmless.
+ * The call allocates the workspace and the counters, owned by the handle, so it
+ * synchronises the device and must not be called while the handle is in use.
+ * Without this call every shape runs unsplit.
+ * Errors: INVALID_ARG, SHAPE, UNSUPPORTED, ALLOC, CUDA.
  */
 xgen_status xgen_patconv_plan(xgen_patconv_packed *packed, int32_t n, int32_t h, int32_t w);
+
+/*
+ * The tuning-decided parameters of a layer (paper Sec. 2.3: the Layerwise
+ * Representation carries "tuning-decided parameters" next to the pattern
+ * information).  xgen_patconv_plan chooses them itself; a caller that has
+ * measured better ones passes them here.  Zero in every field = the library's
+ * own choice.
+ *   splits             channel splits of the planned shape (clamped to what is
+ *                      resident at once and to the number of channel chunks)
+ *   no_copy_engine     stage input tiles with plain loads instead of the tensor
+ *                      copy engine (every later run of the handle)
+ *   no_launch_overlap  launch without programmatic stream serialisation, i.e. a
+ *                      run starts only when its predecessor in the stream has
+ *                      ended (every later run of the handle)
+ *   wait_limit_ms      bound of the device-side waits, milliseconds (default
+ *                      2000, at most 60000)
+ */
+typedef struct {
+    int32_t splits;
+    int32_t no_copy_engine;
+    int32_t no_launch_overlap;
+    int32_t wait_limit_ms;
+} xgen_patconv_tuning;
+
+/* xgen_patconv_plan with the caller's tuning (NULL = xgen_patconv_plan).  Errors as
+ * xgen_patconv_plan, plus INVALID_ARG for a negative field. */
+xgen_status xgen_patconv_plan_tuned(xgen_patconv_packed *packed, int32_t n, int32_t h, int32_t w,
+                                    const xgen_patconv_tuning *tuning);
+
+/* How a run of an n x h x w input would be launched with the handle as it stands. */
+typedef struct {
+    int32_t splits;             /* channel splits (1 = unsplit; > 1 only for the planned shape)   */
+    int32_t chunks_per_split;
+    int32_t tiles;              /* pixel tiles                                                     */
+    int32_t filter_blocks;      /* blocks of output channels                                       */
+    int32_t items;              /* tiles x filter_blocks                                           */
+    int32_t blocks;             /* thread blocks of the launch: items x splits                     */
+    int32_t threads_per_block;
+    int32_t lanes_x, lanes_y, lanes_n;  /* how a warp's 32 lanes tile x, y and images             */
+    int32_t pixels_per_lane;    /* output pixels one lane owns (16 at stride 1, 8 at stride 2)     */
+    int32_t stages;             /* pipeline stages of staged channel chunks                        */
+    int32_t uses_copy_engine;   /* input tiles arrive through the tensor copy engine               */
+    int64_t shared_bytes;       /* dynamic shared memory per block                                 */
+    int64_t workspace_bytes;    /* partial-sum workspace of the planned split, 0 if unsplit        */
+} xgen_patconv_plan_stats;
+
+/* Fill *stats for the shape.  No CUDA work is enqueued.  Errors: INVALID_ARG, SHAPE, UNSUPPORTED. */
+xgen_status xgen_patconv_plan_info(const xgen_patconv_packed *packed, int32_t n, int32_t h, int32_t w,
+                                   xgen_patconv_plan_stats *stats);
+
+/*
+ * Testing aid, not for production use (the paper has no counterpart): make every later
+ * planned split launch of the handle wait for `extra` arrivals more than its own blocks
+ * will ever deliver.  With extra > 0 the wait of every block runs out after the handle's
+ * wait limit (xgen_patconv_tuning.wait_limit_ms), the kernel ends normally, and
+ * xgen_patconv_last_status returns XGEN_ERR_TIMEOUT once; extra = 0 restores normal
+ * operation.  This is how the tests exercise the bounded waits without hanging or
+ * faulting the GPU.  Errors: INVALID_ARG.
+ */
+xgen_status xgen_patconv_test_expect_arrivals(xgen_patconv_packed *packed, int32_t extra);
 
 /* Output extents for an h x w input: ho = (h + 2 - 3) / stride + 1, likewise wo. */
 xgen_status xgen_patconv_out_shape(const xgen_patconv_packed *packed, int32_t h, int32_t w,
@@ -253,7 +329,8 @@ xgen_status xgen_patconv_view(const xgen_patconv_packed *packed, xgen_patconv_ho
  * used on it) and report the first CUDA error seen, as a status (XGEN_OK, XGEN_ERR_CUDA).  The kernels contain no unbounded waits: a wait
  * (for a staged tile, a free stage, or the other blocks of a split) that runs out
  * of its bound marks the handle, the kernel still ends, and this call then returns
- * XGEN_ERR_TIMEOUT once (results are invalid; the split counters are reset). */
+ * XGEN_ERR_TIMEOUT once (results are invalid; the split counters are reset).  The
+ * waits are bounded in time: 2 s unless xgen_patconv_tuning.wait_limit_ms says otherwise. */
 xgen_status xgen_patconv_last_status(const xgen_patconv_packed *packed, void *cuda_stream);
 
 /* Release the handle and its device memory.  NULL is allowed. */

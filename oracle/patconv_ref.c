@@ -28,7 +28,9 @@
  *
  * Parity status: pinned (hand-computed cases, impulse response, constant-input
  * closed forms, pruned-contributes-nothing, linearity, a library convolution on
- * the masked dense tensor, a scatter-form brute force) -- see the CPU tests.
+ * the masked dense tensor, a scatter-form brute force; the error scale s_abs by a
+ * hand-computed case, by S == y for non-negative terms, by S(x, W, b) ==
+ * y(|x|, |W|, |b|) and by homogeneity) -- see the CPU tests.
  */
 #include <stdint.h>
 #include <stdlib.h>

@@ -23,6 +23,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_PATTERN", 3: "SHAPE", 4: "UNS
 
 EXPORTS = ["xgen_patconv_pack", "xgen_patconv_run", "xgen_patconv_run_static_scratch",
            "xgen_patconv_run_host", "xgen_patconv_enqueue_host", "xgen_patconv_plan",
+           "xgen_patconv_plan_tuned", "xgen_patconv_plan_info", "xgen_patconv_test_expect_arrivals",
            "xgen_patconv_out_shape", "xgen_patconv_query", "xgen_patconv_view",
            "xgen_patconv_last_status", "xgen_patconv_free", "xgen_strerror",
            "xgen_patconv_launch_count"]
@@ -37,13 +38,28 @@ class Desc(ctypes.Structure):
 class Stats(ctypes.Structure):
     _fields_ = [("kernels_total", ctypes.c_int64), ("kernels_surviving", ctypes.c_int64),
                 ("macs_per_pixel", ctypes.c_int64), ("weight_bytes", ctypes.c_int64),
-                ("index_bytes", ctypes.c_int64), ("csr_index_bytes", ctypes.c_int64),
+                ("index_bytes", ctypes.c_int64), ("compact_index_bytes", ctypes.c_int64),
+                ("csr_index_bytes", ctypes.c_int64),
                 ("stream_bytes", ctypes.c_int64),
                 ("filters_per_group", ctypes.c_int32), ("groups_per_block", ctypes.c_int32),
                 ("n_blocks", ctypes.c_int32), ("channels_per_chunk", ctypes.c_int32),
                 ("n_chunks", ctypes.c_int32), ("patterns_compiled", ctypes.c_int32),
                 ("max_segment_slots", ctypes.c_int32),
                 ("load_commands", ctypes.c_int64), ("group_imbalance", ctypes.c_double)]
+
+
+class Tuning(ctypes.Structure):
+    _fields_ = [("splits", ctypes.c_int32), ("no_copy_engine", ctypes.c_int32),
+                ("no_launch_overlap", ctypes.c_int32), ("wait_limit_ms", ctypes.c_int32)]
+
+
+class PlanStats(ctypes.Structure):
+    _fields_ = [("splits", ctypes.c_int32), ("chunks_per_split", ctypes.c_int32), ("tiles", ctypes.c_int32),
+                ("filter_blocks", ctypes.c_int32), ("items", ctypes.c_int32), ("blocks", ctypes.c_int32),
+                ("threads_per_block", ctypes.c_int32), ("lanes_x", ctypes.c_int32), ("lanes_y", ctypes.c_int32),
+                ("lanes_n", ctypes.c_int32), ("pixels_per_lane", ctypes.c_int32), ("stages", ctypes.c_int32),
+                ("uses_copy_engine", ctypes.c_int32), ("shared_bytes", ctypes.c_int64),
+                ("workspace_bytes", ctypes.c_int64)]
 
 
 class HostView(ctypes.Structure):
@@ -76,6 +92,9 @@ def lib():
         L.xgen_patconv_run_host.argtypes = [P, P, I, I, I, P, I, P]
         L.xgen_patconv_enqueue_host.argtypes = [P, P, I, I, I, P, I, P, P]
         L.xgen_patconv_plan.argtypes = [P, I, I, I]
+        L.xgen_patconv_plan_tuned.argtypes = [P, I, I, I, ctypes.POINTER(Tuning)]
+        L.xgen_patconv_plan_info.argtypes = [P, I, I, I, ctypes.POINTER(PlanStats)]
+        L.xgen_patconv_test_expect_arrivals.argtypes = [P, I]
         L.xgen_patconv_out_shape.argtypes = [P, I, I, ctypes.POINTER(I), ctypes.POINTER(I)]
         L.xgen_patconv_query.argtypes = [P, ctypes.POINTER(Stats)]
         L.xgen_patconv_view.argtypes = [P, ctypes.POINTER(HostView)]
@@ -156,8 +175,21 @@ class Packed:
             "masks": arr(v.compiled_masks, npc, ctypes.c_uint16, np.uint16),
         }
 
-    def plan(self, n, h, w):
-        _check(lib().xgen_patconv_plan(self._h, n, h, w), "xgen_patconv_plan")
+    def plan(self, n, h, w, splits=0, no_copy_engine=False, no_launch_overlap=False, wait_limit_ms=0):
+        """xgen_patconv_plan, or xgen_patconv_plan_tuned when any tuning field is given."""
+        if splits or no_copy_engine or no_launch_overlap or wait_limit_ms:
+            t = Tuning(int(splits), int(bool(no_copy_engine)), int(bool(no_launch_overlap)), int(wait_limit_ms))
+            _check(lib().xgen_patconv_plan_tuned(self._h, n, h, w, ctypes.byref(t)), "xgen_patconv_plan_tuned")
+        else:
+            _check(lib().xgen_patconv_plan(self._h, n, h, w), "xgen_patconv_plan")
+
+    def plan_info(self, n, h, w) -> dict:
+        s = PlanStats()
+        _check(lib().xgen_patconv_plan_info(self._h, n, h, w, ctypes.byref(s)), "xgen_patconv_plan_info")
+        return {k: getattr(s, k) for k, _ in PlanStats._fields_}
+
+    def test_expect_arrivals(self, extra):
+        _check(lib().xgen_patconv_test_expect_arrivals(self._h, int(extra)), "xgen_patconv_test_expect_arrivals")
 
     def run(self, x_ptr, n, h, w, bias_ptr, relu, y_ptr, stream=0):
         """Enqueue the layer; all pointers are device addresses (ints)."""

@@ -3,7 +3,8 @@
 // Compact FKW Storage").  Pure C++, no CUDA.
 //
 // Layout idea.  A warp owns one *filter group* (J consecutive output channels) for a
-// tile of output pixels; each thread keeps J x 8 running sums (in tensor memory).  For every
+// tile of output pixels; each thread keeps J x T running sums in tensor memory (T = 16
+// output pixels per thread at stride 1, 8 at stride 2).  For every
 // input channel the group is connected to, the warp loads the activation patch
 // of its pixels once into registers (a LOAD command) and then executes one
 // *kernel command* per surviving kernel of that channel: the command names the
@@ -167,8 +168,9 @@ xgen_status build_layout(PackedHost &out, const PackConfig &cfg) {
     // channels (so a thread can store a pixel's J results as one contiguous piece);
     // what is reordered is which groups share a thread block.  Groups are sorted by
     // (surviving kernels desc, pattern histogram, index) and taken wpc at a time: the
-    // warps of a block, which meet at a barrier once per channel chunk, then carry
-    // similar numbers of kernels.
+    // warps of a block, which share the staged chunks of the input tile (a fast warp can
+    // run ahead only by the number of pipeline stages), then carry similar numbers of
+    // kernels.
     const int n_runs = (cout + J - 1) / J;
     std::vector<int> cnt(n_runs, 0);
     std::vector<std::vector<int>> hist(n_runs, std::vector<int>(np, 0));
@@ -246,7 +248,9 @@ xgen_status build_layout(PackedHost &out, const PackConfig &cfg) {
     s.macs_per_pixel = 4 * k_surv;
     const int wbytes = out.dtype == XGEN_F32 ? 4 : (out.dtype == XGEN_F16_F32ACC ? 2 : 1);
     s.weight_bytes = 4 * k_surv * wbytes;
-    s.index_bytes = n_slots * 2 + (int64_t)out.seg_off.size() * 4 + (int64_t)out.slot_oc.size() * 4;
+    const int64_t table_bytes = (int64_t)out.seg_off.size() * 4 + (int64_t)out.slot_oc.size() * 4;
+    s.compact_index_bytes = n_slots * 2 + table_bytes;
+    s.index_bytes = n_slots * kDevSlotBytes + table_bytes - s.weight_bytes;
     s.csr_index_bytes = 4 * k_surv * 4 + (int64_t)(cout + 1) * 4;
     s.stream_bytes = n_slots * kDevSlotBytes;
     s.filters_per_group = J; s.groups_per_block = wpc; s.n_blocks = n_blocks;

@@ -91,6 +91,7 @@ struct KParams {
     uint32_t *counters;
     uint32_t target;                     // counter value at which every split of an item has arrived
     int n_splits;
+    uint32_t wait_us;                    // bound of every device-side wait, microseconds
 };
 
 // ---- small PTX wrappers -----------------------------------------------------
@@ -123,17 +124,31 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t mbar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");
 }
 
-// Wait for an mbarrier phase with a bound: on expiry the block-wide abort flag and the
-// device status word are set and every later wait returns at once; the warps then leave
-// their loops, so the kernel still runs to its end (releasing tensor memory) with
-// results the host can tell are invalid.
-__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, volatile int *abort_flag, int *status) {
-    for (int it = 0; it < 400000; ++it) {
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Wait for an mbarrier phase with a bound in time (limit_us microseconds, plus a cap on the
+// polls in case the timer stands still): on expiry the block-wide abort flag and the device
+// status word are set and every later wait returns at once; the warps then leave their
+// loops, so the kernel still runs to its end (releasing tensor memory) with results the
+// host can tell are invalid.
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, volatile int *abort_flag, int *status,
+                                          uint32_t limit_us) {
+    uint64_t t0 = 0;
+    for (uint32_t it = 0; it < 40000000u; ++it) {
         uint32_t ok;
         asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
                      : "=r"(ok) : "r"(mbar), "r"(parity), "r"(2000u) : "memory");
         if (ok) return true;
         if (*abort_flag) return false;
+        if ((it & 7u) == 7u) {
+            const uint64_t t = global_ns();
+            if (t0 == 0) t0 = t;
+            else if (t - t0 > (uint64_t)limit_us * 1000ull) break;
+        }
     }
     *abort_flag = 1;
     if (status) atomicExch(status, 1);
@@ -394,7 +409,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
 
     if (producer) {
         // ===== producer warps: fill stage after stage; warp 0 also drives the copy engine =====
-        if (!P.use_tma) asm volatile("griddepcontrol.wait;" ::: "memory");   // they read x themselves
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // they read x themselves, or wait (with a bound) for its copies
         const int ptid = pw * 32 + lane;
         // Offsets of the next chunk's commands (the consumer warps' copy in shared memory may not
         // be written yet), fetched one chunk ahead by the thread that hands them to the copy engine.
@@ -404,7 +419,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         // chunk k uses stage s = k mod NS in its round ph = (k / NS) mod 2
         for (int c = c_begin, s = 0, ph = 0; c < c_end; ++c, s = (s + 1 == NS ? 0 : s + 1), ph ^= (s == 0)) {
             const int k = c - c_begin;
-            if (k >= NS && !mbar_wait(bar_empty(s), (uint32_t)(ph ^ 1), &abort_s, P.status)) break;
+            if (k >= NS && !mbar_wait(bar_empty(s), (uint32_t)(ph ^ 1), &abort_s, P.status, P.wait_us)) break;
             if (cmd_thread && k >= NS) {              // the first NS chunks' commands are on their way already
                 issue_commands(s, cmd_s0, cmd_s1);
                 if (c + 1 < c_end) { cmd_s0 = __ldg(seg_g + (k + 1) * (P.wpc + 1)); cmd_s1 = __ldg(seg_g + (k + 1) * (P.wpc + 1) + P.wpc); }
@@ -414,7 +429,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                 const int q = div_by(c, P.mg_spb), sub = c - q * spb;
                 const int r = (q - q0) % kRawStages;
                 if ((k == 0 || sub == 0) &&
-                    !mbar_wait(bar_raw(r), (uint32_t)(((q - q0) / kRawStages) & 1), &abort_s, P.status)) break;
+                    !mbar_wait(bar_raw(r), (uint32_t)(((q - q0) / kRawStages) & 1), &abort_s, P.status, P.wait_us)) break;
                 // the copy engine delivered [pixel][channel]; spread this chunk's channels into the
                 // fp32 operand planes
                 const int len = P.cc * XB, pix_bytes = P.rc * XB;          // bytes per pixel: chunk, box
@@ -461,7 +476,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                     // the box is refilled once every producer warp has read its share of it
                     if (lane == 0) mbar_arrive(bar_rawfree(r));
                     if (pw == 0) {
-                        if (!mbar_wait(bar_rawfree(r), (uint32_t)(((q - q0) / kRawStages) & 1), &abort_s, P.status)) break;
+                        if (!mbar_wait(bar_rawfree(r), (uint32_t)(((q - q0) / kRawStages) & 1), &abort_s, P.status, P.wait_us)) break;
                         if (lane == 0) {
                             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // reads of the box before its reuse
                             issue_box(q + kRawStages);
@@ -522,12 +537,15 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         const uint32_t thr_off = (uint32_t)(l_n * P.img_stride + l_y * BH * STRIDE * P.pitch + l_x * 4) * 4u;
         const uint32_t half_bytes = (uint32_t)P.half_stride * 4u;
 
+        // The first bounded wait below must not start counting while an earlier kernel of the
+        // stream still runs (the copies it waits for are issued only after that kernel).
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         // --- main loop over channel chunks --------------------------------------------
         for (int c = c_begin, s = 0, ph = 0; c < c_end; ++c, s = (s + 1 == NS ? 0 : s + 1), ph ^= (s == 0)) {
             const int k = c - c_begin;
             const uint32_t par = (uint32_t)ph;
-            if (!mbar_wait(bar_full(s), par, &abort_s, P.status)) break;
-            if (!mbar_wait(bar_cmd(s), par, &abort_s, P.status)) break;
+            if (!mbar_wait(bar_full(s), par, &abort_s, P.status, P.wait_us)) break;
+            if (!mbar_wait(bar_cmd(s), par, &abort_s, P.status, P.wait_us)) break;
             const int s0 = seg[k * (P.wpc + 1)], sg = seg[k * (P.wpc + 1) + warp];
             const uint32_t sp = smem_base + (uint32_t)(P.cmd_off_words + s * P.cmd_stage_words) * 4u +
                                 (uint32_t)(sg - s0) * (kDevSlotWords * 4u);
@@ -598,11 +616,17 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
             uint32_t *cnt = P.counters + item;
             asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(cnt) : "memory");
             bool ok = false;
-            for (int it = 0; it < 2000000 && !abort_s; ++it) {
+            uint64_t t0 = 0;
+            for (uint32_t it = 0; it < 40000000u && !abort_s; ++it) {
                 uint32_t v;
                 asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(cnt) : "memory");
                 if ((int)(v - P.target) >= 0) { ok = true; break; }
                 __nanosleep(100);
+                if ((it & 15u) == 15u) {
+                    const uint64_t t = global_ns();
+                    if (t0 == 0) t0 = t;
+                    else if (t - t0 > (uint64_t)P.wait_us * 1000ull) break;
+                }
             }
             if (!ok) { abort_s = 1; if (P.status) atomicExch(P.status, 1); }
         }
@@ -708,6 +732,12 @@ patconv_reduce_kernel(const uint32_t *__restrict__ partial, int splits, size_t o
 // ---- host side ----------------------------------------------------------------------
 static std::atomic<int64_t> g_launches{0};
 
+// The one environment switch, read once when the library is first used.
+static bool log_enabled() {
+    static const bool on = getenv("XGEN_PATCONV_LOG") != nullptr;
+    return on;
+}
+
 static inline int pixels_per_thread_x(int stride) { return stride == 1 ? 4 : 2; }
 static inline int pixels_per_thread(int stride) { return 4 * pixels_per_thread_x(stride); }
 
@@ -773,6 +803,28 @@ static Geometry choose_geometry(int n, int ho, int wo, int stride) {
     return best;
 }
 
+// Everything about a launch that depends only on the layer and the input shape: tile
+// geometry, shared-memory layout, tensor-memory columns.
+struct Layout {
+    Geometry g;
+    KParams kp;          // pointers, split and tensor-map fields left empty
+    size_t smem;
+    int items;           // (tile, filter block) pairs = blocks of an unsplit launch
+};
+
+// One prepared launch of a handle: the layout of a shape and the tensor map of an input
+// address.  xgen_patconv_run looks its shape up here instead of redoing the geometry search
+// and the tensor-map encoding on every call.
+struct LaunchEntry {
+    int n = 0, h = 0, w = 0;
+    const void *x = nullptr;
+    bool y32 = false;
+    Layout L;
+    CUtensorMap tm;
+    uint64_t stamp = 0;
+};
+constexpr int kLaunchCache = 4;
+
 }  // namespace patconv
 
 using namespace patconv;
@@ -789,8 +841,16 @@ struct xgen_patconv_packed {
     size_t partial_bytes = 0;
     uint32_t *d_counters = nullptr;     // one arrival counter per (tile, filter block) of the planned shape
     size_t counter_bytes = 0;
-    mutable std::atomic<uint32_t> split_seq{0};   // planned split launches so far (counters only grow)
+    mutable std::mutex split_mu;        // orders the launches of planned splits (the counters only grow)
+    mutable uint32_t split_seq = 0;     // planned split launches enqueued so far
     int *d_status = nullptr;            // set by a kernel whose bounded wait ran out
+    xgen_patconv_tuning tuning{};       // caller's overrides (xgen_patconv_plan_tuned)
+    uint32_t wait_us = 2000000;         // bound of every device-side wait
+    int hook_extra_arrivals = 0;        // testing aid: arrivals a planned split waits for beyond its own
+    // prepared launches (shape, input address)
+    mutable std::mutex cache_mu;
+    mutable LaunchEntry cache[kLaunchCache];
+    mutable uint64_t cache_stamp = 0;
     // device staging buffers of xgen_patconv_run_host, kept between calls (grow only)
     mutable std::mutex host_mu;
     mutable void *d_hx = nullptr, *d_hy = nullptr, *d_hb = nullptr;
@@ -843,7 +903,7 @@ static xgen_status upload_layout(xgen_patconv_packed *h) {
 
 // With XGEN_PATCONV_LOG set, failed CUDA calls are named on stderr.
 static cudaError_t log_cuda(cudaError_t e, const char *what) {
-    if (e != cudaSuccess && getenv("XGEN_PATCONV_LOG"))
+    if (e != cudaSuccess && log_enabled())
         fprintf(stderr, "libpatconv: %s: %s\n", what, cudaGetErrorString(e));
     return e;
 }
@@ -854,11 +914,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 static EncodeTiledFn encode_tiled_fn() {
     static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    static std::mutex m;
-    std::lock_guard<std::mutex> lock(m);
-    if (!tried) {
-        tried = true;
+    static std::once_flag once;
+    std::call_once(once, [] {
         void *ptr = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
@@ -866,7 +923,7 @@ static EncodeTiledFn encode_tiled_fn() {
             fn = (EncodeTiledFn)ptr;
         else
             cudaGetLastError();
-    }
+    });
     return fn;
 }
 
@@ -904,6 +961,253 @@ static cudaError_t allow_large_smem(const void *kern) {
 
 static int next_pow2(int v) { int p = 32; while (p < v) p <<= 1; return p; }
 
+static xgen_status make_layout(const PackedHost &p, int n, int hh, int ww, bool y_aligned32, bool tma_ok, Layout &L) {
+    const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
+    const Geometry g = choose_geometry(n, ho, wo, p.stride);
+    L.g = g;
+    KParams kp{};
+    kp.n = n; kp.h = hh; kp.w = ww; kp.ho = ho; kp.wo = wo; kp.c_in = p.c_in; kp.c_out = p.c_out;
+    kp.J = p.J; kp.wpc = p.wpc; kp.cc = p.cc; kp.n_chunks = p.n_chunks;
+    kp.lx_log = g.lx_log; kp.ly_log = g.ly_log; kp.ln_log = g.ln_log;
+    kp.tiles_x = g.tiles_x; kp.tiles_y = g.tiles_y;
+    kp.tin_w = g.tin_w; kp.tin_h = g.tin_h;
+    kp.pitch = g.pitch; kp.img_stride = g.img_stride; kp.plane_stride = g.plane_stride;
+    kp.half_stride = g.half_stride;
+    const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
+    const int npix_box = (g.tin_w * g.tin_h) << g.ln_log;
+    // A box carries at least 16 bytes of channels per pixel; a chunk may be a part of it.
+    // The copy engine needs 16-byte multiples in every global stride.
+    kp.rc = p.cc * xb >= 16 ? p.cc : 16 / xb;
+    kp.spb = kp.rc / p.cc;
+    auto magic = [](int d) { return d <= 1 ? 0u : (uint32_t)((1ull << 32) / (uint64_t)d + 1ull); };
+    kp.mg_tiles_x = magic(g.tiles_x); kp.mg_tiles_y = magic(g.tiles_y);
+    kp.mg_tin_w = magic(g.tin_w); kp.mg_tin_h = magic(g.tin_h); kp.mg_spb = magic(kp.spb);
+    kp.use_tma = tma_ok && ((p.cc * xb) % 4 == 0) && (((size_t)p.c_in * xb) % 16 == 0) && g.tin_w <= 256 && g.tin_h <= 256;
+    kp.box_bytes = npix_box * kp.rc * xb;
+    // widest aligned store per 8-channel piece: 8 words (32-byte aligned rows), 4, or scalar
+    kp.vec_out = ((p.c_out % 8) == 0 && y_aligned32) ? 8 : ((p.c_out % 4) == 0 ? 4 : 0);
+    const bool is_i8 = p.dtype == XGEN_I8_I32;
+    const int T = pixels_per_thread(p.stride);
+    kp.flush_chunks = 16777216 / (p.cc * 4 * 32640);
+    if (kp.flush_chunks < 1) return XGEN_ERR_UNSUPPORTED;
+    kp.fold = (is_i8 && p.n_chunks > kp.flush_chunks) ? 1 : 0;
+    kp.cols_per_warp = p.J * T * (kp.fold ? 2 : 1);
+    kp.tmem_cols = next_pow2(((p.wpc + 3) / 4) * kp.cols_per_warp);
+    if (kp.tmem_cols > 512) return XGEN_ERR_UNSUPPORTED;
+    // Shared-memory layout (words): raw boxes | plane stages | command stages | tables | barriers.
+    kp.cmd_stage_words = ((p.max_seg_slots + 2) * kDevSlotWords + 31) & ~31;
+    kp.plane_stage_words = (p.cc * g.plane_stride + 31) & ~31;
+    const int max_ctas = 512 / kp.tmem_cols;          // blocks per SM that tensor memory has columns for
+    const size_t seg_words = ((size_t)p.n_chunks * (p.wpc + 1) + 1) & ~(size_t)1;
+    auto smem_words = [&](int stages, int tma) {
+        size_t w = (size_t)(tma ? kRawStages * ((kp.box_bytes / 4 + 31) & ~31) : 0);
+        w += (size_t)stages * (kp.plane_stage_words + kp.cmd_stage_words);
+        w += 2 * (size_t)npix_box + (tma ? 0 : ((size_t)npix_box + 1) & ~(size_t)1) + 32 * (size_t)T + seg_words;
+        return w + 2 * (3 * kMaxStages + 2 * kRawStages + 2);     // + mbarriers
+    };
+    auto occupancy = [&](size_t words) {
+        int o = (int)((size_t)kSmemPerSM / (words * 4 + 2112));     // + static and per-block reserved shared memory
+        return o < max_ctas ? o : max_ctas;
+    };
+    if (kp.use_tma && smem_words(2, 1) * 4 > (size_t)kSmemMaxDynamic) kp.use_tma = 0;   // the raw boxes do not fit
+    // Stage count: as many as fit (up to 4) without lowering the number of blocks per SM.
+    int n_stages = 2;
+    for (int st = 3; st <= kMaxStages; ++st)
+        if (smem_words(st, kp.use_tma) * 4 <= (size_t)kSmemMaxDynamic &&
+            occupancy(smem_words(st, kp.use_tma)) >= occupancy(smem_words(2, kp.use_tma))) n_stages = st;
+    kp.n_stages = n_stages;
+    kp.raw_stage_words = kp.use_tma ? ((kp.box_bytes / 4 + 31) & ~31) : 0;
+    kp.raw_off_words = 0;
+    kp.plane_off_words = kp.use_tma ? kRawStages * kp.raw_stage_words : 0;
+    kp.cmd_off_words = kp.plane_off_words + n_stages * kp.plane_stage_words;
+    kp.tab_off_words = kp.cmd_off_words + n_stages * kp.cmd_stage_words;
+    kp.src_off_words = kp.tab_off_words + 2 * npix_box;
+    kp.ptab_off_words = kp.src_off_words + (kp.use_tma ? 0 : ((npix_box + 1) & ~1));
+    kp.seg_off_words = kp.ptab_off_words + 32 * T;
+    kp.mbar_off_words = kp.seg_off_words + (int)seg_words;
+    size_t smem = smem_words(n_stages, kp.use_tma) * 4;
+    // Never let more blocks share an SM than tensor memory has columns for.
+    const size_t floor_bytes = (size_t)kSmemPerSM / (max_ctas + 1);
+    if (smem < floor_bytes) smem = floor_bytes;
+    if (smem > (size_t)kSmemMaxDynamic) return XGEN_ERR_UNSUPPORTED;
+    kp.out_elems = (size_t)n * ho * wo * p.c_out;
+    L.kp = kp;
+    L.smem = smem;
+    L.items = g.tiles_x * g.tiles_y * g.tiles_n * p.n_blocks;
+    return XGEN_OK;
+}
+
+// 1 KB rows of partial sums one (item, split) writes in a split run reduced inside the kernel.
+static size_t rows_per_item(const PackedHost &p) {
+    return (size_t)p.wpc * ((p.J + 7) / 8) * pixels_per_thread(p.stride);
+}
+
+// The prepared launch of (shape, input address, alignment class of y): from the handle's
+// small cache, or built now (geometry, shared-memory layout, tensor map) and kept.
+static xgen_status prepared_launch(const xgen_patconv_packed *h, const void *x, int n, int hh, int ww, bool y32,
+                                   Layout &L, CUtensorMap &tm) {
+    std::lock_guard<std::mutex> lock(h->cache_mu);
+    LaunchEntry *victim = &h->cache[0];
+    for (LaunchEntry &e : h->cache) {
+        if (e.stamp && e.n == n && e.h == hh && e.w == ww && e.x == x && e.y32 == y32) {
+            e.stamp = ++h->cache_stamp;
+            L = e.L; tm = e.tm;
+            return XGEN_OK;
+        }
+        if (e.stamp < victim->stamp) victim = &e;
+    }
+    const PackedHost &p = h->host;
+    EncodeTiledFn encode = h->tuning.no_copy_engine ? nullptr : encode_tiled_fn();
+    LaunchEntry ne;
+    xgen_status ls = make_layout(p, n, hh, ww, y32, encode != nullptr, ne.L);
+    if (ls != XGEN_OK) return ls;
+    memset(&ne.tm, 0, sizeof(ne.tm));
+    if (ne.L.kp.use_tma) {
+        const Geometry &g = ne.L.g;
+        const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
+        const cuuint64_t gdim[4] = {(cuuint64_t)p.c_in, (cuuint64_t)ww, (cuuint64_t)hh, (cuuint64_t)n};
+        const cuuint64_t gstr[3] = {(cuuint64_t)p.c_in * xb, (cuuint64_t)ww * p.c_in * xb, (cuuint64_t)hh * ww * p.c_in * xb};
+        const cuuint32_t box[4] = {(cuuint32_t)ne.L.kp.rc, (cuuint32_t)g.tin_w, (cuuint32_t)g.tin_h, (cuuint32_t)(1 << g.ln_log)};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        const CUtensorMapDataType dt = p.dtype == XGEN_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                     : (p.dtype == XGEN_F16_F32ACC ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
+        const CUresult cr = encode(&ne.tm, dt, 4, const_cast<void *>(x), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                   CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (cr != CUDA_SUCCESS) {          // stage with plain loads instead
+            if (log_enabled()) fprintf(stderr, "libpatconv: cuTensorMapEncodeTiled failed (%d)\n", (int)cr);
+            memset(&ne.tm, 0, sizeof(ne.tm));
+            ls = make_layout(p, n, hh, ww, y32, false, ne.L);
+            if (ls != XGEN_OK) return ls;
+        }
+    }
+    ne.n = n; ne.h = hh; ne.w = ww; ne.x = x; ne.y32 = y32;
+    ne.stamp = ++h->cache_stamp;
+    *victim = ne;
+    L = ne.L; tm = ne.tm;
+    return XGEN_OK;
+}
+
+static void forget_prepared_launches(xgen_patconv_packed *h) {
+    std::lock_guard<std::mutex> lock(h->cache_mu);
+    for (LaunchEntry &e : h->cache) e.stamp = 0;
+}
+
+// Where a run keeps the partial sums of a split, when the caller (not the plan) decides.
+struct SplitChoice { int splits, chunks_per_split; uint32_t *partial; };
+
+static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
+                             const void *bias, int32_t relu, void *y, void *stream, const SplitChoice *forced) {
+    if (!h || !x || !y) return XGEN_ERR_INVALID_ARG;
+    if (((uintptr_t)x & 15) || ((uintptr_t)y & 15) || ((uintptr_t)bias & 3)) return XGEN_ERR_INVALID_ARG;
+    if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
+    const PackedHost &p = h->host;
+    if (h->device < 0) return XGEN_ERR_CUDA;
+    const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
+    if ((int64_t)n * hh * ww * p.c_in > 0x7FFFFFFFLL || (int64_t)n * ho * wo * p.c_out > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
+    const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
+    {
+        const char *xa = (const char *)x, *ya = (const char *)y;
+        const int yb = p.dtype == XGEN_F16_F32ACC ? 2 : 4;
+        const char *xe = xa + (size_t)n * hh * ww * p.c_in * xb, *ye = ya + (size_t)n * ho * wo * p.c_out * yb;
+        if (xa < ye && ya < xe) return XGEN_ERR_INVALID_ARG;   // overlap
+    }
+    Layout L;
+    CUtensorMap tm;
+    xgen_status ls = prepared_launch(h, x, n, hh, ww, ((uintptr_t)y & 31) == 0, L, tm);
+    if (ls != XGEN_OK) return ls;
+    KParams kp = L.kp;
+    const size_t smem = L.smem;
+    kp.x = x; kp.y = y; kp.bias = bias;
+    kp.slots = h->d_slots; kp.seg_off = h->d_seg_off; kp.slot_oc = h->d_slot_oc;
+    kp.relu = relu ? 1 : 0;
+    kp.status = h->d_status;
+    kp.wait_us = h->wait_us;
+    // Split runs: a caller-chosen split keeps [split][output] sums for a second kernel; the
+    // planned split is reduced inside the kernel (rows of partial sums plus arrival counters).
+    const bool planned = !forced && h->plan_splits > 1 && h->plan_n == n && h->plan_h == hh && h->plan_w == ww &&
+                         h->d_partial && h->d_counters;
+    const bool split = forced ? forced->splits > 1 : planned;
+    const int n_splits = forced ? forced->splits : h->plan_splits;
+    kp.chunks_per_split = split ? (forced ? forced->chunks_per_split : h->plan_cps) : 0;
+    kp.partial = (split && forced) ? forced->partial : nullptr;
+    kp.n_splits = split ? n_splits : 1;
+
+    int prev = 0;
+    if (cudaGetDevice(&prev) != cudaSuccess) return XGEN_ERR_CUDA;
+    if (prev != h->device && cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
+    dim3 grid((unsigned)(L.g.tiles_x * L.g.tiles_y * L.g.tiles_n), (unsigned)p.n_blocks, (unsigned)(split ? n_splits : 1)), block((unsigned)((p.wpc + kProducerWarps) * 32), 1, 1);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (log_enabled())
+        fprintf(stderr, "libpatconv: grid %u x %u x %u, %u threads, %zu bytes shared, %d stages, lanes %dx%dx%d, tile in %dx%d, tma %d, cc %d, fused split %d\n",
+                grid.x, grid.y, grid.z, block.x, smem, kp.n_stages, 1 << L.g.lx_log, 1 << L.g.ly_log, 1 << L.g.ln_log,
+                L.g.tin_w, L.g.tin_h, kp.use_tma, p.cc, planned ? 1 : 0);
+    const void *kern = kernel_for(p);
+    cudaError_t e = allow_large_smem(kern);
+    if (e == cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        // Programmatic stream serialisation: this kernel may be scheduled while its predecessor
+        // in the stream drains (it waits for it, griddepcontrol.wait, before touching memory), and
+        // it lets its successor do the same.  A dependent grid starts only after every block of
+        // this one has started, so the blocks of a split, which wait for each other and which the
+        // planner keeps within what the GPU holds at once, are never kept out by a successor.
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = h->tuning.no_launch_overlap ? 0 : 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        void *args[2] = {(void *)&kp, (void *)&tm};
+        if (planned) {
+            // The arrival counters of a planned split only grow: launch k waits for k x splits
+            // arrivals.  The sequence number moves on only when the launch was accepted.
+            std::lock_guard<std::mutex> lock(h->split_mu);
+            kp.ws = h->d_partial;
+            kp.counters = h->d_counters;
+            kp.target = (h->split_seq + 1u) * (uint32_t)n_splits + (uint32_t)h->hook_extra_arrivals;
+            e = cudaLaunchKernelExC(&cfg, kern, args);
+            if (e == cudaSuccess) e = cudaGetLastError();
+            if (e == cudaSuccess) ++h->split_seq;
+        } else {
+            e = cudaLaunchKernelExC(&cfg, kern, args);
+            if (e == cudaSuccess) e = cudaGetLastError();
+        }
+        e = log_cuda(e, "kernel launch");
+    }
+    if (e == cudaSuccess && split && forced) {
+        const int vec = kp.vec_out >= 4 ? 1 : 0;
+        const size_t items = vec ? kp.out_elems / 4 : kp.out_elems;
+        const unsigned blocks = (unsigned)((items + 255) / 256);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(blocks, 1, 1); cfg.blockDim = dim3(256, 1, 1); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        const uint32_t *part_c = forced->partial;
+        const size_t oe = kp.out_elems;
+        const int co = p.c_out, rl = kp.relu;
+        const void *bias_c = bias;
+        if (p.dtype == XGEN_F32)
+            e = cudaLaunchKernelEx(&cfg, patconv_reduce_kernel<XGEN_F32>, part_c, n_splits, oe, co, bias_c, rl, y, vec);
+        else if (p.dtype == XGEN_F16_F32ACC)
+            e = cudaLaunchKernelEx(&cfg, patconv_reduce_kernel<XGEN_F16_F32ACC>, part_c, n_splits, oe, co, bias_c, rl, y, vec);
+        else
+            e = cudaLaunchKernelEx(&cfg, patconv_reduce_kernel<XGEN_I8_I32>, part_c, n_splits, oe, co, bias_c, rl, y, vec);
+        if (e == cudaSuccess) e = cudaGetLastError();
+        e = log_cuda(e, "reduce launch");
+        if (e == cudaSuccess) g_launches.fetch_add(1);
+    }
+    if (prev != h->device) cudaSetDevice(prev);
+    if (e != cudaSuccess) return XGEN_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return XGEN_OK;
+}
+
+// The library's own scratch for xgen_patconv_run_static_scratch: partial sums of a split run.
+// It lives in every CUDA context that loads this library, until the process exits.
+static __device__ __align__(256) uint32_t g_static_scratch[XGEN_PATCONV_STATIC_SCRATCH_BYTES / 4];
+static uint32_t *g_static_scratch_addr[64];        // device address per device ordinal, resolved once
+static std::mutex g_static_scratch_mutex;
+
 extern "C" {
 
 const char *xgen_strerror(xgen_status s) {
@@ -931,18 +1235,11 @@ xgen_status xgen_patconv_pack(const xgen_patconv_desc *desc, const void *dense_w
     xgen_status st;
     try {
         PackConfig cfg = choose_pack_config(desc->c_in, desc->c_out, desc->dtype, desc->stride);
-        // a group is stored in pieces of 8 adjacent channels (32-byte stores): whole pieces only
-        if (const char *e = getenv("XGEN_PATCONV_J")) { int v = atoi(e); if (v == 8 || v == 16) {
-            cfg.filters_per_group = v;
-            int groups = (desc->c_out + v - 1) / v; cfg.groups_per_block = groups < kMaxWarps ? groups : kMaxWarps; } }
-        if (const char *e = getenv("XGEN_PATCONV_WPC")) { int v = atoi(e); if (v >= 1 && v <= kMaxWarps) {
-            int groups = (desc->c_out + cfg.filters_per_group - 1) / cfg.filters_per_group; cfg.groups_per_block = groups < v ? groups : v; } }
-        if (const char *e = getenv("XGEN_PATCONV_CC")) { int v = atoi(e); if (v == 2 || v == 4 || v == 8 || v == 16) cfg.channels_per_chunk = v; }
         if (desc->dtype == XGEN_I8_I32 && cfg.channels_per_chunk < 4) cfg.channels_per_chunk = 4;
         st = pack_host(*desc, dense_w_host, pattern_id_host, cfg, h->host);
         // A stage of the kernel's pipeline holds the commands of one chunk for the whole
         // block: halve the chunk until the longest segment fits the command buffer.
-        while (st == XGEN_OK && !getenv("XGEN_PATCONV_CC") && cfg.channels_per_chunk > 4 &&
+        while (st == XGEN_OK && cfg.channels_per_chunk > 4 &&
                (size_t)h->host.max_seg_slots * kDevSlotBytes > kCmdStageBudget) {
             cfg.channels_per_chunk /= 2;
             st = build_layout(h->host, cfg);
@@ -1010,253 +1307,61 @@ xgen_status xgen_patconv_last_status(const xgen_patconv_packed *h, void *stream)
     if (h->s_out && cudaStreamSynchronize(h->s_out) != cudaSuccess) return XGEN_ERR_CUDA;   // copies out of host-buffer calls
     if (cudaGetLastError() != cudaSuccess) return XGEN_ERR_CUDA;
     if (h->d_status) {
-        // a kernel whose bounded wait for a tile copy ran out leaves a mark here
+        // a kernel whose bounded wait ran out leaves a mark here
         int flag = 0;
         if (cudaMemcpy(&flag, h->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return XGEN_ERR_CUDA;
         if (flag) {
             cudaMemset(h->d_status, 0, sizeof(int));
             // a run that gave up may have left the arrival counters of a split half way
+            std::lock_guard<std::mutex> lock(h->split_mu);
             if (h->d_counters) cudaMemset(h->d_counters, 0, h->counter_bytes);
-            h->split_seq.store(0);
+            h->split_seq = 0;
             return XGEN_ERR_TIMEOUT;
         }
     }
     return XGEN_OK;
 }
 
-}  // extern "C"
-
-// Everything about a launch that depends only on the layer and the input shape: tile
-// geometry, shared-memory layout, tensor-memory columns.
-struct Layout {
-    Geometry g;
-    KParams kp;          // pointers, split and tensor-map fields left empty
-    size_t smem;
-    int items;           // (tile, filter block) pairs = blocks of an unsplit launch
-};
-
-static xgen_status make_layout(const PackedHost &p, int n, int hh, int ww, bool y_aligned32, bool tma_ok, Layout &L) {
-    const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
-    const Geometry g = choose_geometry(n, ho, wo, p.stride);
-    L.g = g;
-    KParams kp{};
-    kp.n = n; kp.h = hh; kp.w = ww; kp.ho = ho; kp.wo = wo; kp.c_in = p.c_in; kp.c_out = p.c_out;
-    kp.J = p.J; kp.wpc = p.wpc; kp.cc = p.cc; kp.n_chunks = p.n_chunks;
-    kp.lx_log = g.lx_log; kp.ly_log = g.ly_log; kp.ln_log = g.ln_log;
-    kp.tiles_x = g.tiles_x; kp.tiles_y = g.tiles_y;
-    kp.tin_w = g.tin_w; kp.tin_h = g.tin_h;
-    kp.pitch = g.pitch; kp.img_stride = g.img_stride; kp.plane_stride = g.plane_stride;
-    kp.half_stride = g.half_stride;
-    const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
-    const int npix_box = (g.tin_w * g.tin_h) << g.ln_log;
-    // A box carries at least 16 bytes of channels per pixel; a chunk may be a part of it.
-    // The copy engine needs 16-byte multiples in every global stride.
-    kp.rc = p.cc * xb >= 16 ? p.cc : 16 / xb;
-    kp.spb = kp.rc / p.cc;
-    auto magic = [](int d) { return d <= 1 ? 0u : (uint32_t)((1ull << 32) / (uint64_t)d + 1ull); };
-    kp.mg_tiles_x = magic(g.tiles_x); kp.mg_tiles_y = magic(g.tiles_y);
-    kp.mg_tin_w = magic(g.tin_w); kp.mg_tin_h = magic(g.tin_h); kp.mg_spb = magic(kp.spb);
-    kp.use_tma = tma_ok && ((p.cc * xb) % 4 == 0) && (((size_t)p.c_in * xb) % 16 == 0) && g.tin_w <= 256 && g.tin_h <= 256 &&
-                 !getenv("XGEN_PATCONV_NO_TMA");
-    kp.box_bytes = npix_box * kp.rc * xb;
-    // widest aligned store per 8-channel piece: 8 words (32-byte aligned rows), 4, or scalar
-    kp.vec_out = ((p.c_out % 8) == 0 && y_aligned32) ? 8 : ((p.c_out % 4) == 0 ? 4 : 0);
-    const bool is_i8 = p.dtype == XGEN_I8_I32;
-    const int T = pixels_per_thread(p.stride);
-    kp.flush_chunks = 16777216 / (p.cc * 4 * 32640);
-    if (kp.flush_chunks < 1) return XGEN_ERR_UNSUPPORTED;
-    kp.fold = (is_i8 && p.n_chunks > kp.flush_chunks) ? 1 : 0;
-    kp.cols_per_warp = p.J * T * (kp.fold ? 2 : 1);
-    kp.tmem_cols = next_pow2(((p.wpc + 3) / 4) * kp.cols_per_warp);
-    if (kp.tmem_cols > 512) return XGEN_ERR_UNSUPPORTED;
-    // Shared-memory layout (words): raw boxes | plane stages | command stages | tables | barriers.
-    kp.cmd_stage_words = ((p.max_seg_slots + 2) * kDevSlotWords + 31) & ~31;
-    kp.plane_stage_words = (p.cc * g.plane_stride + 31) & ~31;
-    const int max_ctas = 512 / kp.tmem_cols;          // blocks per SM that tensor memory has columns for
-    const size_t seg_words = ((size_t)p.n_chunks * (p.wpc + 1) + 1) & ~(size_t)1;
-    auto smem_words = [&](int stages, int tma) {
-        size_t w = (size_t)(tma ? kRawStages * ((kp.box_bytes / 4 + 31) & ~31) : 0);
-        w += (size_t)stages * (kp.plane_stage_words + kp.cmd_stage_words);
-        w += 2 * (size_t)npix_box + (tma ? 0 : ((size_t)npix_box + 1) & ~(size_t)1) + 32 * (size_t)T + seg_words;
-        return w + 2 * (3 * kMaxStages + 2 * kRawStages + 2);     // + mbarriers
-    };
-    auto occupancy = [&](size_t words) {
-        int o = (int)((size_t)kSmemPerSM / (words * 4 + 2112));     // + static and per-block reserved shared memory
-        return o < max_ctas ? o : max_ctas;
-    };
-    if (kp.use_tma && smem_words(2, 1) * 4 > (size_t)kSmemMaxDynamic) kp.use_tma = 0;   // the raw boxes do not fit
-    // Stage count: as many as fit (up to 4) without lowering the number of blocks per SM.
-    int n_stages = 2;
-    for (int st = 3; st <= kMaxStages; ++st)
-        if (smem_words(st, kp.use_tma) * 4 <= (size_t)kSmemMaxDynamic &&
-            occupancy(smem_words(st, kp.use_tma)) >= occupancy(smem_words(2, kp.use_tma))) n_stages = st;
-    if (const char *e = getenv("XGEN_PATCONV_STAGES")) { int v = atoi(e); if (v >= 2 && v <= kMaxStages && smem_words(v, kp.use_tma) * 4 <= (size_t)kSmemMaxDynamic) n_stages = v; }
-    kp.n_stages = n_stages;
-    kp.raw_stage_words = kp.use_tma ? ((kp.box_bytes / 4 + 31) & ~31) : 0;
-    kp.raw_off_words = 0;
-    kp.plane_off_words = kp.use_tma ? kRawStages * kp.raw_stage_words : 0;
-    kp.cmd_off_words = kp.plane_off_words + n_stages * kp.plane_stage_words;
-    kp.tab_off_words = kp.cmd_off_words + n_stages * kp.cmd_stage_words;
-    kp.src_off_words = kp.tab_off_words + 2 * npix_box;
-    kp.ptab_off_words = kp.src_off_words + (kp.use_tma ? 0 : ((npix_box + 1) & ~1));
-    kp.seg_off_words = kp.ptab_off_words + 32 * T;
-    kp.mbar_off_words = kp.seg_off_words + (int)seg_words;
-    size_t smem = smem_words(n_stages, kp.use_tma) * 4;
-    // Never let more blocks share an SM than tensor memory has columns for.
-    const size_t floor_bytes = (size_t)kSmemPerSM / (max_ctas + 1);
-    if (smem < floor_bytes) smem = floor_bytes;
-    if (smem > (size_t)kSmemMaxDynamic) return XGEN_ERR_UNSUPPORTED;
-    kp.out_elems = (size_t)n * ho * wo * p.c_out;
-    L.kp = kp;
-    L.smem = smem;
-    L.items = g.tiles_x * g.tiles_y * g.tiles_n * p.n_blocks;
-    return XGEN_OK;
-}
-
-// 1 KB rows of partial sums one (item, split) writes in a split run reduced inside the kernel.
-static size_t rows_per_item(const PackedHost &p) {
-    return (size_t)p.wpc * ((p.J + 7) / 8) * pixels_per_thread(p.stride);
-}
-
-// Where a run keeps the partial sums of a split, when the caller (not the plan) decides.
-struct SplitChoice { int splits, chunks_per_split; uint32_t *partial; };
-
-static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
-                             const void *bias, int32_t relu, void *y, void *stream, const SplitChoice *forced) {
-    if (!h || !x || !y) return XGEN_ERR_INVALID_ARG;
-    if (((uintptr_t)x & 15) || ((uintptr_t)y & 15) || ((uintptr_t)bias & 15)) return XGEN_ERR_INVALID_ARG;
+// What a launch of this shape looks like with the handle as it stands.
+xgen_status xgen_patconv_plan_info(const xgen_patconv_packed *h, int32_t n, int32_t hh, int32_t ww,
+                                   xgen_patconv_plan_stats *out) {
+    if (!h || !out) return XGEN_ERR_INVALID_ARG;
     if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
     const PackedHost &p = h->host;
-    if (h->device < 0) return XGEN_ERR_CUDA;
-    const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
-    if ((int64_t)n * hh * ww * p.c_in > 0x7FFFFFFFLL || (int64_t)n * ho * wo * p.c_out > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
-    const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
-    {
-        const char *xa = (const char *)x, *ya = (const char *)y;
-        const int yb = p.dtype == XGEN_F16_F32ACC ? 2 : 4;
-        const char *xe = xa + (size_t)n * hh * ww * p.c_in * xb, *ye = ya + (size_t)n * ho * wo * p.c_out * yb;
-        if (xa < ye && ya < xe) return XGEN_ERR_INVALID_ARG;   // overlap
-    }
-    EncodeTiledFn encode = encode_tiled_fn();
     Layout L;
-    xgen_status ls = make_layout(p, n, hh, ww, ((uintptr_t)y & 31) == 0, encode != nullptr, L);
+    const bool tma_ok = !h->tuning.no_copy_engine && (h->device < 0 || encode_tiled_fn() != nullptr);
+    xgen_status ls = make_layout(p, n, hh, ww, true, tma_ok, L);
     if (ls != XGEN_OK) return ls;
-    CUtensorMap tm;
-    memset(&tm, 0, sizeof(tm));
-    if (L.kp.use_tma) {
-        const Geometry &g = L.g;
-        const cuuint64_t gdim[4] = {(cuuint64_t)p.c_in, (cuuint64_t)ww, (cuuint64_t)hh, (cuuint64_t)n};
-        const cuuint64_t gstr[3] = {(cuuint64_t)p.c_in * xb, (cuuint64_t)ww * p.c_in * xb, (cuuint64_t)hh * ww * p.c_in * xb};
-        const cuuint32_t box[4] = {(cuuint32_t)L.kp.rc, (cuuint32_t)g.tin_w, (cuuint32_t)g.tin_h, (cuuint32_t)(1 << g.ln_log)};
-        const cuuint32_t estr[4] = {1, 1, 1, 1};
-        const CUtensorMapDataType dt = p.dtype == XGEN_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
-                                     : (p.dtype == XGEN_F16_F32ACC ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
-        const CUresult cr = encode(&tm, dt, 4, const_cast<void *>(x), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                   CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (cr != CUDA_SUCCESS) {          // fall back to plain loads
-            if (getenv("XGEN_PATCONV_LOG")) fprintf(stderr, "libpatconv: cuTensorMapEncodeTiled failed (%d)\n", (int)cr);
-            memset(&tm, 0, sizeof(tm));
-            ls = make_layout(p, n, hh, ww, ((uintptr_t)y & 31) == 0, false, L);
-            if (ls != XGEN_OK) return ls;
-        }
-    }
-    KParams kp = L.kp;
-    const size_t smem = L.smem;
-    kp.x = x; kp.y = y; kp.bias = bias;
-    kp.slots = h->d_slots; kp.seg_off = h->d_seg_off; kp.slot_oc = h->d_slot_oc;
-    kp.relu = relu ? 1 : 0;
-    kp.status = h->d_status;
-    // Split runs: a caller-chosen split keeps [split][output] sums for a second kernel; the
-    // planned split is reduced inside the kernel (rows of partial sums plus arrival counters).
-    const bool planned = !forced && h->plan_splits > 1 && h->plan_n == n && h->plan_h == hh && h->plan_w == ww &&
-                         h->d_partial && h->d_counters;
-    const bool split = forced ? forced->splits > 1 : planned;
-    const int n_splits = forced ? forced->splits : h->plan_splits;
-    kp.chunks_per_split = split ? (forced ? forced->chunks_per_split : h->plan_cps) : 0;
-    kp.partial = (split && forced) ? forced->partial : nullptr;
-    kp.n_splits = split ? n_splits : 1;
-    if (planned) {
-        kp.ws = h->d_partial;
-        kp.counters = h->d_counters;
-        kp.target = (h->split_seq.fetch_add(1) + 1u) * (uint32_t)n_splits;
-    }
-
-    int prev = 0;
-    if (cudaGetDevice(&prev) != cudaSuccess) return XGEN_ERR_CUDA;
-    if (prev != h->device && cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
-    dim3 grid((unsigned)(L.g.tiles_x * L.g.tiles_y * L.g.tiles_n), (unsigned)p.n_blocks, (unsigned)(split ? n_splits : 1)), block((unsigned)((p.wpc + kProducerWarps) * 32), 1, 1);
-    cudaStream_t st = (cudaStream_t)stream;
-    if (getenv("XGEN_PATCONV_LOG"))
-        fprintf(stderr, "libpatconv: grid %u x %u x %u, %u threads, %zu bytes shared, %d stages, lanes %dx%dx%d, tile in %dx%d, tma %d, cc %d, fused split %d\n",
-                grid.x, grid.y, grid.z, block.x, smem, kp.n_stages, 1 << L.g.lx_log, 1 << L.g.ly_log, 1 << L.g.ln_log,
-                L.g.tin_w, L.g.tin_h, kp.use_tma, p.cc, planned ? 1 : 0);
-    const void *kern = kernel_for(p);
-    cudaError_t e = allow_large_smem(kern);
-    if (e == cudaSuccess) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
-        // Programmatic stream serialisation: this kernel may be scheduled while its predecessor
-        // in the stream drains (it waits for it, griddepcontrol.wait, before touching memory), and
-        // it lets its successor do the same.  A dependent grid starts only after every block of
-        // this one has started, so the blocks of a split, which wait for each other and which the
-        // planner keeps within what the GPU holds at once, are never kept out by a successor.
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = getenv("XGEN_PATCONV_NO_PDL") ? 0 : 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        void *args[2] = {(void *)&kp, (void *)&tm};
-        e = cudaLaunchKernelExC(&cfg, kern, args);
-        if (e == cudaSuccess) e = cudaGetLastError();
-        e = log_cuda(e, "kernel launch");
-    }
-    if (e == cudaSuccess && split && forced) {
-        const int vec = kp.vec_out >= 4 ? 1 : 0;
-        const size_t items = vec ? kp.out_elems / 4 : kp.out_elems;
-        const unsigned blocks = (unsigned)((items + 255) / 256);
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(blocks, 1, 1); cfg.blockDim = dim3(256, 1, 1); cfg.dynamicSmemBytes = 0; cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        const uint32_t *part_c = forced->partial;
-        const size_t oe = kp.out_elems;
-        const int co = p.c_out, rl = kp.relu;
-        const void *bias_c = bias;
-        if (p.dtype == XGEN_F32)
-            e = cudaLaunchKernelEx(&cfg, patconv_reduce_kernel<XGEN_F32>, part_c, n_splits, oe, co, bias_c, rl, y, vec);
-        else if (p.dtype == XGEN_F16_F32ACC)
-            e = cudaLaunchKernelEx(&cfg, patconv_reduce_kernel<XGEN_F16_F32ACC>, part_c, n_splits, oe, co, bias_c, rl, y, vec);
-        else
-            e = cudaLaunchKernelEx(&cfg, patconv_reduce_kernel<XGEN_I8_I32>, part_c, n_splits, oe, co, bias_c, rl, y, vec);
-        if (e == cudaSuccess) e = cudaGetLastError();
-        e = log_cuda(e, "reduce launch");
-        if (e == cudaSuccess) g_launches.fetch_add(1);
-    }
-    if (prev != h->device) cudaSetDevice(prev);
-    if (e != cudaSuccess) return XGEN_ERR_CUDA;
-    g_launches.fetch_add(1);
+    const bool planned = h->plan_splits > 1 && h->plan_n == n && h->plan_h == hh && h->plan_w == ww;
+    memset(out, 0, sizeof(*out));
+    out->splits = planned ? h->plan_splits : 1;
+    out->chunks_per_split = planned ? h->plan_cps : p.n_chunks;
+    out->tiles = L.g.tiles_x * L.g.tiles_y * L.g.tiles_n;
+    out->filter_blocks = p.n_blocks;
+    out->items = L.items;
+    out->blocks = L.items * out->splits;
+    out->threads_per_block = (p.wpc + kProducerWarps) * 32;
+    out->lanes_x = 1 << L.g.lx_log; out->lanes_y = 1 << L.g.ly_log; out->lanes_n = 1 << L.g.ln_log;
+    out->pixels_per_lane = pixels_per_thread(p.stride);
+    out->stages = L.kp.n_stages;
+    out->uses_copy_engine = L.kp.use_tma;
+    out->shared_bytes = (int64_t)L.smem;
+    out->workspace_bytes = planned ? (int64_t)((size_t)L.items * (size_t)h->plan_splits * rows_per_item(p) * 1024) : 0;
     return XGEN_OK;
 }
 
-
-// The library's own scratch for xgen_patconv_run_static_scratch: partial sums of a split run.
-// It lives in every CUDA context that loads this library, until the process exits.
-static __device__ __align__(256) uint32_t g_static_scratch[XGEN_PATCONV_STATIC_SCRATCH_BYTES / 4];
-static uint32_t *g_static_scratch_addr[64];        // device address per device ordinal, resolved once
-static std::mutex g_static_scratch_mutex;
-
-extern "C" {
-
-xgen_status xgen_patconv_plan(xgen_patconv_packed *h, int32_t n, int32_t hh, int32_t ww) {
+xgen_status xgen_patconv_plan_tuned(xgen_patconv_packed *h, int32_t n, int32_t hh, int32_t ww,
+                                    const xgen_patconv_tuning *tuning) {
     if (!h) return XGEN_ERR_INVALID_ARG;
     if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
     if (h->device < 0) return XGEN_ERR_CUDA;
+    if (tuning && (tuning->splits < 0 || tuning->wait_limit_ms < 0)) return XGEN_ERR_INVALID_ARG;
     const PackedHost &p = h->host;
     const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
     if ((int64_t)n * ho * wo * p.c_out > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
+    const xgen_patconv_tuning tn = tuning ? *tuning : xgen_patconv_tuning{};
     Layout L;
-    xgen_status ls = make_layout(p, n, hh, ww, true, encode_tiled_fn() != nullptr, L);
+    xgen_status ls = make_layout(p, n, hh, ww, true, !tn.no_copy_engine && encode_tiled_fn() != nullptr, L);
     if (ls != XGEN_OK) return ls;
     int prev = 0;
     if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
@@ -1276,7 +1381,7 @@ xgen_status xgen_patconv_plan(xgen_patconv_packed *h, int32_t n, int32_t hh, int
     // and epilogue plus its multiply-adds at the rate an SM sustains with the warps it then
     // hosts; a split run adds the exchange of the partial sums.
     const int64_t capacity = (int64_t)sms * bps;
-    const int64_t max_splits = std::min<int64_t>(p.n_chunks, L.items > 0 ? capacity / L.items : 1);
+    const int64_t max_splits = std::max<int64_t>(1, std::min<int64_t>(p.n_chunks, L.items > 0 ? capacity / L.items : 1));
     const double slot_macs_item = 4.0 * (double)p.stats.kernels_surviving / (double)p.n_blocks * 32.0 * pixels_per_thread(p.stride);
     auto sm_rate = [&](int warps) { return 50.0 * std::pow((double)std::min(warps, 16) / 16.0, 0.65); };   // multiply-adds per cycle
     auto estimate = [&](int64_t k) {
@@ -1295,8 +1400,7 @@ xgen_status xgen_patconv_plan(xgen_patconv_packed *h, int32_t n, int32_t hh, int
         const double t = estimate(k);
         if (t < 0.97 * best_t) { best_t = t; splits = k; }
     }
-    if (const char *e = getenv("XGEN_PATCONV_SPLIT")) { int v = atoi(e); if (v >= 1) splits = std::min<int64_t>(v, std::max<int64_t>(1, max_splits)); }
-    if (splits < 1) splits = 1;
+    if (tn.splits >= 1) splits = std::min<int64_t>(tn.splits, max_splits);
     const int cps = (int)((p.n_chunks + splits - 1) / splits);
     splits = (p.n_chunks + cps - 1) / cps;
     if (rs == XGEN_OK && cudaDeviceSynchronize() != cudaSuccess) rs = XGEN_ERR_CUDA;
@@ -1316,12 +1420,28 @@ xgen_status xgen_patconv_plan(xgen_patconv_packed *h, int32_t n, int32_t hh, int
             else h->counter_bytes = need_c;
         }
         if (rs == XGEN_OK && cudaMemset(h->d_counters, 0, h->counter_bytes) != cudaSuccess) rs = XGEN_ERR_CUDA;
-        h->split_seq.store(0);
     }
     cudaSetDevice(prev);
+    {
+        std::lock_guard<std::mutex> lock(h->split_mu);
+        h->split_seq = 0;
+    }
+    forget_prepared_launches(h);
     if (rs != XGEN_OK) { h->plan_splits = 1; h->plan_n = 0; return rs; }
+    h->tuning = tn;
+    h->wait_us = tn.wait_limit_ms > 0 ? (uint32_t)std::min<int64_t>((int64_t)tn.wait_limit_ms * 1000, 60000000) : 2000000u;
     h->plan_n = n; h->plan_h = hh; h->plan_w = ww;
     h->plan_splits = (int)splits; h->plan_cps = cps;
+    return XGEN_OK;
+}
+
+xgen_status xgen_patconv_plan(xgen_patconv_packed *h, int32_t n, int32_t hh, int32_t ww) {
+    return xgen_patconv_plan_tuned(h, n, hh, ww, nullptr);
+}
+
+xgen_status xgen_patconv_test_expect_arrivals(xgen_patconv_packed *h, int32_t extra) {
+    if (!h || extra < 0) return XGEN_ERR_INVALID_ARG;
+    h->hook_extra_arrivals = extra;
     return XGEN_OK;
 }
 
@@ -1344,7 +1464,7 @@ xgen_status xgen_patconv_run_static_scratch(const xgen_patconv_packed *h, const 
     const int cps = (p.n_chunks + splits - 1) / splits;
     const int eff = (p.n_chunks + cps - 1) / cps;                 // splits that actually get chunks
     if (eff > 1 && (uint64_t)out_elems * 4u * (uint64_t)eff > (uint64_t)XGEN_PATCONV_STATIC_SCRATCH_BYTES) {
-        if (getenv("XGEN_PATCONV_LOG"))
+        if (log_enabled())
             fprintf(stderr, "libpatconv: %d splits x %lld outputs x 4 bytes exceed the %u-byte static scratch\n",
                     eff, (long long)out_elems, (unsigned)XGEN_PATCONV_STATIC_SCRATCH_BYTES);
         return XGEN_ERR_SHAPE;
@@ -1399,12 +1519,13 @@ xgen_status xgen_patconv_enqueue_host(const xgen_patconv_packed *h, const void *
         if (e == cudaSuccess) h->hy_bytes = ybytes;
     }
     if (e == cudaSuccess && bias && !h->d_hb) e = cudaMalloc(&h->d_hb, (size_t)p.c_out * 4);
+    if (e != cudaSuccess) { rs = (e == cudaErrorMemoryAllocation) ? XGEN_ERR_ALLOC : XGEN_ERR_CUDA; cudaGetLastError(); }
     if (e == cudaSuccess && !h->s_in) e = cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking);
     if (e == cudaSuccess && !h->s_out) e = cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking);
     if (e == cudaSuccess && !h->ev_in) e = cudaEventCreateWithFlags(&h->ev_in, cudaEventDisableTiming);
     if (e == cudaSuccess && !h->ev_run) e = cudaEventCreateWithFlags(&h->ev_run, cudaEventDisableTiming);
     if (e == cudaSuccess && !h->ev_out) e = cudaEventCreateWithFlags(&h->ev_out, cudaEventDisableTiming);
-    if (e != cudaSuccess) { rs = XGEN_ERR_ALLOC; cudaGetLastError(); }
+    if (rs == XGEN_OK && e != cudaSuccess) { rs = XGEN_ERR_CUDA; cudaGetLastError(); }
     void *dx = h->d_hx, *dy = h->d_hy, *db = bias ? h->d_hb : nullptr;
     // Copy in on the handle's first stream, the layer on the caller's, copy out on the handle's
     // second stream: the caller's stream carries kernels only, so the copies of one handle

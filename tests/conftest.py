@@ -24,3 +24,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter):
+    try:
+        from _gpu_util import FP16_ULP_STATS as st
+    except Exception:
+        return
+    if st["compared"]:
+        terminalreporter.write_line(
+            "fp16 results against the oracle rounded to fp16: %d compared (|ref| >= 0.01 S), "
+            "%d beyond one ulp, worst %d ulps" % (st["compared"], st["beyond_one_ulp"], st["worst_ulp"]))

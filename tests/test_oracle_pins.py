@@ -320,3 +320,55 @@ def test_fp16_inputs_are_used_as_stored():
     y16 = oracle.conv(d.x, d.w, d.pid, d.masks)
     y64 = oracle.conv(d.x.astype(np.float64), d.w.astype(np.float64), d.pid, d.masks)
     assert np.array_equal(y16, y64)
+
+
+# ---- the error scale S = |bias| + sum |w * x| (every floating-point tolerance uses it) --------
+def test_scale_hand_computed():
+    x = np.arange(1, 10, dtype=np.float64).reshape(1, 3, 3, 1)
+    w = np.arange(1, 10, dtype=np.float64).reshape(1, 1, 3, 3)
+    w[0, 0, 0, 1] = -2.0
+    w[0, 0, 1, 0] = -4.0
+    masks = np.array([_mask_of([0, 1, 3, 4])], dtype=np.uint16)
+    y, s = oracle.conv(x, w, np.zeros((1, 1), np.int16), masks, bias=np.array([-3.0]), with_scale=True)
+    rows = _read_gold("hand_scale_3x3.txt")
+    assert len(rows) == 4
+    for (oy, ox), (ey, es) in rows:
+        assert y[0, oy, ox, 0] == ey and s[0, oy, ox, 0] == es, (oy, ox, y[0, oy, ox, 0], s[0, oy, ox, 0])
+
+
+@pytest.mark.parametrize("stride", [1, 2])
+def test_scale_equals_output_for_nonnegative_terms(stride):
+    # x >= 0, kept weights >= 0, bias >= 0: every term is its own magnitude, so S == y, bit for bit
+    d = _small_case(51, n=2, ci=6, co=5, h=7, w=6, stride=stride)
+    x, w, b = np.abs(d.x), np.abs(d.w), np.abs(d.bias)
+    for relu in (False, True):
+        y, s = oracle.conv(x, w, d.pid, d.masks, bias=b, relu=relu, stride=stride, with_scale=True)
+        assert np.array_equal(y, s)
+        assert (s > 0).any()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16"])
+def test_scale_is_the_layer_on_magnitudes(dtype):
+    # S(x, W, bias) == y(|x|, |W|, |bias|) exactly: same loop order, and |w*x| == |w|*|x| in binary fp
+    d = _small_case(52, n=1, ci=7, co=6, h=6, w=7, dtype=dtype, stride=1)
+    assert (d.x < 0).any() or dtype == "f16"
+    assert (d.w < 0).any() and (d.bias < 0).any()
+    _, s = oracle.conv(d.x, d.w, d.pid, d.masks, bias=d.bias, relu=True, with_scale=True)
+    y_abs = oracle.conv(np.abs(d.x), np.abs(d.w), d.pid, d.masks, bias=np.abs(d.bias), relu=False)
+    assert np.array_equal(s, y_abs)
+    # without a bias the bias term is gone, and only then
+    _, s0 = oracle.conv(d.x, d.w, d.pid, d.masks, bias=None, with_scale=True)
+    assert np.allclose(s - s0, np.abs(d.bias).astype(np.float64)[None, None, None, :], rtol=0, atol=1e-12)
+
+
+def test_scale_ignores_relu_and_pruned_weights_and_is_homogeneous():
+    d = _small_case(53, n=1, ci=5, co=4, h=5, w=5)
+    _, s_lin = oracle.conv(d.x, d.w, d.pid, d.masks, bias=d.bias, relu=False, with_scale=True)
+    _, s_relu = oracle.conv(d.x, d.w, d.pid, d.masks, bias=d.bias, relu=True, with_scale=True)
+    assert np.array_equal(s_lin, s_relu)
+    w2 = np.where(_masked_dense(d) != 0, d.w, 1e6)             # garbage at pruned positions
+    _, s_g = oracle.conv(d.x, w2, d.pid, d.masks, bias=d.bias, with_scale=True)
+    assert np.array_equal(s_lin, s_g)
+    _, s2 = oracle.conv(2.0 * d.x.astype(np.float64), d.w, d.pid, d.masks, bias=2.0 * d.bias.astype(np.float64),
+                        with_scale=True)
+    assert np.array_equal(s2, 2.0 * s_lin)                     # doubling every term doubles S exactly

@@ -88,7 +88,19 @@ def test_index_overhead_below_csr_and_balance():
     pk = binding.Packed(spec.c_in, spec.c_out, 1, "f32", wl.pattern_library(8), w, pid, device=-1)
     st = pk.stats()
     assert st["kernels_surviving"] == spec.k_surv
-    assert st["index_bytes"] < st["csr_index_bytes"] / 4
+    # information content of the layout (one opcode and one operand byte per command plus the
+    # tables) against CSR's one 4-byte index per weight
+    assert st["compact_index_bytes"] < st["csr_index_bytes"] / 4
+    # what the device copy really stores beyond the kept weights: 48-byte slots and the tables
+    v = pk.view()
+    tables = 4 * (v["seg_off"].size + v["slot_oc"].size)
+    assert st["stream_bytes"] == 48 * len(v["slots"])
+    assert st["index_bytes"] == st["stream_bytes"] + tables - st["weight_bytes"]
+    assert st["weight_bytes"] == 16 * st["kernels_surviving"]
+    # per kernel that is 32 bytes (opcode, operand and the duplicate of the weights) plus the
+    # LOAD and END slots: about twice CSR's 16 bytes -- the price of decoding a command with
+    # two vector loads straight into the operand pairs of the packed FMAs
+    assert 1.5 * st["csr_index_bytes"] < st["index_bytes"] < 4 * st["csr_index_bytes"]
     assert 1.0 <= st["group_imbalance"] < 1.05
     assert st["patterns_compiled"] == 8
 

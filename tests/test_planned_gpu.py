@@ -1,0 +1,145 @@
+"""GPU parity of planned runs (xgen_patconv_plan before xgen_patconv_run), i.e. of the launch
+configuration bench.py times: channel splits exchanged and reduced inside the kernel, over
+several pixel tiles and several blocks of output channels.  Every comparison is against the CPU
+oracle, through the C ABI."""
+import numpy as np
+import pytest
+
+from paper_2206_10620_b200 import binding, workloads as wl
+from _gpu_util import compare, pack, run_gpu, guarded_output, check_guards
+
+pytestmark = pytest.mark.gpu
+
+
+def _layer(dtype, n, ci, co, h, w, stride=1, prune=0.5, lib=8, seed=1, idx=0):
+    xd = {"f32": "upm1", "f16": "relu_normal", "i8": "u01"}[dtype]
+    spec = wl.LayerSpec("t", n, ci, co, h, w, stride, dtype, prune, lib, "he", xd, 0.05, True, idx)
+    return wl.make_layer(spec, seed=seed)
+
+
+def test_vgg16_planned_every_layer_every_element():
+    """The benchmark's own stack, planned as the benchmark plans it: 11 of the 13 layers run as
+    in-kernel splits over several (tile x filter block) items."""
+    split_layers, most_items = 0, 0
+    for spec in wl.config_vgg16():
+        d = wl.make_layer(spec)
+        pk = pack(d)
+        y = run_gpu(pk, d.x, d.bias, True, plan=True)
+        info = pk.plan_info(spec.n, spec.h, spec.w)
+        assert info["blocks"] == info["items"] * info["splits"]
+        if info["splits"] > 1:
+            split_layers += 1
+            most_items = max(most_items, info["items"])
+            assert info["workspace_bytes"] > 0
+        compare(d, y)
+    assert split_layers >= 8 and most_items >= 4
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "i8"])
+@pytest.mark.parametrize("stride", [1, 2])
+def test_planned_split_over_several_tiles_and_filter_blocks(dtype, stride):
+    d = _layer(dtype, 2, 128, 264, 40, 40, stride, prune=0.6, lib=8, seed=61)
+    pk = pack(d)
+    pk.plan(2, 40, 40, splits=3)
+    info = pk.plan_info(2, 40, 40)
+    assert info["splits"] == 3 and info["tiles"] > 1 and info["filter_blocks"] > 1
+    assert info["items"] == info["tiles"] * info["filter_blocks"] and info["items"] > 4
+    y = run_gpu(pk, d.x, d.bias, True)
+    compare(d, y)
+    y2 = run_gpu(pk, d.x, None, False)
+    compare(d, y2, bias=None, relu=False)
+    assert np.array_equal(run_gpu(pk, d.x, d.bias, True), y)        # fixed reduction order
+
+
+def _sampled_batch_planned(spec, images):
+    d = wl.make_layer(spec)
+    pk = pack(d)
+    y = run_gpu(pk, d.x, d.bias, True, plan=True)
+    for i in images:
+        compare(d, y[i:i + 1], x=d.x[i:i + 1])
+    return pk.plan_info(spec.n, spec.h, spec.w)
+
+
+def test_resnet50_planned_one_layer_per_shape():
+    seen, splits = set(), []
+    for spec in wl.config_resnet50():
+        key = (spec.c_in, spec.h, spec.stride)
+        if key in seen:
+            continue
+        seen.add(key)
+        splits.append(_sampled_batch_planned(spec, [0, spec.n - 1])["splits"])
+    assert max(splits) > 1
+
+
+def test_resnet18_planned_one_layer_per_shape():
+    seen, splits = set(), []
+    for spec in wl.config_resnet18():
+        key = (spec.c_in, spec.c_out, spec.h, spec.stride)
+        if key in seen:
+            continue
+        seen.add(key)
+        splits.append(_sampled_batch_planned(spec, [0, spec.n - 1])["splits"])
+    assert max(splits) > 1
+
+
+@pytest.mark.parametrize("lib", [4, 8, 12])
+def test_sweep_every_point_planned(lib):
+    """All 48 points of the single-layer sweep (16 per library size), planned as in the benchmark;
+    the first and the last image of every batch against the oracle."""
+    pts = [s for s in wl.config_sweep() if s.lib_size == lib]
+    assert len(pts) == 16 and sorted({s.n for s in pts}) == [1, 8, 64, 256]
+    for spec in pts:
+        _sampled_batch_planned(spec, [0] if spec.n == 1 else [0, spec.n - 1])
+
+
+@pytest.mark.parametrize("dtype,stride", [("f32", 2), ("f16", 1), ("f16", 2), ("i8", 1), ("i8", 2)])
+def test_universal_table_other_variants(dtype, stride):
+    d = _layer(dtype, 2, 24, 40, 13, 15, stride, prune=0.4, lib=4, seed=71)
+    d.masks = np.array([0x00F, 0x1E0, 0x145, 0x0AA], dtype=np.uint16)     # none of the built-in shapes
+    pk = pack(d)
+    assert pk.stats()["patterns_compiled"] == 126
+    compare(d, run_gpu(pk, d.x, d.bias, True))
+
+
+@pytest.mark.parametrize("knob", ["no_copy_engine", "no_launch_overlap"])
+@pytest.mark.parametrize("dtype", ["f32", "i8"])
+def test_tuning_switches_keep_the_result(knob, dtype):
+    d = _layer(dtype, 2, 64, 48, 22, 22, 1, prune=0.5, lib=8, seed=81)
+    pk = pack(d)
+    pk.plan(2, 22, 22, splits=2)
+    assert pk.plan_info(2, 22, 22)["uses_copy_engine"] == 1
+    y0 = run_gpu(pk, d.x, d.bias, True)
+    pk.plan(2, 22, 22, splits=2, **{knob: True})
+    info = pk.plan_info(2, 22, 22)
+    assert info["splits"] == 2
+    if knob == "no_copy_engine":
+        assert info["uses_copy_engine"] == 0
+    y1 = run_gpu(pk, d.x, d.bias, True)
+    compare(d, y1)
+    assert np.array_equal(y0, y1)        # same sums in the same order, whatever stages the tiles
+
+
+def test_bounded_wait_runs_out_and_the_handle_recovers():
+    """A planned split told to expect one arrival that never comes: every block's wait runs out
+    after the (shortened) limit, the kernel ends by itself, xgen_patconv_last_status reports
+    the timeout once, and the next ordinary run is correct again.  Nothing traps or spins on."""
+    import torch
+    d = _layer("f32", 1, 128, 32, 12, 12, 1, prune=0.5, lib=8, seed=91)
+    pk = pack(d)
+    pk.plan(1, 12, 12, splits=4, wait_limit_ms=20)
+    assert pk.plan_info(1, 12, 12)["splits"] == 4
+    compare(d, run_gpu(pk, d.x, d.bias, True))
+    pk.test_expect_arrivals(1)
+    x = torch.from_numpy(d.x).cuda()
+    b = torch.from_numpy(d.bias).cuda()
+    buf, y = guarded_output((1, 12, 12, 32), torch.float32)
+    st = torch.cuda.current_stream().cuda_stream
+    pk.run(x.data_ptr(), 1, 12, 12, b.data_ptr(), True, y.data_ptr(), st)      # only enqueues: OK
+    with pytest.raises(binding.PatconvError) as e:
+        pk.sync(st)
+    assert e.value.status == 7
+    check_guards(buf)
+    pk.sync(st)                                                                # reported once
+    pk.test_expect_arrivals(0)
+    compare(d, run_gpu(pk, d.x, d.bias, True))
+    compare(d, run_gpu(pk, d.x, d.bias, True))

@@ -7,7 +7,9 @@ sums in an array built into the library.  This file checks that entry point,
 through the C ABI, against the ordinary xgen_patconv_run on the same inputs:
 twice in a row (the array is shared between calls and keeps old contents), for
 the three numeric variants, and that a request beyond the array's size is
-refused.  It is collected last on purpose and does not depend on other tests.
+refused.  Both results are also compared with the CPU oracle, and the free
+device memory is read before and after the calls: it must not move.  The file is
+collected last on purpose and does not depend on other tests.
 """
 import numpy as np
 import pytest
@@ -49,19 +51,31 @@ def test_matches_ordinary_run_twice_in_a_row(dtype, stride):
     pk.run(x.data_ptr(), s.n, s.h, s.w, b.data_ptr(), True, y_ref.data_ptr(), st)
     pk.sync(st)
     ref = y_ref.cpu().numpy()
-    if dtype != "i8":
-        _, S = oracle.conv(d.x, d.w, d.pid, d.masks, bias=d.bias, relu=True, stride=stride, with_scale=True)
-    for splits in (6, 3):                                  # two calls in a row, different splits
-        y = mk()
+    if dtype == "i8":
+        truth = oracle.conv(d.x, d.w, d.pid, d.masks, bias=d.bias, relu=True, stride=stride)
+        assert np.array_equal(ref.astype(np.int64), truth)
+    else:
+        truth, S = oracle.conv(d.x, d.w, d.pid, d.masks, bias=d.bias, relu=True, stride=stride, with_scale=True)
+    outs = [mk(), mk()]                                    # allocated before the memory reading
+    pk.run_static_scratch(x.data_ptr(), s.n, s.h, s.w, b.data_ptr(), True, outs[0].data_ptr(), 2, st)   # first call
+    pk.sync(st)                                            # on this device: resolves the array's address
+    outs[0].fill_(77)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for y, splits in zip(outs, (6, 3)):                    # two calls in a row, different splits
         pk.run_static_scratch(x.data_ptr(), s.n, s.h, s.w, b.data_ptr(), True, y.data_ptr(), splits, st)
-        pk.sync(st)
+    pk.sync(st)
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "the call that must not allocate changed the free device memory"
+    for y in outs:
         got = y.cpu().numpy()
         if dtype == "i8":
-            assert np.array_equal(got, ref)
+            assert np.array_equal(got, ref)                # the ordinary entry point
+            assert np.array_equal(got.astype(np.int64), truth)   # and the oracle
         else:
-            err = np.abs(got.astype(np.float64) - ref.astype(np.float64))
-            bound = TOL[dtype] * np.maximum(np.abs(ref.astype(np.float64)), 0.01 * S) + 1e-30
-            assert (err <= bound).all()
+            bound = TOL[dtype] * np.maximum(np.abs(truth), 0.01 * S) + 1e-30
+            assert (np.abs(got.astype(np.float64) - truth) <= bound).all()                       # the oracle
+            assert (np.abs(got.astype(np.float64) - ref.astype(np.float64)) <= 2 * bound).all()  # the ordinary entry point
     # a second layer through the same array right after: old contents must not leak
     d2 = _layer(dtype, 1, 64, 24, 9, stride, seed=22)
     s2 = d2.spec
