@@ -339,6 +339,27 @@ void xgen_patconv_free(xgen_patconv_packed *packed);
 /* Static, human-readable name of a status code. */
 const char *xgen_strerror(xgen_status status);
 
+/*
+ * Measurement aid (the paper has no counterpart): rates of the arithmetic pipes that bound
+ * the convolution kernels, from register-only microbenchmarks at full occupancy, and the
+ * cost of launching a kernel shaped like them.  Runs a few kernels of about a millisecond
+ * on the device's default stream and waits for them.
+ *   ffma_tflops       scalar fp32 fused multiply-add (2 flop each)
+ *   ffma2_tflops      packed two-wide fp32 fused multiply-add (the instruction the kernels use)
+ *   dp4a_tmacs        u8 x s8 four-way dot product into int32, in 10^12 multiply-adds per second
+ *   launch_floor_us   microseconds per launch over 200 back-to-back launches of an empty kernel
+ *                     with the convolution kernels' block size, shared-memory carve-out,
+ *                     tensor-memory allocation and launch attribute (128 blocks)
+ *   single_launch_us  one such launch, from the event before it to the event after it
+ *   sm_count, sm_clock_mhz  as the device reports them (the clock is the rated maximum)
+ * Errors: INVALID_ARG, ALLOC, CUDA.
+ */
+typedef struct {
+    double ffma_tflops, ffma2_tflops, dp4a_tmacs, launch_floor_us, single_launch_us;
+    int32_t sm_count, sm_clock_mhz;
+} xgen_patconv_probe_result;
+xgen_status xgen_patconv_probe(int device, xgen_patconv_probe_result *result);
+
 /* Number of kernel launches this library has enqueued in this process. */
 int64_t xgen_patconv_launch_count(void);
 

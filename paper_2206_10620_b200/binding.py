@@ -26,7 +26,7 @@ EXPORTS = ["xgen_patconv_pack", "xgen_patconv_run", "xgen_patconv_run_static_scr
            "xgen_patconv_plan_tuned", "xgen_patconv_plan_info", "xgen_patconv_test_expect_arrivals",
            "xgen_patconv_out_shape", "xgen_patconv_query", "xgen_patconv_view",
            "xgen_patconv_last_status", "xgen_patconv_free", "xgen_strerror",
-           "xgen_patconv_launch_count"]
+           "xgen_patconv_launch_count", "xgen_patconv_probe"]
 
 
 class Desc(ctypes.Structure):
@@ -60,6 +60,12 @@ class PlanStats(ctypes.Structure):
                 ("lanes_n", ctypes.c_int32), ("pixels_per_lane", ctypes.c_int32), ("stages", ctypes.c_int32),
                 ("uses_copy_engine", ctypes.c_int32), ("shared_bytes", ctypes.c_int64),
                 ("workspace_bytes", ctypes.c_int64)]
+
+
+class ProbeResult(ctypes.Structure):
+    _fields_ = [("ffma_tflops", ctypes.c_double), ("ffma2_tflops", ctypes.c_double), ("dp4a_tmacs", ctypes.c_double),
+                ("launch_floor_us", ctypes.c_double), ("single_launch_us", ctypes.c_double),
+                ("sm_count", ctypes.c_int32), ("sm_clock_mhz", ctypes.c_int32)]
 
 
 class HostView(ctypes.Structure):
@@ -104,6 +110,7 @@ def lib():
         L.xgen_strerror.argtypes = [ctypes.c_int]
         L.xgen_strerror.restype = ctypes.c_char_p
         L.xgen_patconv_launch_count.restype = ctypes.c_int64
+        L.xgen_patconv_probe.argtypes = [ctypes.c_int, ctypes.POINTER(ProbeResult)]
         for name in EXPORTS:
             if name not in ("xgen_patconv_free", "xgen_strerror", "xgen_patconv_launch_count"):
                 getattr(L, name).restype = ctypes.c_int
@@ -236,6 +243,13 @@ class Packed:
 
 def launch_count() -> int:
     return int(lib().xgen_patconv_launch_count())
+
+
+def probe(device=0) -> dict:
+    """xgen_patconv_probe: measured pipe rates and launch floor of the device."""
+    r = ProbeResult()
+    _check(lib().xgen_patconv_probe(int(device), ctypes.byref(r)), "xgen_patconv_probe")
+    return {k: getattr(r, k) for k, _ in ProbeResult._fields_}
 
 
 def strerror(status: int) -> str:

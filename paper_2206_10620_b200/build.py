@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_HERE, "csrc")
 _INC = os.path.join(os.path.dirname(_HERE), "include")
 LIB_PATH = os.path.join(_HERE, "libpatconv.so")
-_SOURCES = ["patconv.cu", "pack.cpp"]
+_SOURCES = ["patconv.cu", "probe.cu", "pack.cpp"]
 _DEPS = _SOURCES + ["patconv_internal.h", "gen_core.py", os.path.join(_INC, "patconv.h")]
 
 
