@@ -292,12 +292,16 @@ typedef struct {
     int32_t items;              /* tiles x filter_blocks                                           */
     int32_t blocks;             /* thread blocks of the launch: items x splits                     */
     int32_t threads_per_block;
+    int32_t row_tiling;         /* 0: a tile is a box of lanes_x x lanes_y blocks of lanes_n images;
+                                   1: a tile is 32 consecutive blocks of the row-by-row numbering
+                                   of all images' blocks (lanes_x = blocks per image row)         */
     int32_t lanes_x, lanes_y, lanes_n;  /* how a warp's 32 lanes tile x, y and images             */
     int32_t pixels_per_lane;    /* output pixels one lane owns (16 at stride 1, 8 at stride 2)     */
     int32_t stages;             /* pipeline stages of staged channel chunks                        */
     int32_t uses_copy_engine;   /* input tiles arrive through the tensor copy engine               */
     int64_t shared_bytes;       /* dynamic shared memory per block                                 */
     int64_t workspace_bytes;    /* partial-sum workspace of the planned split, 0 if unsplit        */
+    double  covered;            /* output pixels / pixel slots of all tiles (lanes x pixels each)  */
 } xgen_patconv_plan_stats;
 
 /* Fill *stats for the shape.  No CUDA work is enqueued.  Errors: INVALID_ARG, SHAPE, UNSUPPORTED. */

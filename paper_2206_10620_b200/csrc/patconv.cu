@@ -59,7 +59,16 @@ struct KParams {
     int relu;
     int J, wpc, cc, n_chunks;
     int rc;                              // channels per tile box (a multiple of cc)
-    int lx_log, ly_log, ln_log;          // lanes along x, y and images: 2^.. each, product 32
+    int lx_log, ly_log, ln_log;          // grid tiling: lanes along x, y and images: 2^.. each, product 32
+    // Row tiling (rows != 0): the 4x4 (2x4) pixel blocks of all images are numbered row by row
+    // (image, block row, block column) and a tile is 32 consecutive blocks, one per lane; the
+    // block rows it touches are staged one "slot" each (full image width, own halo rows).
+    int rows;
+    int bxn, byn;                        // blocks per image row, block rows per image
+    uint32_t mg_bxn, mg_byn;
+    int blocks_total;                    // n * byn * bxn
+    int n_slots;                         // staged slots per tile: images (grid tiling) or block rows (row tiling)
+    int slot_bytes;                      // bytes one tensor copy delivers in row tiling (one slot)
     int tiles_x, tiles_y;
     int tin_w, tin_h;                    // staged tile extents, input pixels
     uint32_t mg_tiles_x, mg_tiles_y, mg_tin_w, mg_tin_h, mg_spb;   // division by these as a multiplication (div_by)
@@ -234,6 +243,13 @@ __device__ __forceinline__ void store_piece(const KParams &P, const uint32_t (&r
 // exact while n * d < 2^32.
 __device__ __forceinline__ int div_by(int n, uint32_t m) { return m ? (int)__umulhi((uint32_t)n, m) : n; }
 
+// Where a lane works: the first output pixel of its block, its image, and the word offset of
+// its patch origin inside a channel plane (half 0).
+struct LaneSite { int on, oy0, ox0, off; bool valid; };
+
+// Where a staged slot comes from: image and input coordinates of its first staged pixel.
+struct SlotOrigin { int gn, gy0, gx0; bool used; };
+
 // ---- the kernel -----------------------------------------------------------------
 template <int DT, int STRIDE, int NP>
 __global__ void __launch_bounds__((kMaxWarps + kProducerWarps) * 32)
@@ -253,17 +269,49 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     const int b = blockIdx.y;
     const int item = (int)(blockIdx.x + gridDim.x * blockIdx.y);   // (tile, filter block)
     const int tile = blockIdx.x;
+    // grid tiling: tile -> (tx, ty, first image)
     const int tile_r = div_by(tile, P.mg_tiles_x);
     const int tx = tile - tile_r * P.tiles_x;
     const int tn = div_by(tile_r, P.mg_tiles_y);
     const int ty = tile_r - tn * P.tiles_y;
-    const int LX = 1 << P.lx_log, LY = 1 << P.ly_log;
-    const int l_x = lane & (LX - 1), l_y = (lane >> P.lx_log) & (LY - 1), l_n = lane >> (P.lx_log + P.ly_log);
+    const int LX = P.rows ? P.bxn : (1 << P.lx_log), LY = 1 << P.ly_log;
     const int TW = BW * LX, TH = BH * LY;
     const int n0 = tn << P.ln_log;                   // first image of the tile
-    const int gy0 = ty * TH * STRIDE - 1, gx0 = tx * TW * STRIDE - 1;   // input coords of tile (0,0)
+    // row tiling: the tile's blocks 32*tile .. 32*tile+31 lie in block rows g_first .. g_last
+    const int g_first = div_by(tile * 32, P.mg_bxn);
+    const int g_last = div_by(min(tile * 32 + 31, P.blocks_total - 1), P.mg_bxn);
+    auto lane_site = [&](int l) {
+        LaneSite r;
+        if (P.rows) {
+            const int bl = tile * 32 + l;
+            const int g = div_by(bl, P.mg_bxn), bx = bl - g * P.bxn;
+            const int n = div_by(g, P.mg_byn), by = g - n * P.byn;
+            r.on = n; r.oy0 = by * BH; r.ox0 = bx * BW;
+            r.valid = bl < P.blocks_total;
+            r.off = r.valid ? (g - g_first) * P.img_stride + bx * 4 : 0;   // idle lanes read slot 0
+        } else {
+            const int l_x = l & (LX - 1), l_y = (l >> P.lx_log) & (LY - 1), l_n = l >> (P.lx_log + P.ly_log);
+            r.on = n0 + l_n; r.oy0 = ty * TH + l_y * BH; r.ox0 = tx * TW + l_x * BW;
+            r.off = l_n * P.img_stride + l_y * BH * STRIDE * P.pitch + l_x * 4;
+            r.valid = true;
+        }
+        return r;
+    };
+    auto slot_origin = [&](int sl) {
+        SlotOrigin r;
+        if (P.rows) {
+            const int g = g_first + sl;
+            const int n = div_by(g, P.mg_byn), by = g - n * P.byn;
+            r.gn = n; r.gy0 = by * BH * STRIDE - 1; r.gx0 = -1; r.used = g <= g_last;
+        } else {
+            r.gn = n0 + sl; r.gy0 = ty * TH * STRIDE - 1; r.gx0 = tx * TW * STRIDE - 1; r.used = true;
+        }
+        return r;
+    };
+    const int slots_used = P.rows ? g_last - g_first + 1 : P.n_slots;
     const int NS = P.n_stages;
-    const int npix = (P.tin_w * P.tin_h) << P.ln_log;
+    const int npix = P.tin_w * P.tin_h * slots_used;       // staged pixels that are read
+    const int npix_tab = P.tin_w * P.tin_h * P.n_slots;    // entries of the per-pixel tables
 
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t mbar0 = smem_base + (uint32_t)P.mbar_off_words * 4u;
@@ -310,9 +358,20 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     auto issue_box = [&](int q) {
         const int r = (q - q0) % kRawStages;
         const uint32_t dst = smem_base + (uint32_t)(P.raw_off_words + r * P.raw_stage_words) * 4u;
-        mbar_expect_tx(bar_raw(r), (uint32_t)P.box_bytes);
-        asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-                     ::"r"(dst), "l"(&tmap), "r"(q * P.rc), "r"(gx0), "r"(gy0), "r"(n0), "r"(bar_raw(r)) : "memory");
+        if (P.rows) {
+            // one copy per block row the tile touches: full image width, own halo rows
+            mbar_expect_tx(bar_raw(r), (uint32_t)(P.slot_bytes * slots_used));
+            for (int sl = 0; sl < slots_used; ++sl) {
+                const SlotOrigin o = slot_origin(sl);
+                asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                             ::"r"(dst + (uint32_t)(sl * P.slot_bytes)), "l"(&tmap), "r"(q * P.rc), "r"(o.gx0), "r"(o.gy0), "r"(o.gn), "r"(bar_raw(r)) : "memory");
+            }
+        } else {
+            const SlotOrigin o = slot_origin(0);
+            mbar_expect_tx(bar_raw(r), (uint32_t)P.box_bytes);
+            asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                         ::"r"(dst), "l"(&tmap), "r"(q * P.rc), "r"(o.gx0), "r"(o.gy0), "r"(o.gn), "r"(bar_raw(r)) : "memory");
+        }
     };
     if (pw == 0 && lane == 0 && P.use_tma) {
         asm volatile("griddepcontrol.wait;" ::: "memory");       // x is complete
@@ -345,7 +404,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     // pixel therefore lands in at most two places.
     int2 *tab = reinterpret_cast<int2 *>(smem + P.tab_off_words);
     int *srct = reinterpret_cast<int *>(smem + P.src_off_words);
-    for (int q = tid; q < npix; q += nthreads) {
+    for (int q = tid; q < npix_tab; q += nthreads) {
         const int t2 = div_by(q, P.mg_tin_w), col = q - t2 * P.tin_w;
         const int im = div_by(t2, P.mg_tin_h), row = t2 - im * P.tin_h;
         const int base = im * P.img_stride + row * P.pitch;
@@ -367,8 +426,9 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         }
         tab[q] = make_int2(d0, d1);
         if (!P.use_tma) {
-            const int gy = gy0 + row, gx = gx0 + col, gn = n0 + im;
-            const bool ok = gn < P.n && gy >= 0 && gy < P.h && gx >= 0 && gx < P.w;
+            const SlotOrigin o = slot_origin(im);
+            const int gy = o.gy0 + row, gx = o.gx0 + col, gn = o.gn;
+            const bool ok = o.used && gn < P.n && gy >= 0 && gy < P.h && gx >= 0 && gx < P.w;
             srct[q] = ok ? ((gn * P.h + gy) * P.w + gx) * P.c_in : -1;
         }
     }
@@ -385,11 +445,11 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     int *ptab = reinterpret_cast<int *>(smem + P.ptab_off_words);
     for (int i = tid; !producer && i < 32 * T; i += cthreads) {
         const int t = i >> 5, l2 = i & 31;
-        const int p_x = l2 & (LX - 1), p_y = (l2 >> P.lx_log) & (LY - 1), p_n = l2 >> (P.lx_log + P.ly_log);
+        const LaneSite ls = lane_site(l2);
         const int py = STRIDE == 1 ? (t >> 2) : (t >> 1);
         const int px = STRIDE == 1 ? (((t >> 1) & 1) + 2 * (t & 1)) : (t & 1);
-        const int ox = tx * TW + p_x * BW + px, oy = ty * TH + p_y * BH + py, on = n0 + p_n;
-        ptab[i] = (on < P.n && oy < P.ho && ox < P.wo) ? (on * P.ho + oy) * P.wo + ox : -1;
+        const int ox = ls.ox0 + px, oy = ls.oy0 + py, on = ls.on;
+        ptab[i] = (ls.valid && on < P.n && oy < P.ho && ox < P.wo) ? (on * P.ho + oy) * P.wo + ox : -1;
     }
     // Segment offsets of this block's chunks.
     int *seg = reinterpret_cast<int *>(smem + P.seg_off_words);
@@ -438,6 +498,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
 #pragma unroll 2
                 for (int i = ptid; i < npix; i += kProducerWarps * 32) {
                     const int2 d = tab[i];
+                    if (d.x < 0) continue;                 // a padding column of a slot: no lane reads it
                     float *d0 = pl + d.x, *d1 = pl + (d.y >= 0 ? d.y : d.x);
                     const char *src = rawb + (size_t)i * pix_bytes;
                     auto word = [&](uint32_t w, int e) {                   // one 32-bit word = 4 / XB channels from e on
@@ -489,6 +550,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                 const int ic0 = c * P.cc;
                 for (int i = ptid; i < npix; i += kProducerWarps * 32) {
                     const int2 d = tab[i];
+                    if (d.x < 0) continue;
                     const int src = srct[i];
                     float *d0 = pl + d.x, *d1 = pl + (d.y >= 0 ? d.y : d.x);
 #pragma unroll 4
@@ -534,7 +596,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
             tmem_wait_st();
         };
 
-        const uint32_t thr_off = (uint32_t)(l_n * P.img_stride + l_y * BH * STRIDE * P.pitch + l_x * 4) * 4u;
+        const uint32_t thr_off = (uint32_t)lane_site(lane).off * 4u;
         const uint32_t half_bytes = (uint32_t)P.half_stride * 4u;
 
         // The first bounded wait below must not start counting while an earlier kernel of the
@@ -743,19 +805,17 @@ static inline int pixels_per_thread(int stride) { return 4 * pixels_per_thread_x
 
 struct Geometry {
     int lx_log, ly_log, ln_log, tiles_x, tiles_y, tiles_n;
+    int rows, bxn, byn, blocks_total, n_slots, tiles;   // row tiling (rows != 0); n_slots, tiles: either tiling
     int tin_w, tin_h, pitch, img_stride, half_stride, plane_stride;
+    double covered;                                      // output pixels / pixel slots of all tiles
 };
 
-// Worst bank multiplicity of a thread's 128-bit patch-row load for a candidate layout:
-// a lane reads 4 words at (image, its first tile row, its lane column x 4).
-static int row_load_conflicts(int stride, int lx_log, int ly_log, int pitch, int img_stride) {
-    const int LX = 1 << lx_log, LY = 1 << ly_log;
-    auto addr = [&](int lane) {
-        int x = lane & (LX - 1), y = (lane >> lx_log) & (LY - 1), n = lane >> (lx_log + ly_log);
-        return n * img_stride + y * 4 * stride * pitch + x * 4;   // words
-    };
+// Worst bank multiplicity of a thread's 128-bit patch-row load: `addr` gives the word offset of a
+// lane's patch origin inside a plane; 128-bit accesses go out 8 lanes per wavefront.
+template <typename F>
+static int row_load_conflicts(F addr) {
     int worst = 0;
-    for (int ph = 0; ph < 4; ++ph) {                      // 128-bit accesses: 8 lanes per wavefront
+    for (int ph = 0; ph < 4; ++ph) {
         int cnt[32] = {0};
         for (int l = 0; l < 8; ++l) {
             int a = addr(ph * 8 + l);
@@ -766,7 +826,9 @@ static int row_load_conflicts(int stride, int lx_log, int ly_log, int pitch, int
     return worst;
 }
 
-static Geometry choose_geometry(int n, int ho, int wo, int stride) {
+// Grid tiling: the 32 lanes of a warp tile LX x LY x LN (powers of two) blocks of 4x4 (2x4)
+// pixels; chosen to cover the most output pixels per tile.
+static Geometry grid_geometry(int n, int ho, int wo, int stride) {
     Geometry best{};
     double best_eff = -1.0;
     const int bw = pixels_per_thread_x(stride), bh = 4;
@@ -784,6 +846,10 @@ static Geometry choose_geometry(int n, int ho, int wo, int stride) {
         }
     const int TW = bw << best.lx_log, TH = bh << best.ly_log, LN = 1 << best.ln_log;
     best.tiles_x = (wo + TW - 1) / TW; best.tiles_y = (ho + TH - 1) / TH; best.tiles_n = (n + LN - 1) / LN;
+    best.tiles = best.tiles_x * best.tiles_y * best.tiles_n;
+    best.n_slots = LN;
+    best.blocks_total = 1 << 30;
+    best.covered = best_eff;
     best.tin_w = stride == 1 ? TW + 2 : 2 * TW + 1;
     best.tin_h = stride == 1 ? TH + 2 : 2 * TH + 1;
     // One half of a plane row holds 4 words per lane column; pad the row and the image so
@@ -793,7 +859,11 @@ static Geometry choose_geometry(int n, int ho, int wo, int stride) {
     for (int p = p0; p <= p0 + 12; p += 4)
         for (int ipad = 0; ipad <= (LN > 1 ? 28 : 0); ipad += 4) {
             const int istr = best.tin_h * p + ipad;
-            const int c = row_load_conflicts(stride, best.lx_log, best.ly_log, p, istr);
+            const int LX = 1 << best.lx_log, LY = 1 << best.ly_log;
+            const int c = row_load_conflicts([&](int lane) {
+                int x = lane & (LX - 1), y = (lane >> best.lx_log) & (LY - 1), nn = lane >> (best.lx_log + best.ly_log);
+                return nn * istr + y * 4 * stride * p + x * 4;
+            });
             if (c < best_c) { best_c = c; best_p = p; best_i = istr; }
         }
     best.pitch = best_p;
@@ -801,6 +871,46 @@ static Geometry choose_geometry(int n, int ho, int wo, int stride) {
     best.half_stride = LN * best.img_stride;
     best.plane_stride = 2 * best.half_stride;
     return best;
+}
+
+// Row tiling: the blocks of all images are numbered (image, block row, block column) and a
+// tile takes 32 consecutive ones, so only the last tile of the launch has idle lanes; what is
+// lost is the part of edge blocks that hangs over the image.  Every block row a tile touches is
+// staged as a slot of its own: the full image width plus halo, with its own halo rows.
+static bool row_geometry(int n, int ho, int wo, int stride, Geometry &g) {
+    const int bw = pixels_per_thread_x(stride), bh = 4;
+    const int bxn = (wo + bw - 1) / bw, byn = (ho + bh - 1) / bh;
+    if (bxn > 32) return false;
+    const int64_t total = (int64_t)n * byn * bxn;
+    if (total > (int64_t)1 << 26) return false;
+    g = Geometry{};
+    g.rows = 1; g.bxn = bxn; g.byn = byn; g.blocks_total = (int)total;
+    g.tiles = (int)((total + 31) / 32);
+    g.tiles_x = g.tiles; g.tiles_y = 1; g.tiles_n = 1;
+    g.n_slots = std::min<int64_t>((31 + bxn - 1) / bxn + 1, (int64_t)n * byn);   // most block rows 32 consecutive blocks touch
+    g.covered = (double)n * ho * wo / ((double)g.tiles * 32.0 * bw * bh);
+    g.tin_w = stride == 1 ? bxn * bw + 2 : 2 * bxn * bw + 1;
+    g.tin_h = stride == 1 ? bh + 2 : 2 * bh + 1;
+    // pad the row pitch and the slot stride so that a quarter warp's 128-bit loads spread over the banks,
+    // whatever block column the tile starts at
+    const int p0 = 4 * bxn;
+    int best_p = p0, best_i = g.tin_h * p0, best_c = 1 << 30;
+    for (int p = p0; p <= p0 + 12; p += 4)
+        for (int ipad = 0; ipad <= 28; ipad += 4) {
+            const int istr = g.tin_h * p + ipad;
+            int c = 0;
+            for (int start = 0; start < bxn; ++start)
+                c = std::max(c, row_load_conflicts([&](int lane) {
+                    const int bl = start + lane;
+                    return (bl / bxn) * istr + (bl % bxn) * 4;
+                }));
+            if (c < best_c) { best_c = c; best_p = p; best_i = istr; }
+        }
+    g.pitch = best_p;
+    g.img_stride = best_i;
+    g.half_stride = g.n_slots * g.img_stride;
+    g.plane_stride = 2 * g.half_stride;
+    return true;
 }
 
 // Everything about a launch that depends only on the layer and the input shape: tile
@@ -961,20 +1071,31 @@ static cudaError_t allow_large_smem(const void *kern) {
 
 static int next_pow2(int v) { int p = 32; while (p < v) p <<= 1; return p; }
 
-static xgen_status make_layout(const PackedHost &p, int n, int hh, int ww, bool y_aligned32, bool tma_ok, Layout &L) {
+static xgen_status layout_for(const PackedHost &p, const Geometry &g_in, int n, int hh, int ww, bool y_aligned32,
+                              bool tma_ok, Layout &L) {
     const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
-    const Geometry g = choose_geometry(n, ho, wo, p.stride);
+    Geometry g = g_in;
+    if (g.rows) {
+        // Every slot is the destination of a tensor copy of its own and must start on a
+        // 128-byte boundary of shared memory: widen the staged rows (the extra columns are
+        // copied, or zero-filled beyond the image, and never used) until a slot is a
+        // multiple of 128 bytes.
+        const int xb0 = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
+        const int rc0 = p.cc * xb0 >= 16 ? p.cc : 16 / xb0;
+        while ((g.tin_w * g.tin_h * rc0 * xb0) % 128 != 0) ++g.tin_w;
+    }
     L.g = g;
     KParams kp{};
     kp.n = n; kp.h = hh; kp.w = ww; kp.ho = ho; kp.wo = wo; kp.c_in = p.c_in; kp.c_out = p.c_out;
     kp.J = p.J; kp.wpc = p.wpc; kp.cc = p.cc; kp.n_chunks = p.n_chunks;
     kp.lx_log = g.lx_log; kp.ly_log = g.ly_log; kp.ln_log = g.ln_log;
+    kp.rows = g.rows; kp.bxn = g.bxn; kp.byn = g.byn; kp.blocks_total = g.blocks_total; kp.n_slots = g.n_slots;
     kp.tiles_x = g.tiles_x; kp.tiles_y = g.tiles_y;
     kp.tin_w = g.tin_w; kp.tin_h = g.tin_h;
     kp.pitch = g.pitch; kp.img_stride = g.img_stride; kp.plane_stride = g.plane_stride;
     kp.half_stride = g.half_stride;
     const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
-    const int npix_box = (g.tin_w * g.tin_h) << g.ln_log;
+    const int npix_box = g.tin_w * g.tin_h * g.n_slots;
     // A box carries at least 16 bytes of channels per pixel; a chunk may be a part of it.
     // The copy engine needs 16-byte multiples in every global stride.
     kp.rc = p.cc * xb >= 16 ? p.cc : 16 / xb;
@@ -982,8 +1103,10 @@ static xgen_status make_layout(const PackedHost &p, int n, int hh, int ww, bool 
     auto magic = [](int d) { return d <= 1 ? 0u : (uint32_t)((1ull << 32) / (uint64_t)d + 1ull); };
     kp.mg_tiles_x = magic(g.tiles_x); kp.mg_tiles_y = magic(g.tiles_y);
     kp.mg_tin_w = magic(g.tin_w); kp.mg_tin_h = magic(g.tin_h); kp.mg_spb = magic(kp.spb);
+    kp.mg_bxn = magic(g.bxn); kp.mg_byn = magic(g.byn);
     kp.use_tma = tma_ok && ((p.cc * xb) % 4 == 0) && (((size_t)p.c_in * xb) % 16 == 0) && g.tin_w <= 256 && g.tin_h <= 256;
     kp.box_bytes = npix_box * kp.rc * xb;
+    kp.slot_bytes = g.tin_w * g.tin_h * kp.rc * xb;
     // widest aligned store per 8-channel piece: 8 words (32-byte aligned rows), 4, or scalar
     kp.vec_out = ((p.c_out % 8) == 0 && y_aligned32) ? 8 : ((p.c_out % 4) == 0 ? 4 : 0);
     const bool is_i8 = p.dtype == XGEN_I8_I32;
@@ -1033,8 +1156,32 @@ static xgen_status make_layout(const PackedHost &p, int n, int hh, int ww, bool 
     kp.out_elems = (size_t)n * ho * wo * p.c_out;
     L.kp = kp;
     L.smem = smem;
-    L.items = g.tiles_x * g.tiles_y * g.tiles_n * p.n_blocks;
+    L.items = g.tiles * p.n_blocks;
     return XGEN_OK;
+}
+
+// The launch layout of a shape.  Row tiling is taken where it covers clearly more of the pixel
+// slots than the best grid tiling (it stages more halo per pixel, so a small gain does not pay)
+// and where its larger staged tile still fits shared memory together with the copy engine's
+// boxes; otherwise grid tiling.  *rows_wanted tells the caller that row tiling was preferred
+// (whether or not it fitted), so that a planner may try again with smaller channel chunks.
+static xgen_status make_layout(const PackedHost &p, int n, int hh, int ww, bool y_aligned32, bool tma_ok, Layout &L,
+                               bool *rows_wanted = nullptr) {
+    const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
+    const Geometry grid = grid_geometry(n, ho, wo, p.stride);
+    Geometry rows;
+    const bool want = row_geometry(n, ho, wo, p.stride, rows) && rows.covered > 1.08 * grid.covered;
+    if (rows_wanted) *rows_wanted = want;
+    const xgen_status gs = layout_for(p, grid, n, hh, ww, y_aligned32, tma_ok, L);
+    if (want) {
+        Layout Lr;
+        if (layout_for(p, rows, n, hh, ww, y_aligned32, tma_ok, Lr) == XGEN_OK &&
+            (gs != XGEN_OK || Lr.kp.use_tma >= L.kp.use_tma)) {
+            L = Lr;
+            return XGEN_OK;
+        }
+    }
+    return gs;
 }
 
 // 1 KB rows of partial sums one (item, split) writes in a split run reduced inside the kernel.
@@ -1067,7 +1214,7 @@ static xgen_status prepared_launch(const xgen_patconv_packed *h, const void *x, 
         const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
         const cuuint64_t gdim[4] = {(cuuint64_t)p.c_in, (cuuint64_t)ww, (cuuint64_t)hh, (cuuint64_t)n};
         const cuuint64_t gstr[3] = {(cuuint64_t)p.c_in * xb, (cuuint64_t)ww * p.c_in * xb, (cuuint64_t)hh * ww * p.c_in * xb};
-        const cuuint32_t box[4] = {(cuuint32_t)ne.L.kp.rc, (cuuint32_t)g.tin_w, (cuuint32_t)g.tin_h, (cuuint32_t)(1 << g.ln_log)};
+        const cuuint32_t box[4] = {(cuuint32_t)ne.L.kp.rc, (cuuint32_t)g.tin_w, (cuuint32_t)g.tin_h, (cuuint32_t)(g.rows ? 1 : g.n_slots)};
         const cuuint32_t estr[4] = {1, 1, 1, 1};
         const CUtensorMapDataType dt = p.dtype == XGEN_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
                                      : (p.dtype == XGEN_F16_F32ACC ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
@@ -1135,12 +1282,13 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     int prev = 0;
     if (cudaGetDevice(&prev) != cudaSuccess) return XGEN_ERR_CUDA;
     if (prev != h->device && cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
-    dim3 grid((unsigned)(L.g.tiles_x * L.g.tiles_y * L.g.tiles_n), (unsigned)p.n_blocks, (unsigned)(split ? n_splits : 1)), block((unsigned)((p.wpc + kProducerWarps) * 32), 1, 1);
+    dim3 grid((unsigned)L.g.tiles, (unsigned)p.n_blocks, (unsigned)(split ? n_splits : 1)), block((unsigned)((p.wpc + kProducerWarps) * 32), 1, 1);
     cudaStream_t st = (cudaStream_t)stream;
     if (log_enabled())
-        fprintf(stderr, "libpatconv: grid %u x %u x %u, %u threads, %zu bytes shared, %d stages, lanes %dx%dx%d, tile in %dx%d, tma %d, cc %d, fused split %d\n",
-                grid.x, grid.y, grid.z, block.x, smem, kp.n_stages, 1 << L.g.lx_log, 1 << L.g.ly_log, 1 << L.g.ln_log,
-                L.g.tin_w, L.g.tin_h, kp.use_tma, p.cc, planned ? 1 : 0);
+        fprintf(stderr, "libpatconv: grid %u x %u x %u, %u threads, %zu bytes shared, %d stages, %s lanes %dx%dx%d, tile in %dx%d x %d slots, tma %d, cc %d, fused split %d\n",
+                grid.x, grid.y, grid.z, block.x, smem, kp.n_stages, L.g.rows ? "row tiling," : "grid tiling,",
+                L.g.rows ? L.g.bxn : 1 << L.g.lx_log, L.g.rows ? 1 : 1 << L.g.ly_log, L.g.rows ? 1 : 1 << L.g.ln_log,
+                L.g.tin_w, L.g.tin_h, L.g.n_slots, kp.use_tma, p.cc, planned ? 1 : 0);
     const void *kern = kernel_for(p);
     cudaError_t e = allow_large_smem(kern);
     if (e == cudaSuccess) {
@@ -1336,12 +1484,15 @@ xgen_status xgen_patconv_plan_info(const xgen_patconv_packed *h, int32_t n, int3
     memset(out, 0, sizeof(*out));
     out->splits = planned ? h->plan_splits : 1;
     out->chunks_per_split = planned ? h->plan_cps : p.n_chunks;
-    out->tiles = L.g.tiles_x * L.g.tiles_y * L.g.tiles_n;
+    out->tiles = L.g.tiles;
     out->filter_blocks = p.n_blocks;
     out->items = L.items;
     out->blocks = L.items * out->splits;
     out->threads_per_block = (p.wpc + kProducerWarps) * 32;
-    out->lanes_x = 1 << L.g.lx_log; out->lanes_y = 1 << L.g.ly_log; out->lanes_n = 1 << L.g.ln_log;
+    out->row_tiling = L.g.rows;
+    out->lanes_x = L.g.rows ? L.g.bxn : 1 << L.g.lx_log; out->lanes_y = L.g.rows ? 1 : 1 << L.g.ly_log;
+    out->lanes_n = L.g.rows ? 1 : 1 << L.g.ln_log;
+    out->covered = L.g.covered;
     out->pixels_per_lane = pixels_per_thread(p.stride);
     out->stages = L.kp.n_stages;
     out->uses_copy_engine = L.kp.use_tma;
@@ -1360,12 +1511,31 @@ xgen_status xgen_patconv_plan_tuned(xgen_patconv_packed *h, int32_t n, int32_t h
     const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
     if ((int64_t)n * ho * wo * p.c_out > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
     const xgen_patconv_tuning tn = tuning ? *tuning : xgen_patconv_tuning{};
+    const bool tma_ok = !tn.no_copy_engine && encode_tiled_fn() != nullptr;
     Layout L;
-    xgen_status ls = make_layout(p, n, hh, ww, true, !tn.no_copy_engine && encode_tiled_fn() != nullptr, L);
+    bool rows_wanted = false;
+    xgen_status ls = make_layout(p, n, hh, ww, true, tma_ok, L, &rows_wanted);
     if (ls != XGEN_OK) return ls;
     int prev = 0;
     if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
     xgen_status rs = XGEN_OK;
+    if (rows_wanted && !L.g.rows && p.cc > 4) {
+        // Row tiling covers more of this shape but its staged tile (one slot per block row)
+        // does not fit with the chunk size chosen at pack time: rebuild the command stream
+        // with half the channels per chunk (the kept weights are still in the handle) and
+        // upload it again.  Every later run of the handle uses the new layout.
+        if (cudaDeviceSynchronize() != cudaSuccess) rs = XGEN_ERR_CUDA;
+        if (rs == XGEN_OK) {
+            try {
+                rs = build_layout(h->host, PackConfig{p.J, p.wpc, p.cc / 2});
+            } catch (const std::bad_alloc &) {
+                rs = XGEN_ERR_ALLOC;
+            }
+        }
+        if (rs == XGEN_OK) rs = upload_layout(h);
+        if (rs == XGEN_OK) rs = make_layout(p, n, hh, ww, true, tma_ok, L);
+        if (rs != XGEN_OK) { cudaSetDevice(prev); h->plan_splits = 1; h->plan_n = 0; forget_prepared_launches(h); return rs; }
+    }
     int sms = 148, bps = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
     const void *kern = kernel_for(p);

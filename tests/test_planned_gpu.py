@@ -92,6 +92,37 @@ def test_sweep_every_point_planned(lib):
         _sampled_batch_planned(spec, [0] if spec.n == 1 else [0, spec.n - 1])
 
 
+@pytest.mark.parametrize("dtype", ["f32", "f16", "i8"])
+@pytest.mark.parametrize("case", [
+    (3, 28, 28, 1, True),      # 7 x 7 blocks per image: 147 blocks, 4.6 tiles; tiles straddle images
+    (5, 30, 27, 1, True),      # ragged: blocks hang over the right and the bottom edge
+    (9, 20, 12, 1, True),      # 3 blocks per row: a tile touches up to 11 block rows
+    (2, 56, 56, 1, False),     # 14 blocks per row: the staged slots may not fit; any tiling must be right
+    (4, 56, 56, 2, False),     # stride 2: 14 x 7 blocks of 2 x 4 pixels
+    (7, 26, 30, 2, False),
+])
+def test_row_tiling(dtype, case):
+    """Shapes for which a tile is 32 consecutive pixel blocks of the row-by-row numbering over all
+    images (every block row staged as a slot of its own).  Planning the shape may rebuild the
+    command stream with smaller channel chunks so that the slots fit shared memory."""
+    n, h, w, stride, expect_rows = case
+    d = _layer(dtype, n, 48, 40, h, w, stride, prune=0.5, lib=8, seed=101 + n)
+    pk = pack(d)
+    compare(d, run_gpu(pk, d.x, d.bias, True))               # as packed, whatever tiling fits
+    pk.plan(n, h, w, splits=1)
+    info = pk.plan_info(n, h, w)
+    if expect_rows:
+        assert info["row_tiling"] == 1 and info["covered"] > 0.8 and info["tiles"] > 1
+        assert info["uses_copy_engine"] == 1
+    compare(d, run_gpu(pk, d.x, d.bias, True))
+    pk.plan(n, h, w, splits=2)
+    assert pk.plan_info(n, h, w)["splits"] == 2
+    compare(d, run_gpu(pk, d.x, d.bias, True))
+    pk.plan(n, h, w, splits=2, no_copy_engine=True)
+    assert pk.plan_info(n, h, w)["uses_copy_engine"] == 0
+    compare(d, run_gpu(pk, d.x, None, False), bias=None, relu=False)
+
+
 @pytest.mark.parametrize("dtype,stride", [("f32", 2), ("f16", 1), ("f16", 2), ("i8", 1), ("i8", 2)])
 def test_universal_table_other_variants(dtype, stride):
     d = _layer(dtype, 2, 24, 40, 13, 15, stride, prune=0.4, lib=4, seed=71)
