@@ -234,7 +234,9 @@ xgen_status xgen_patconv_enqueue_host(const xgen_patconv_packed *packed, const v
  * pixels do not fill the GPU with (pixel tile x filter block) work items; for
  * such a shape this call lets later xgen_patconv_run calls split the input
  * channels across thread blocks (the paper does not discuss this; it is the
- * cross-channel reduction of this implementation).  The blocks of a split write
+ * cross-channel reduction of this implementation).  Shapes with more items
+ * than the GPU holds blocks run in waves; there the items of the last, partly
+ * filled wave are split the same way, so that the wave ends sooner.  The blocks of a split write
  * their partial sums to a workspace, count themselves in, wait (with a bound in
  * time) for the others and each reduce a share, all inside the one kernel.
  * Because they wait for each other, the split count is chosen so that every
@@ -290,7 +292,9 @@ typedef struct {
     int32_t tiles;              /* pixel tiles                                                     */
     int32_t filter_blocks;      /* blocks of output channels                                       */
     int32_t items;              /* tiles x filter_blocks                                           */
-    int32_t blocks;             /* thread blocks of the launch: items x splits                     */
+    int32_t whole_items;        /* items that run as one block; the other items, numbered last,
+                                   run as `splits` blocks each                                     */
+    int32_t blocks;             /* thread blocks of the launch: whole_items + (items - whole_items) x splits */
     int32_t threads_per_block;
     int32_t row_tiling;         /* 0: a tile is a box of lanes_x x lanes_y blocks of lanes_n images;
                                    1: a tile is 32 consecutive blocks of the row-by-row numbering

@@ -55,7 +55,8 @@ class Tuning(ctypes.Structure):
 
 class PlanStats(ctypes.Structure):
     _fields_ = [("splits", ctypes.c_int32), ("chunks_per_split", ctypes.c_int32), ("tiles", ctypes.c_int32),
-                ("filter_blocks", ctypes.c_int32), ("items", ctypes.c_int32), ("blocks", ctypes.c_int32),
+                ("filter_blocks", ctypes.c_int32), ("items", ctypes.c_int32), ("whole_items", ctypes.c_int32),
+                ("blocks", ctypes.c_int32),
                 ("threads_per_block", ctypes.c_int32), ("row_tiling", ctypes.c_int32),
                 ("lanes_x", ctypes.c_int32), ("lanes_y", ctypes.c_int32),
                 ("lanes_n", ctypes.c_int32), ("pixels_per_lane", ctypes.c_int32), ("stages", ctypes.c_int32),

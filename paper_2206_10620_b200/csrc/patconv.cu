@@ -89,7 +89,13 @@ struct KParams {
     int box_bytes;                       // bytes one tensor copy delivers (the whole box, padding included)
     int *status;                         // device word: set to 1 if a bounded wait ran out
     int fold;                            // i8: keep int32 totals in a second row and fold periodically
-    int chunks_per_split;                // grid.z splits the channel chunks; 0 = no split
+    // Block numbering of a launch (one-dimensional grid): blocks 0 .. whole_items-1 each run one whole
+    // item (tile, filter block); the remaining items follow, each as n_splits blocks that take
+    // chunks_per_split channel chunks each.  A launch without splits has whole_items = all items.
+    int whole_items;
+    uint32_t mg_splits, mg_tiles;        // division by n_splits and by the number of tiles
+    int n_tiles;
+    int chunks_per_split;                // chunks one block of a split item takes
     uint32_t *partial;                   // split runs reduced by a second kernel: [split][n*ho*wo*c_out] raw sums
     size_t out_elems;                    // n*ho*wo*c_out
     // Split runs reduced inside this kernel: every block writes its raw sums as rows of
@@ -266,9 +272,15 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     const int nthreads = blockDim.x;
     const bool producer = warp >= P.wpc;
     const int pw = warp - P.wpc;                     // producer warp number
-    const int b = blockIdx.y;
-    const int item = (int)(blockIdx.x + gridDim.x * blockIdx.y);   // (tile, filter block)
-    const int tile = blockIdx.x;
+    // block -> (item, split); item -> (tile, block of output channels)
+    const int blk = (int)blockIdx.x;
+    const bool split_item = blk >= P.whole_items;
+    const int tail = blk - P.whole_items;
+    const int item = split_item ? P.whole_items + div_by(tail, P.mg_splits) : blk;
+    const int zsplit = split_item ? tail - (item - P.whole_items) * P.n_splits : 0;
+    const int sitem = item - P.whole_items;          // number of the item among the split ones
+    const int b = div_by(item, P.mg_tiles);          // block of output channels
+    const int tile = item - b * P.n_tiles;
     // grid tiling: tile -> (tx, ty, first image)
     const int tile_r = div_by(tile, P.mg_tiles_x);
     const int tx = tile - tile_r * P.tiles_x;
@@ -321,8 +333,10 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     auto bar_raw = [&](int r) { return mbar0 + 8u * (uint32_t)(3 * NS + r); };  // a tile box landed
     auto bar_rawfree = [&](int r) { return mbar0 + 8u * (uint32_t)(3 * NS + kRawStages + r); };   // every producer warp done with a box
 
-    const int c_begin = P.chunks_per_split ? (int)blockIdx.z * P.chunks_per_split : 0;
-    const int c_end = P.chunks_per_split ? min(P.n_chunks, c_begin + P.chunks_per_split) : P.n_chunks;
+    const int c_begin = split_item ? zsplit * P.chunks_per_split : 0;
+    const int c_end = split_item ? min(P.n_chunks, c_begin + P.chunks_per_split) : P.n_chunks;
+    uint32_t *const ws_rows = split_item ? P.ws : nullptr;       // rows of partial sums exchanged inside the kernel
+    uint32_t *const part_sums = split_item ? P.partial : nullptr; // or partial sums left to a second kernel
 
     // Launched with programmatic stream serialisation: the next kernel of the stream may be
     // scheduled as soon as SMs free up (its launch latency then overlaps this kernel's tail);
@@ -393,7 +407,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         for (int k = 0; k < NS && c_begin + k < c_end; ++k)
             issue_commands(k, __ldg(seg_g + k * (P.wpc + 1)), __ldg(seg_g + k * (P.wpc + 1) + P.wpc));
     // Global reads of the tables below, started before the index arithmetic they do not need.
-    const int soc_v = tid < P.wpc * P.J ? __ldg(P.slot_oc + (size_t)blockIdx.y * P.wpc * P.J + tid) : -1;
+    const int soc_v = tid < P.wpc * P.J ? __ldg(P.slot_oc + (size_t)b * P.wpc * P.J + tid) : -1;
     const int n_seg = (c_end - c_begin) * (P.wpc + 1);
     const int seg_v = tid < n_seg ? __ldg(seg_g + tid) : 0;
 
@@ -629,9 +643,9 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         const int oc_base = soc[0];
         if (oc_base >= 0) {
             const int *pt = ptab + lane;
-            uint32_t *const part = P.partial ? P.partial + (size_t)blockIdx.z * P.out_elems : nullptr;
+            uint32_t *const part = part_sums ? part_sums + (size_t)zsplit * P.out_elems : nullptr;
             const int K8 = (P.J + 7) >> 3;
-            uint32_t *const wrow = P.ws ? P.ws + ((((size_t)item * P.n_splits + blockIdx.z) * (size_t)(P.wpc * K8 * T)
+            uint32_t *const wrow = ws_rows ? ws_rows + ((((size_t)sitem * P.n_splits + zsplit) * (size_t)(P.wpc * K8 * T)
                                                    + (size_t)warp * K8 * T) * 32 + lane) * 8 : nullptr;
             for (int j0 = 0; j0 < P.J; j0 += 8) {
                 const int oc0 = oc_base + j0;
@@ -669,13 +683,13 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         }
     }
 
-    if (P.ws) {
-        // ===== split run: wait for the other splits of this item, then reduce a share =====
+    if (ws_rows) {
+        // ===== split item: wait for the other splits of this item, then reduce a share =====
         asm volatile("griddepcontrol.wait;" ::: "memory");       // the producer warps join in here
         __threadfence();
         __syncthreads();
         if (tid == 0) {
-            uint32_t *cnt = P.counters + item;
+            uint32_t *cnt = P.counters + sitem;
             asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(cnt) : "memory");
             bool ok = false;
             uint64_t t0 = 0;
@@ -696,8 +710,8 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         if (!abort_s) {
             const int K8 = (P.J + 7) >> 3;
             const int R = P.wpc * K8 * T, S = P.n_splits, nwarps = nthreads >> 5;
-            const uint32_t *base = P.ws + (size_t)item * S * R * 256;
-            for (int row = (int)blockIdx.z + S * warp; row < R; row += S * nwarps) {
+            const uint32_t *base = ws_rows + (size_t)sitem * S * R * 256;
+            for (int row = zsplit + S * warp; row < R; row += S * nwarps) {
                 const int t = row % T, k8 = (row / T) % K8, w = row / (T * K8);
                 const int ocb = soc_s[w * P.J];
                 const int oc0 = ocb + k8 * 8;
@@ -947,6 +961,7 @@ struct xgen_patconv_packed {
     int32_t *d_slot_oc = nullptr;
     // set by xgen_patconv_plan: split the channel chunks of this shape across blocks
     int plan_n = 0, plan_h = 0, plan_w = 0, plan_splits = 1, plan_cps = 0;
+    int plan_whole = 0;                 // items of the planned shape that run whole (the others are split)
     uint32_t *d_partial = nullptr;      // partial sums of the planned split, reduced inside the kernel
     size_t partial_bytes = 0;
     uint32_t *d_counters = nullptr;     // one arrival counter per (tile, filter block) of the planned shape
@@ -1274,19 +1289,28 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     const bool planned = !forced && h->plan_splits > 1 && h->plan_n == n && h->plan_h == hh && h->plan_w == ww &&
                          h->d_partial && h->d_counters;
     const bool split = forced ? forced->splits > 1 : planned;
-    const int n_splits = forced ? forced->splits : h->plan_splits;
-    kp.chunks_per_split = split ? (forced ? forced->chunks_per_split : h->plan_cps) : 0;
+    const int n_splits = split ? (forced ? forced->splits : h->plan_splits) : 1;
+    // block numbering: whole items first, then the split items, n_splits blocks each
+    const int whole = split ? (forced ? 0 : h->plan_whole) : L.items;
+    const int64_t n_blocks_launch = (int64_t)whole + (int64_t)(L.items - whole) * n_splits;
+    if (n_blocks_launch > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
+    auto magic = [](int d) { return d <= 1 ? 0u : (uint32_t)((1ull << 32) / (uint64_t)d + 1ull); };
+    kp.whole_items = whole;
+    kp.n_splits = n_splits;
+    kp.mg_splits = magic(n_splits);
+    kp.n_tiles = L.g.tiles;
+    kp.mg_tiles = magic(L.g.tiles);
+    kp.chunks_per_split = split ? (forced ? forced->chunks_per_split : h->plan_cps) : p.n_chunks;
     kp.partial = (split && forced) ? forced->partial : nullptr;
-    kp.n_splits = split ? n_splits : 1;
 
     int prev = 0;
     if (cudaGetDevice(&prev) != cudaSuccess) return XGEN_ERR_CUDA;
     if (prev != h->device && cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
-    dim3 grid((unsigned)L.g.tiles, (unsigned)p.n_blocks, (unsigned)(split ? n_splits : 1)), block((unsigned)((p.wpc + kProducerWarps) * 32), 1, 1);
+    dim3 grid((unsigned)n_blocks_launch, 1, 1), block((unsigned)((p.wpc + kProducerWarps) * 32), 1, 1);
     cudaStream_t st = (cudaStream_t)stream;
     if (log_enabled())
-        fprintf(stderr, "libpatconv: grid %u x %u x %u, %u threads, %zu bytes shared, %d stages, %s lanes %dx%dx%d, tile in %dx%d x %d slots, tma %d, cc %d, fused split %d\n",
-                grid.x, grid.y, grid.z, block.x, smem, kp.n_stages, L.g.rows ? "row tiling," : "grid tiling,",
+        fprintf(stderr, "libpatconv: %u blocks = %d whole items + %d items x %d splits (%d tiles x %d filter blocks), %u threads, %zu bytes shared, %d stages, %s lanes %dx%dx%d, tile in %dx%d x %d slots, tma %d, cc %d, fused split %d\n",
+                grid.x, whole, L.items - whole, n_splits, L.g.tiles, p.n_blocks, block.x, smem, kp.n_stages, L.g.rows ? "row tiling," : "grid tiling,",
                 L.g.rows ? L.g.bxn : 1 << L.g.lx_log, L.g.rows ? 1 : 1 << L.g.ly_log, L.g.rows ? 1 : 1 << L.g.ln_log,
                 L.g.tin_w, L.g.tin_h, L.g.n_slots, kp.use_tma, p.cc, planned ? 1 : 0);
     const void *kern = kernel_for(p);
@@ -1487,7 +1511,8 @@ xgen_status xgen_patconv_plan_info(const xgen_patconv_packed *h, int32_t n, int3
     out->tiles = L.g.tiles;
     out->filter_blocks = p.n_blocks;
     out->items = L.items;
-    out->blocks = L.items * out->splits;
+    out->whole_items = planned ? h->plan_whole : L.items;
+    out->blocks = out->whole_items + (L.items - out->whole_items) * out->splits;
     out->threads_per_block = (p.wpc + kProducerWarps) * 32;
     out->row_tiling = L.g.rows;
     out->lanes_x = L.g.rows ? L.g.bxn : 1 << L.g.lx_log; out->lanes_y = L.g.rows ? 1 : 1 << L.g.ly_log;
@@ -1497,7 +1522,7 @@ xgen_status xgen_patconv_plan_info(const xgen_patconv_packed *h, int32_t n, int3
     out->stages = L.kp.n_stages;
     out->uses_copy_engine = L.kp.use_tma;
     out->shared_bytes = (int64_t)L.smem;
-    out->workspace_bytes = planned ? (int64_t)((size_t)L.items * (size_t)h->plan_splits * rows_per_item(p) * 1024) : 0;
+    out->workspace_bytes = planned ? (int64_t)((size_t)(L.items - h->plan_whole) * (size_t)h->plan_splits * rows_per_item(p) * 1024) : 0;
     return XGEN_OK;
 }
 
@@ -1545,38 +1570,61 @@ xgen_status xgen_patconv_plan_tuned(xgen_patconv_packed *h, int32_t n, int32_t h
         rs = XGEN_ERR_CUDA;
     }
     bps = std::min(bps, 512 / L.kp.tmem_cols);
-    // The splits of an item wait for each other inside the kernel, so every block of the
-    // launch must be resident at once: items x splits <= SMs x blocks per SM.  Within that,
-    // pick the split count with a small cost model (cycles): a block costs a fixed prologue
-    // and epilogue plus its multiply-adds at the rate an SM sustains with the warps it then
-    // hosts; a split run adds the exchange of the partial sums.
-    const int64_t capacity = (int64_t)sms * bps;
-    const int64_t max_splits = std::max<int64_t>(1, std::min<int64_t>(p.n_chunks, L.items > 0 ? capacity / L.items : 1));
+    // The splits of an item wait for each other inside the kernel, so all blocks of split items
+    // must be resident at once: (split items) x splits <= SMs x blocks per SM.  Two cases.
+    // Few items (not more than the GPU holds blocks): every item is split, and the split count
+    // comes from a small cost model (cycles): a block costs a fixed prologue and epilogue plus
+    // its multiply-adds at the rate an SM sustains with the warps it then hosts; a split adds
+    // the exchange of the partial sums.  Many items: the GPU works through them in waves of
+    // `capacity` blocks, and the last wave is only partly filled; the items of that last wave
+    // are split (they are numbered last, so their blocks start as the wave before them drains),
+    // all earlier items run whole.
+    const int64_t capacity = std::max<int64_t>(1, (int64_t)sms * bps);
     const double slot_macs_item = 4.0 * (double)p.stats.kernels_surviving / (double)p.n_blocks * 32.0 * pixels_per_thread(p.stride);
     auto sm_rate = [&](int warps) { return 50.0 * std::pow((double)std::min(warps, 16) / 16.0, 0.65); };   // multiply-adds per cycle
-    auto estimate = [&](int64_t k) {
-        const int cps_k = (int)((p.n_chunks + k - 1) / k);
-        const int64_t parts = (p.n_chunks + cps_k - 1) / cps_k;
-        const int64_t blocks = L.items * parts;
-        const int per_sm = (int)((blocks + sms - 1) / sms);
-        const double work = slot_macs_item * (double)cps_k / (double)p.n_chunks;
-        double t = 9000.0 + work * per_sm / sm_rate(per_sm * p.wpc);
-        if (parts > 1) t += 5000.0 + 150.0 * (double)parts;
-        return t;
-    };
-    int64_t splits = 1;
-    double best_t = estimate(1);
-    for (int64_t k = 2; k <= max_splits; ++k) {
-        const double t = estimate(k);
-        if (t < 0.97 * best_t) { best_t = t; splits = k; }
+    int64_t splits = 1, whole = L.items;
+    if (L.items <= capacity) {
+        const int64_t max_splits = std::max<int64_t>(1, std::min<int64_t>(p.n_chunks, capacity / std::max(1, L.items)));
+        auto estimate = [&](int64_t k) {
+            const int cps_k = (int)((p.n_chunks + k - 1) / k);
+            const int64_t parts = (p.n_chunks + cps_k - 1) / cps_k;
+            const int64_t blocks = L.items * parts;
+            const int per_sm = (int)((blocks + sms - 1) / sms);
+            const double work = slot_macs_item * (double)cps_k / (double)p.n_chunks;
+            double t = 9000.0 + work * per_sm / sm_rate(per_sm * p.wpc);
+            if (parts > 1) t += 5000.0 + 150.0 * (double)parts;
+            return t;
+        };
+        double best_t = estimate(1);
+        for (int64_t k = 2; k <= max_splits; ++k) {
+            const double t = estimate(k);
+            if (t < 0.97 * best_t) { best_t = t; splits = k; }
+        }
+        if (tn.splits >= 1) splits = std::min<int64_t>(tn.splits, max_splits);
+        whole = 0;
+    } else {
+        const int64_t rest = L.items % capacity;               // items of the last, partly filled wave
+        const int64_t max_splits = rest > 0 ? std::min<int64_t>(p.n_chunks, capacity / rest) : 1;
+        const double t_item = 9000.0 + slot_macs_item / sm_rate(bps * p.wpc);
+        double best_t = t_item;                                  // the last wave with whole items
+        for (int64_t k = 2; k <= max_splits; ++k) {
+            const int cps_k = (int)((p.n_chunks + k - 1) / k);
+            const int64_t parts = (p.n_chunks + cps_k - 1) / cps_k;
+            const double t = 9000.0 + slot_macs_item * (double)cps_k / (double)p.n_chunks / sm_rate(bps * p.wpc) +
+                             5000.0 + 150.0 * (double)parts;
+            if (t < 0.9 * best_t) { best_t = t; splits = k; }
+        }
+        if (tn.splits >= 1) splits = std::max<int64_t>(1, std::min<int64_t>(tn.splits, max_splits));
+        whole = splits > 1 ? L.items - rest : L.items;
     }
-    if (tn.splits >= 1) splits = std::min<int64_t>(tn.splits, max_splits);
     const int cps = (int)((p.n_chunks + splits - 1) / splits);
     splits = (p.n_chunks + cps - 1) / cps;
+    if (splits <= 1) whole = L.items;
+    const int64_t split_items = L.items - whole;
     if (rs == XGEN_OK && cudaDeviceSynchronize() != cudaSuccess) rs = XGEN_ERR_CUDA;
     if (rs == XGEN_OK && splits > 1) {
-        const size_t need = (size_t)L.items * (size_t)splits * rows_per_item(p) * 1024;
-        const size_t need_c = (size_t)L.items * sizeof(uint32_t);
+        const size_t need = (size_t)split_items * (size_t)splits * rows_per_item(p) * 1024;
+        const size_t need_c = (size_t)split_items * sizeof(uint32_t);
         if (need > h->partial_bytes) {
             if (h->d_partial) cudaFree(h->d_partial);
             h->d_partial = nullptr; h->partial_bytes = 0;
@@ -1601,7 +1649,7 @@ xgen_status xgen_patconv_plan_tuned(xgen_patconv_packed *h, int32_t n, int32_t h
     h->tuning = tn;
     h->wait_us = tn.wait_limit_ms > 0 ? (uint32_t)std::min<int64_t>((int64_t)tn.wait_limit_ms * 1000, 60000000) : 2000000u;
     h->plan_n = n; h->plan_h = hh; h->plan_w = ww;
-    h->plan_splits = (int)splits; h->plan_cps = cps;
+    h->plan_splits = (int)splits; h->plan_cps = cps; h->plan_whole = (int)whole;
     return XGEN_OK;
 }
 

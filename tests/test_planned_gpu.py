@@ -26,7 +26,7 @@ def test_vgg16_planned_every_layer_every_element():
         pk = pack(d)
         y = run_gpu(pk, d.x, d.bias, True, plan=True)
         info = pk.plan_info(spec.n, spec.h, spec.w)
-        assert info["blocks"] == info["items"] * info["splits"]
+        assert info["blocks"] == info["whole_items"] + (info["items"] - info["whole_items"]) * info["splits"]
         if info["splits"] > 1:
             split_layers += 1
             most_items = max(most_items, info["items"])
@@ -49,6 +49,25 @@ def test_planned_split_over_several_tiles_and_filter_blocks(dtype, stride):
     y2 = run_gpu(pk, d.x, None, False)
     compare(d, y2, bias=None, relu=False)
     assert np.array_equal(run_gpu(pk, d.x, d.bias, True), y)        # fixed reduction order
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "i8"])
+def test_last_wave_is_split(dtype):
+    """More items than the GPU holds blocks: the items of the last, partly filled wave are split
+    (and reduced inside the kernel), all earlier items run whole -- in one launch."""
+    d = _layer(dtype, 60, 32, 16, 40, 40, 1, prune=0.5, lib=8, seed=111)
+    pk = pack(d)
+    pk.plan(60, 40, 40, splits=2)
+    info = pk.plan_info(60, 40, 40)
+    assert 150 < info["items"] < 220             # 188 tiles of 32 blocks (row tiling) x 1 filter block
+    if info["splits"] == 2:                      # a GPU with 148 block slots: 148 whole + 40 x 2
+        assert 0 < info["whole_items"] < info["items"]
+        assert info["blocks"] == info["whole_items"] + (info["items"] - info["whole_items"]) * 2
+    before = binding.launch_count()
+    y = run_gpu(pk, d.x, d.bias, True)
+    assert binding.launch_count() - before == 1
+    compare(d, y)
+    assert np.array_equal(run_gpu(pk, d.x, d.bias, True), y)
 
 
 def _sampled_batch_planned(spec, images):
