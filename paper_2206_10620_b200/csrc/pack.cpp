@@ -14,6 +14,7 @@
 // register operands there is no per-tap index and no branch inside a kernel.
 #include <algorithm>
 #include <array>
+#include <cmath>
 #include <cstring>
 #include <numeric>
 
@@ -61,23 +62,25 @@ static float half_bits_to_float(uint16_t h) {
     return f;
 }
 
-PackConfig choose_pack_config(int c_in, int c_out, xgen_dtype dtype, int stride) {
+PackConfig choose_pack_config(int c_in, int c_out, xgen_dtype dtype, int stride, bool int_totals) {
     PackConfig c;
     c.channels_per_chunk = c_in <= 4 ? 4 : 8;
     // A warp's running sums take J x (pixels per thread) tensor-memory columns, and an SM
-    // has 4 x 512 of them: 128 columns per warp lets 16 warps share an SM.  Long integer
-    // layers keep a second row per filter (int32 totals), so they group half as many.
-    const int n_chunks = (c_in + c.channels_per_chunk - 1) / c.channels_per_chunk;
-    const bool fold = dtype == XGEN_I8_I32 && n_chunks > 16777216 / (c.channels_per_chunk * 4 * 32640);
+    // has 4 x 512 of them: 128 columns per warp lets 16 warps share an SM.  Integer layers
+    // whose exact fp32 partial sums could leave the 24-bit range keep a second row per
+    // filter (int32 totals), so they group half as many.
+    (void)dtype;
     c.filters_per_group = 128 / pix_per_thread(stride);
-    if (fold && stride == 2) c.filters_per_group /= 2;
+    if (int_totals && stride == 2) c.filters_per_group /= 2;
+    // Stride 2 groups 16 filters per warp; a layer with fewer than 16 such groups would leave
+    // warp slots of its thread block empty, so it groups 8 and runs twice as many warps.
+    if (stride == 2 && !int_totals && (c_out + 15) / 16 < 16) c.filters_per_group = 8;
     int groups = (c_out + c.filters_per_group - 1) / c.filters_per_group;
-    c.groups_per_block = std::min(groups, fold && stride == 1 ? 8 : 16);
+    c.groups_per_block = std::min(groups, int_totals && stride == 1 ? 8 : 16);
     return c;
 }
 
-xgen_status pack_host(const xgen_patconv_desc &d, const void *dense_w, const int16_t *pid_in,
-                      const PackConfig &cfg, PackedHost &out) {
+xgen_status parse_layer(const xgen_patconv_desc &d, const void *dense_w, const int16_t *pid_in, PackedHost &out) {
     const int16_t *pid = pid_in;
     if (!dense_w || !pid || !d.pattern_masks) return XGEN_ERR_INVALID_ARG;
     if (d.c_in < 1 || d.c_out < 1) return XGEN_ERR_INVALID_ARG;
@@ -145,7 +148,32 @@ xgen_status pack_host(const xgen_patconv_desc &d, const void *dense_w, const int
     }
     out.stats.kernels_total = (int64_t)cin * cout;
     out.stats.kernels_surviving = k_surv;
-    return build_layout(out, cfg);
+    // Integer layers run on exact fp32 FMAs: a sum of u8 x s8 products is exact while its
+    // magnitude stays below 2^24, and no partial sum of a filter can exceed 255 x (sum of the
+    // magnitudes of its kept weights).  Only if some filter can exceed that are int32 totals
+    // kept beside the fp32 sums (and the fp32 sums folded into them in time).
+    out.int_totals = false;
+    if (d.dtype == XGEN_I8_I32) {
+        for (int oc = 0; oc < cout && !out.int_totals; ++oc) {
+            double sum_abs = 0.0;
+            for (int ic = 0; ic < cin; ++ic) {
+                if (out.kpat[(size_t)oc * cin + ic] < 0) continue;
+                for (int k = 0; k < 4; ++k) {
+                    float f;
+                    std::memcpy(&f, &out.kw4[((size_t)oc * cin + ic) * 4 + k], 4);
+                    sum_abs += std::fabs((double)f);
+                }
+            }
+            if (255.0 * sum_abs >= 16777216.0) out.int_totals = true;
+        }
+    }
+    return XGEN_OK;
+}
+
+xgen_status pack_host(const xgen_patconv_desc &d, const void *dense_w, const int16_t *pid_in,
+                      const PackConfig &cfg, PackedHost &out) {
+    const xgen_status st = parse_layer(d, dense_w, pid_in, out);
+    return st == XGEN_OK ? build_layout(out, cfg) : st;
 }
 
 xgen_status build_layout(PackedHost &out, const PackConfig &cfg) {

@@ -1128,7 +1128,7 @@ static xgen_status layout_for(const PackedHost &p, const Geometry &g_in, int n, 
     const int T = pixels_per_thread(p.stride);
     kp.flush_chunks = 16777216 / (p.cc * 4 * 32640);
     if (kp.flush_chunks < 1) return XGEN_ERR_UNSUPPORTED;
-    kp.fold = (is_i8 && p.n_chunks > kp.flush_chunks) ? 1 : 0;
+    kp.fold = (is_i8 && p.int_totals) ? 1 : 0;
     kp.cols_per_warp = p.J * T * (kp.fold ? 2 : 1);
     kp.tmem_cols = next_pow2(((p.wpc + 3) / 4) * kp.cols_per_warp);
     if (kp.tmem_cols > 512) return XGEN_ERR_UNSUPPORTED;
@@ -1406,9 +1406,13 @@ xgen_status xgen_patconv_pack(const xgen_patconv_desc *desc, const void *dense_w
     if (!h) return XGEN_ERR_ALLOC;
     xgen_status st;
     try {
-        PackConfig cfg = choose_pack_config(desc->c_in, desc->c_out, desc->dtype, desc->stride);
-        if (desc->dtype == XGEN_I8_I32 && cfg.channels_per_chunk < 4) cfg.channels_per_chunk = 4;
-        st = pack_host(*desc, dense_w_host, pattern_id_host, cfg, h->host);
+        st = parse_layer(*desc, dense_w_host, pattern_id_host, h->host);
+        PackConfig cfg{};
+        if (st == XGEN_OK) {
+            cfg = choose_pack_config(desc->c_in, desc->c_out, desc->dtype, desc->stride, h->host.int_totals);
+            if (desc->dtype == XGEN_I8_I32 && cfg.channels_per_chunk < 4) cfg.channels_per_chunk = 4;
+            st = build_layout(h->host, cfg);
+        }
         // A stage of the kernel's pipeline holds the commands of one chunk for the whole
         // block: halve the chunk until the longest segment fits the command buffer.
         while (st == XGEN_OK && cfg.channels_per_chunk > 4 &&

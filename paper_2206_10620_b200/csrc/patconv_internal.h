@@ -44,11 +44,15 @@ struct PackedHost {
     std::vector<uint16_t> masks;                  // [np]
     std::vector<int16_t> kpat;                    // [c_out * c_in] compiled pattern id, -1 = removed
     std::vector<uint32_t> kw4;                    // [c_out * c_in * 4] kept weights as fp32 bits
+    bool int_totals = false;                      // i8: some filter's exact fp32 sums could leave the 24-bit range
     xgen_patconv_stats stats{};
 };
 
-// Default grouping for a layer shape.
-PackConfig choose_pack_config(int c_in, int c_out, xgen_dtype dtype, int stride);
+// Default grouping for a layer shape (int_totals: see PackedHost).
+PackConfig choose_pack_config(int c_in, int c_out, xgen_dtype dtype, int stride, bool int_totals);
+
+// Validate the description and keep the surviving kernels (pattern ids, kept weights).  No CUDA call.
+xgen_status parse_layer(const xgen_patconv_desc &desc, const void *dense_w, const int16_t *pid, PackedHost &out);
 
 // Validate the description and build the host image.  No CUDA call.
 xgen_status pack_host(const xgen_patconv_desc &desc, const void *dense_w, const int16_t *pid,
