@@ -45,6 +45,10 @@ def _load():
         lib.patconv_ref_i64.argtypes = [P, P, P, P, I, P, I, I, I, I, I, I, I, P]
         lib.patconv_ref_i64.restype = I
         lib.patconv_ref_threads.restype = I
+        lib.patconv_ref_fused_f64.argtypes = [P, P, I, I, I, I, I, I, P]
+        lib.patconv_ref_fused_f64.restype = I
+        lib.patconv_ref_fused_i64.argtypes = [P, P, I, I, I, I, I, I, P, I, P, P]
+        lib.patconv_ref_fused_i64.restype = I
         _lib = lib
     return _lib
 
@@ -108,3 +112,42 @@ def conv(x, w, pid, masks, bias=None, relu=False, stride=1, with_scale=False):
     if rc:
         raise ValueError("oracle error %d" % rc)
     return (y, s) if with_scale else y
+
+
+def conv_fused(x, w, pid, masks, bias=None, relu=False, stride=1, residual=None, pool=0,
+               requant_scale=None, zero_point=0):
+    """The layer followed by the operators fused behind it (paper Sec. 2.2): an optional
+    element-wise addition of `residual` (shaped like the convolution's output), the optional
+    ReLU, an optional 2x2 max-pool of stride 2 and, for the integer layer, an optional
+    re-quantisation to uint8 with one fp32 scale per output channel.  The convolution is
+    `conv` (its own pins apply); the operators behind it are plain loops in patconv_ref.c.
+    Returns float64 (int64; uint8 when re-quantised)."""
+    lib = _load()
+    pre = conv(x, w, pid, masks, bias=bias, relu=False, stride=stride)
+    n, ho, wo, c = pre.shape
+    step = 2 if pool == 2 else 1
+    if pool not in (0, 2):
+        raise ValueError("pool must be 0 or 2")
+    oshape = (n, ho // step, wo // step, c)
+    if pre.dtype == np.int64:
+        rc_ = None if residual is None else np.ascontiguousarray(residual, dtype=np.int32)
+        if rc_ is not None and rc_.shape != pre.shape:
+            raise ValueError("residual must be shaped like the convolution's output")
+        sc = None if requant_scale is None else np.ascontiguousarray(requant_scale, dtype=np.float32)
+        out_i = np.empty(oshape, dtype=np.int64) if sc is None else None
+        out_u = np.empty(oshape, dtype=np.uint8) if sc is not None else None
+        rc = lib.patconv_ref_fused_i64(_ptr(pre), _ptr(rc_), int(bool(relu)), int(pool), n, ho, wo, c,
+                                       _ptr(sc), int(zero_point), _ptr(out_i), _ptr(out_u))
+        if rc:
+            raise ValueError("oracle error %d" % rc)
+        return out_i if sc is None else out_u
+    if requant_scale is not None:
+        raise ValueError("re-quantisation belongs to the integer layer")
+    rc_ = None if residual is None else np.ascontiguousarray(residual, dtype=np.float64)
+    if rc_ is not None and rc_.shape != pre.shape:
+        raise ValueError("residual must be shaped like the convolution's output")
+    out = np.empty(oshape, dtype=np.float64)
+    rc = lib.patconv_ref_fused_f64(_ptr(pre), _ptr(rc_), int(bool(relu)), int(pool), n, ho, wo, c, _ptr(out))
+    if rc:
+        raise ValueError("oracle error %d" % rc)
+    return out

@@ -158,3 +158,92 @@ int patconv_ref_i64(const uint8_t *x, const int8_t *wt, const int16_t *pid, cons
     free(wm);
     return 0;
 }
+
+/*
+ * Operators fused behind the convolution (paper Sec. 2.2, "universal operator fusion": the
+ * operators that follow a convolution -- an element-wise addition, the activation, a pooling, a
+ * re-quantisation -- are computed together with it, so the intermediate tensors are never
+ * written).  The fused result is by definition what the separate operators give, applied in this
+ * order to the convolution's output before any activation:
+ *
+ *   v = pre[n,oy,ox,oc] (+ residual[n,oy,ox,oc]);   v = relu ? max(v, 0) : v;
+ *   pool = 2:  out[n,qy,qx,oc] = max of v over oy in {2qy, 2qy+1}, ox in {2qx, 2qx+1}
+ *              (Ho and Wo must be even);   pool = 0: out = v.
+ *
+ * `pre` is what patconv_ref_f64 returns with relu = 0 (bias included).  Plain loops, double.
+ * Returns 0, or 2 for a bad shape.
+ */
+int patconv_ref_fused_f64(const double *pre, const double *residual, int relu, int pool,
+                          int n, int ho, int wo, int c, double *out) {
+    if (n < 0 || ho < 1 || wo < 1 || c < 1 || (pool != 0 && pool != 2)) return 2;
+    if (pool == 2 && ((ho & 1) || (wo & 1))) return 2;
+    const int step = pool == 2 ? 2 : 1;
+    const int po = ho / step, pw = wo / step;
+    for (int in = 0; in < n; ++in)
+        for (int qy = 0; qy < po; ++qy)
+            for (int qx = 0; qx < pw; ++qx)
+                for (int oc = 0; oc < c; ++oc) {
+                    double best = 0.0;
+                    int first = 1;
+                    for (int dy = 0; dy < step; ++dy)
+                        for (int dx = 0; dx < step; ++dx) {
+                            size_t i = (((size_t)in * ho + (qy * step + dy)) * wo + (qx * step + dx)) * c + oc;
+                            double v = pre[i];
+                            if (residual) v += residual[i];
+                            if (relu && v < 0.0) v = 0.0;
+                            if (first || v > best) best = v;
+                            first = 0;
+                        }
+                    out[(((size_t)in * po + qy) * pw + qx) * c + oc] = best;
+                }
+    return 0;
+}
+
+/*
+ * The same for the integer layer, followed, if scale is given, by the re-quantisation to uint8:
+ *
+ *   q = clamp( rne( (float)v * scale[oc] ) + zero_point, 0, 255 )
+ *
+ * The product is an fp32 product of the int32 value converted to fp32 (round to nearest even)
+ * and the fp32 scale; rne rounds it to the nearest integer, ties to even.  fp32 is the
+ * precision in which the device takes this decision, so the oracle takes it in fp32 too: a
+ * quantised code is an integer and has to match exactly.  v must fit int32 (returns 4 if not).
+ * out_i64 receives v (after pooling) when scale is NULL, out_u8 the codes otherwise.
+ */
+int patconv_ref_fused_i64(const int64_t *pre, const int32_t *residual, int relu, int pool,
+                          int n, int ho, int wo, int c, const float *scale, int zero_point,
+                          int64_t *out_i64, uint8_t *out_u8) {
+    if (n < 0 || ho < 1 || wo < 1 || c < 1 || (pool != 0 && pool != 2)) return 2;
+    if (pool == 2 && ((ho & 1) || (wo & 1))) return 2;
+    const int step = pool == 2 ? 2 : 1;
+    const int po = ho / step, pw = wo / step;
+    for (int in = 0; in < n; ++in)
+        for (int qy = 0; qy < po; ++qy)
+            for (int qx = 0; qx < pw; ++qx)
+                for (int oc = 0; oc < c; ++oc) {
+                    int64_t best = 0;
+                    int first = 1;
+                    for (int dy = 0; dy < step; ++dy)
+                        for (int dx = 0; dx < step; ++dx) {
+                            size_t i = (((size_t)in * ho + (qy * step + dy)) * wo + (qx * step + dx)) * c + oc;
+                            int64_t v = pre[i];
+                            if (residual) v += (int64_t)residual[i];
+                            if (relu && v < 0) v = 0;
+                            if (first || v > best) best = v;
+                            first = 0;
+                        }
+                    if (best > 2147483647LL || best < -2147483648LL) return 4;
+                    size_t o = (((size_t)in * po + qy) * pw + qx) * c + oc;
+                    if (scale) {
+                        volatile float prod = (float)(int32_t)best * scale[oc];   /* one fp32 rounding */
+                        float r = nearbyintf(prod);                               /* ties to even */
+                        double q = (double)r + (double)zero_point;
+                        if (q < 0.0) q = 0.0;
+                        if (q > 255.0) q = 255.0;
+                        out_u8[o] = (uint8_t)q;
+                    } else {
+                        out_i64[o] = best;
+                    }
+                }
+    return 0;
+}
