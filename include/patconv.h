@@ -160,6 +160,45 @@ xgen_status xgen_patconv_run(const xgen_patconv_packed *packed, const void *x_de
                              void *y_dev, void *cuda_stream);
 
 /*
+ * The operators that may be fused behind the convolution (paper Sec. 2.2, "universal
+ * operator fusion": operators that follow a convolution are computed with it, so the
+ * intermediate results never travel to memory and back).  With v the convolution's result
+ * including the bias, in this order:
+ *   residual_dev       NULL, or a tensor shaped like the convolution's own output
+ *                      [n][ho][wo][c_out] in the output's element type (fp32, fp16, int32),
+ *                      16-byte aligned: v += residual (the shortcut of a residual block)
+ *   relu               non-zero: v = max(v, 0)
+ *   pool               0, or 2: a 2x2 max-pool of stride 2 (VGG's stage ends); ho and wo must
+ *                      be even, the stored result is [n][ho/2][wo/2][c_out]
+ *   requant_scale_dev  XGEN_I8_I32 only: NULL (int32 result), or [c_out] fp32 scales, 4-byte
+ *                      aligned: the result is stored as uint8 codes
+ *                      clamp(rne(float(v) * scale[oc]) + requant_zero_point, 0, 255), where
+ *                      float(v) is the int32 value rounded to fp32, the product is one fp32
+ *                      multiplication and rne rounds to the nearest integer, ties to even
+ */
+typedef struct {
+    int32_t relu;
+    int32_t pool;
+    const void *residual_dev;
+    const float *requant_scale_dev;
+    int32_t requant_zero_point;
+} xgen_patconv_epilogue;
+
+/*
+ * xgen_patconv_run with the fused operators of *epilogue behind the convolution; `relu` of
+ * xgen_patconv_run is epilogue->relu here.  y_dev holds the stored result as described above
+ * (16-byte aligned; must overlap neither x_dev nor residual_dev).  Planned shapes (splits)
+ * are honoured as in xgen_patconv_run.
+ * Errors as xgen_patconv_run, plus INVALID_ARG (NULL epilogue, misaligned residual or scale),
+ * SHAPE (pooling an odd extent), UNSUPPORTED (pool other than 0 or 2; re-quantisation of a
+ * floating-point layer).
+ */
+xgen_status xgen_patconv_run_fused(const xgen_patconv_packed *packed, const void *x_dev, int32_t n,
+                                   int32_t h, int32_t w, const void *bias_dev,
+                                   const xgen_patconv_epilogue *epilogue, void *y_dev,
+                                   void *cuda_stream);
+
+/*
  * (The paper has no counterpart to this entry point; it exists for callers of this
  * library.)  Run the layer with its input channels split over `splits` groups of thread
  * blocks, like a shape prepared with xgen_patconv_plan, but keep the partial sums in a

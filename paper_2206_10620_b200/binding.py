@@ -26,7 +26,7 @@ EXPORTS = ["xgen_patconv_pack", "xgen_patconv_run", "xgen_patconv_run_static_scr
            "xgen_patconv_plan_tuned", "xgen_patconv_plan_info", "xgen_patconv_test_expect_arrivals",
            "xgen_patconv_out_shape", "xgen_patconv_query", "xgen_patconv_view",
            "xgen_patconv_last_status", "xgen_patconv_free", "xgen_strerror",
-           "xgen_patconv_launch_count", "xgen_patconv_probe"]
+           "xgen_patconv_launch_count", "xgen_patconv_probe", "xgen_patconv_run_fused"]
 
 
 class Desc(ctypes.Structure):
@@ -70,6 +70,11 @@ class ProbeResult(ctypes.Structure):
                 ("sm_count", ctypes.c_int32), ("sm_clock_mhz", ctypes.c_int32)]
 
 
+class Epilogue(ctypes.Structure):
+    _fields_ = [("relu", ctypes.c_int32), ("pool", ctypes.c_int32), ("residual_dev", ctypes.c_void_p),
+                ("requant_scale_dev", ctypes.c_void_p), ("requant_zero_point", ctypes.c_int32)]
+
+
 class HostView(ctypes.Structure):
     _fields_ = [("slots", ctypes.c_void_p), ("n_slots", ctypes.c_int64),
                 ("seg_off", ctypes.c_void_p), ("slot_oc", ctypes.c_void_p),
@@ -97,6 +102,7 @@ def lib():
         L.xgen_patconv_pack.argtypes = [ctypes.POINTER(Desc), P, P, ctypes.c_int, ctypes.POINTER(P)]
         L.xgen_patconv_run.argtypes = [P, P, I, I, I, P, I, P, P]
         L.xgen_patconv_run_static_scratch.argtypes = [P, P, I, I, I, P, I, P, I, P]
+        L.xgen_patconv_run_fused.argtypes = [P, P, I, I, I, P, ctypes.POINTER(Epilogue), P, P]
         L.xgen_patconv_run_host.argtypes = [P, P, I, I, I, P, I, P]
         L.xgen_patconv_enqueue_host.argtypes = [P, P, I, I, I, P, I, P, P]
         L.xgen_patconv_plan.argtypes = [P, I, I, I]
@@ -204,6 +210,14 @@ class Packed:
         """Enqueue the layer; all pointers are device addresses (ints)."""
         _check(lib().xgen_patconv_run(self._h, x_ptr, n, h, w, bias_ptr or None, int(bool(relu)),
                                       y_ptr, stream or None), "xgen_patconv_run")
+
+    def run_fused(self, x_ptr, n, h, w, bias_ptr, y_ptr, stream=0, relu=False, pool=0, residual_ptr=0,
+                  requant_scale_ptr=0, zero_point=0):
+        """xgen_patconv_run_fused: the layer with a residual addition, ReLU, a 2x2 max-pool and
+        (integer layers) a re-quantisation to uint8 fused behind it; device addresses as ints."""
+        ep = Epilogue(int(bool(relu)), int(pool), residual_ptr or None, requant_scale_ptr or None, int(zero_point))
+        _check(lib().xgen_patconv_run_fused(self._h, x_ptr, n, h, w, bias_ptr or None, ctypes.byref(ep), y_ptr,
+                                            stream or None), "xgen_patconv_run_fused")
 
     def run_static_scratch(self, x_ptr, n, h, w, bias_ptr, relu, y_ptr, splits, stream=0):
         """Like run(), with the channel chunks split `splits` ways and the partial sums kept

@@ -57,6 +57,12 @@ struct KParams {
     const uint32_t *slots; const int32_t *seg_off; const int32_t *slot_oc;
     int n, h, w, ho, wo, c_in, c_out;
     int relu;
+    // operators fused behind the convolution (all optional)
+    const void *residual;                // tensor shaped like the unpooled result, result's element type: added before the activation
+    const float *rq_scale;               // integer variant: per-channel scale of the re-quantisation to uint8, or null
+    int rq_zero;                         // its zero point
+    int pool;                            // 0, or 2 = 2x2 max-pool of stride 2
+    int po, pw;                          // extents of the stored result (ho, wo, halved when pooling)
     int J, wpc, cc, n_chunks;
     int rc;                              // channels per tile box (a multiple of cc)
     int lx_log, ly_log, ln_log;          // grid tiling: lanes along x, y and images: 2^.. each, product 32
@@ -199,36 +205,115 @@ template <int DT> __device__ __forceinline__ float load_widened(const char *p) {
     return (float)__ldg(reinterpret_cast<const unsigned char *>(p));
 }
 
-// One piece of the result: 8 adjacent output channels of one pixel.  r holds raw sums (fp32
-// bits, or int32 for the integer variant); bias and ReLU are applied here, then the piece is
-// converted and stored at element offset o of `out`.  raw = store the sums as they are (32-bit).
-template <int DT>
-__device__ __forceinline__ void store_piece(const KParams &P, const uint32_t (&rin)[8], const uint32_t (&bb)[8], int relu,
-                                            void *out, size_t o, int nv, bool raw) {
-    uint32_t r[8];
-    if (raw) {
-#pragma unroll
-        for (int k = 0; k < 8; ++k) r[k] = rin[k];
-    } else if (DT == XGEN_I8_I32) {
-#pragma unroll
-        for (int k = 0; k < 8; ++k) { int q = (int)rin[k] + (int)bb[k]; if (relu) q = max(q, 0); r[k] = (uint32_t)q; }
+// One piece of the result: 8 adjacent output channels of one pixel, as 32-bit values (fp32 bits, or
+// int32 for the integer variant).
+
+// Raw sums stored as they are (partial sums of a split run): element offset o of a 32-bit array.
+__device__ __forceinline__ void store_raw_piece(const KParams &P, const uint32_t (&r)[8], uint32_t *out, size_t o, int nv) {
+    uint32_t *dst = out + o;
+    if (nv == 8 && P.vec_out == 8) {
+        asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
+    } else if (nv == 8 && P.vec_out == 4) {
+        *reinterpret_cast<uint4 *>(dst) = make_uint4(r[0], r[1], r[2], r[3]);
+        *reinterpret_cast<uint4 *>(dst + 4) = make_uint4(r[4], r[5], r[6], r[7]);
     } else {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) { float q = __uint_as_float(rin[k]) + __uint_as_float(bb[k]); if (relu) q = fmaxf(q, 0.f); r[k] = __float_as_uint(q); }
+        for (int k = 0; k < 8; ++k) if (k < nv) dst[k] = r[k];
     }
-    if (raw || DT != XGEN_F16_F32ACC) {
-        uint32_t *dst = (uint32_t *)out + o;
-        if (nv == 8 && P.vec_out == 8) {
-            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
-        } else if (nv == 8 && P.vec_out == 4) {
-            *reinterpret_cast<uint4 *>(dst) = make_uint4(r[0], r[1], r[2], r[3]);
-            *reinterpret_cast<uint4 *>(dst + 4) = make_uint4(r[4], r[5], r[6], r[7]);
-        } else {
+}
+
+// Bias, the fused residual addition and the activation (operator fusion, Sec. 2.2), applied to the
+// raw sums of the piece at channel oc0 of unpooled pixel pidx.
+template <int DT, bool FUSED>
+__device__ __forceinline__ void finish_piece(const KParams &P, const uint32_t (&raw)[8], const uint32_t (&bb)[8],
+                                             int oc0, int nv, int pidx, uint32_t (&v)[8]) {
+    uint32_t res[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (FUSED && P.residual) {
+        const size_t o = (size_t)pidx * P.c_out + oc0;
+        if (DT == XGEN_F16_F32ACC) {
+            const __half *rp = (const __half *)P.residual + o;
+            if (nv == 8 && P.vec_out >= 4 && (P.c_out & 7) == 0) {
+                const uint4 q = __ldg(reinterpret_cast<const uint4 *>(rp));
+                const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-            for (int k = 0; k < 8; ++k) if (k < nv) dst[k] = r[k];
+                for (int k = 0; k < 4; ++k) {
+                    const __half2 hv = *reinterpret_cast<const __half2 *>(&w4[k]);
+                    res[2 * k] = __float_as_uint(__low2float(hv)); res[2 * k + 1] = __float_as_uint(__high2float(hv));
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) if (k < nv) res[k] = __float_as_uint(__half2float(rp[k]));
+            }
+        } else {
+            const uint32_t *rp = (const uint32_t *)P.residual + o;
+            if (nv == 8 && P.vec_out >= 4) {
+                const uint4 a = __ldg(reinterpret_cast<const uint4 *>(rp)), b = __ldg(reinterpret_cast<const uint4 *>(rp) + 1);
+                res[0] = a.x; res[1] = a.y; res[2] = a.z; res[3] = a.w; res[4] = b.x; res[5] = b.y; res[6] = b.z; res[7] = b.w;
+            } else {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) if (k < nv) res[k] = __ldg(rp + k);
+            }
         }
+    }
+    if (DT == XGEN_I8_I32) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { int q = (int)raw[k] + (int)bb[k] + (int)res[k]; if (P.relu) q = max(q, 0); v[k] = (uint32_t)q; }
     } else {
-        __half *dst = (__half *)out + o;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            float q = __fadd_rn(__uint_as_float(raw[k]), __uint_as_float(bb[k]));
+            if (FUSED && P.residual) q = __fadd_rn(q, __uint_as_float(res[k]));
+            if (P.relu) q = fmaxf(q, 0.f);
+            v[k] = __float_as_uint(q);
+        }
+    }
+}
+
+// Element-wise maximum of two finished pieces (max-pool).
+template <int DT>
+__device__ __forceinline__ void max_piece(uint32_t (&a)[8], const uint32_t (&b)[8]) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        if (DT == XGEN_I8_I32) a[k] = (uint32_t)max((int)a[k], (int)b[k]);
+        else a[k] = __float_as_uint(fmaxf(__uint_as_float(a[k]), __uint_as_float(b[k])));
+    }
+}
+
+// Convert a finished piece to the result's element type and store it at element offset o of y:
+// fp32 and int32 as they are, fp16 by one round-to-nearest-even, and the re-quantised integer
+// result as uint8 codes clamp(rne(float(v) * scale) + zero point, 0, 255), decided in fp32.
+// The re-quantised piece (kept out of line: it is rare, and inlined it costs the kernel registers).
+__device__ __noinline__ void emit_requantised(const float *scale, int zero, unsigned char *dst, bool vec, int nv,
+                                              uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3,
+                                              uint32_t r4, uint32_t r5, uint32_t r6, uint32_t r7) {
+    const uint32_t r[8] = {r0, r1, r2, r3, r4, r5, r6, r7};
+    uint32_t code[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const float sc = k < nv ? __ldg(scale + k) : 0.f;
+        const float t = rintf(__fmul_rn((float)(int)r[k], sc)) + (float)zero;
+        code[k] = (uint32_t)fminf(fmaxf(t, 0.f), 255.f);
+    }
+    if (vec) {
+        uint2 pk;
+        pk.x = code[0] | (code[1] << 8) | (code[2] << 16) | (code[3] << 24);
+        pk.y = code[4] | (code[5] << 8) | (code[6] << 16) | (code[7] << 24);
+        *reinterpret_cast<uint2 *>(dst) = pk;
+    } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) if (k < nv) dst[k] = (unsigned char)code[k];
+    }
+}
+
+template <int DT, bool FUSED>
+__device__ __forceinline__ void emit_piece(const KParams &P, const uint32_t (&r)[8], int oc0, size_t o, int nv) {
+    if (FUSED && DT == XGEN_I8_I32 && P.rq_scale) {
+        emit_requantised(P.rq_scale + oc0, P.rq_zero, (unsigned char *)P.y + o, nv == 8 && P.vec_out >= 4 && (P.c_out & 7) == 0, nv,
+                         r[0], r[1], r[2], r[3], r[4], r[5], r[6], r[7]);
+    } else if (DT != XGEN_F16_F32ACC) {
+        store_raw_piece(P, r, (uint32_t *)P.y, o, nv);
+    } else {
+        __half *dst = (__half *)P.y + o;
         if (nv == 8 && P.vec_out >= 4 && (P.c_out & 7) == 0) {
             uint4 pk;
             __half2 h0 = __floats2half2_rn(__uint_as_float(r[0]), __uint_as_float(r[1]));
@@ -245,6 +330,15 @@ __device__ __forceinline__ void store_piece(const KParams &P, const uint32_t (&r
     }
 }
 
+// The four running sums of a thread that one pooled pixel q covers: stride 1 keeps sum
+// 4*py + 2*h + e for pixel (py, h + 2*e) of its 4x4 block, so pooled pixel (qy, qx) = q / 2, q % 2
+// covers py in {2qy, 2qy+1}, h in {0, 1}, e = qx; stride 2 keeps sum 2*py + e of its 2x4 block.
+template <int STRIDE>
+__device__ __forceinline__ int pool_member(int q, int m) {
+    if (STRIDE == 1) return 4 * (2 * (q >> 1) + (m >> 1)) + 2 * (m & 1) + (q & 1);
+    return 4 * q + m;
+}
+
 // n / d for the small divisors of the launch geometry: m = 2^32 / d + 1 (0 stands for d = 1),
 // exact while n * d < 2^32.
 __device__ __forceinline__ int div_by(int n, uint32_t m) { return m ? (int)__umulhi((uint32_t)n, m) : n; }
@@ -257,7 +351,9 @@ struct LaneSite { int on, oy0, ox0, off; bool valid; };
 struct SlotOrigin { int gn, gy0, gx0; bool used; };
 
 // ---- the kernel -----------------------------------------------------------------
-template <int DT, int STRIDE, int NP>
+// FUSED: with the operators fused behind the convolution (residual addition, max-pool,
+// re-quantisation); the plain instances carry none of that code.
+template <int DT, int STRIDE, int NP, bool FUSED>
 __global__ void __launch_bounds__((kMaxWarps + kProducerWarps) * 32)
 patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     extern __shared__ __align__(128) uint32_t smem[];
@@ -465,6 +561,16 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         const int ox = ls.ox0 + px, oy = ls.oy0 + py, on = ls.on;
         ptab[i] = (ls.valid && on < P.n && oy < P.ho && ox < P.wo) ? (on * P.ho + oy) * P.wo + ox : -1;
     }
+    // With the fused 2x2 max-pool: linear index of pooled pixel q of lane l in the stored result
+    // (its window lies inside the image or outside it as a whole: ho and wo are even).
+    int *qtab = ptab + 32 * T;
+    for (int i = tid; FUSED && !producer && P.pool && i < 32 * (T / 4); i += cthreads) {
+        const int q = i >> 5, l2 = i & 31;
+        const LaneSite ls = lane_site(l2);
+        const int qy = STRIDE == 1 ? (q >> 1) : q, qx = STRIDE == 1 ? (q & 1) : 0;
+        const int oy = ls.oy0 + 2 * qy, ox = ls.ox0 + 2 * qx;
+        qtab[i] = (ls.valid && ls.on < P.n && oy < P.ho && ox < P.wo) ? (ls.on * P.po + (oy >> 1)) * P.pw + (ox >> 1) : -1;
+    }
     // Segment offsets of this block's chunks.
     int *seg = reinterpret_cast<int *>(smem + P.seg_off_words);
     if (!producer) {
@@ -654,6 +760,29 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                 uint32_t bb[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k) bb[k] = (P.bias && !part && !wrow && k < nv) ? ((const uint32_t *)P.bias)[oc0 + k] : 0u;
+                if (FUSED && P.pool && !part && !wrow) {
+                    // fused 2x2 max-pool: the four sums of a pooled pixel are columns of this thread
+                    for (int q = 0; q < T / 4; ++q) {
+                        const int qidx = qtab[q * 32 + lane];
+                        uint32_t best[8], u[8], f[8];
+                        for (int m = 0; m < 4; ++m) {
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                if (j0 + k < P.J)
+                                    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];"
+                                                 : "=r"(u[k]) : "r"(tmem_res + (j0 + k) * T + pool_member<STRIDE>(q, m)) : "memory");
+                                else u[k] = 0u;
+                            }
+                            tmem_wait_ld();
+                            if (qidx < 0) continue;
+                            if (m == 0) finish_piece<DT, FUSED>(P, u, bb, oc0, nv, pt[pool_member<STRIDE>(q, 0) * 32], best);
+                            else { finish_piece<DT, FUSED>(P, u, bb, oc0, nv, pt[pool_member<STRIDE>(q, m) * 32], f); max_piece<DT>(best, f); }
+                        }
+                        if (qidx < 0) continue;
+                        emit_piece<DT, FUSED>(P, best, oc0, (size_t)qidx * P.c_out + oc0, nv);
+                    }
+                    continue;
+                }
                 for (int t0 = 0; t0 < T; t0 += 4) {
                     uint32_t v[8][4];
 #pragma unroll
@@ -675,8 +804,10 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                         }
                         const int pidx = pt[(t0 + tt) * 32];
                         if (pidx < 0) continue;
-                        if (part) store_piece<XGEN_F32>(P, r, bb, false, part, (size_t)pidx * P.c_out + oc0, nv, true);
-                        else store_piece<DT>(P, r, bb, P.relu, P.y, (size_t)pidx * P.c_out + oc0, nv, false);
+                        if (part) { store_raw_piece(P, r, part, (size_t)pidx * P.c_out + oc0, nv); continue; }
+                        uint32_t f[8];
+                        finish_piece<DT, FUSED>(P, r, bb, oc0, nv, pidx, f);
+                        emit_piece<DT, FUSED>(P, f, oc0, (size_t)pidx * P.c_out + oc0, nv);
                     }
                 }
             }
@@ -711,14 +842,11 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
             const int K8 = (P.J + 7) >> 3;
             const int R = P.wpc * K8 * T, S = P.n_splits, nwarps = nthreads >> 5;
             const uint32_t *base = ws_rows + (size_t)sitem * S * R * 256;
-            for (int row = zsplit + S * warp; row < R; row += S * nwarps) {
-                const int t = row % T, k8 = (row / T) % K8, w = row / (T * K8);
-                const int ocb = soc_s[w * P.J];
-                const int oc0 = ocb + k8 * 8;
-                const int pidx = ptab[t * 32 + lane];
-                if (ocb < 0 || oc0 >= P.c_out || pidx < 0) continue;
-                const int nv = min(8, P.c_out - oc0);
-                uint32_t acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            const size_t zstride = (size_t)R * 64;                // uint4 per split
+            // the sums of row `row` (one running sum of every lane, 8 channels) over all splits, in split order
+            auto sum_row = [&](int row, uint32_t (&acc)[8]) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) acc[k] = 0u;
                 auto add8 = [&](const uint4 &lo, const uint4 &hi) {
                     const uint32_t q[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
 #pragma unroll
@@ -727,7 +855,6 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                         else acc[k] = __float_as_uint(__uint_as_float(acc[k]) + __uint_as_float(q[k]));
                     }
                 };
-                const size_t zstride = (size_t)R * 64;                // uint4 per split
                 const uint4 *src = reinterpret_cast<const uint4 *>(base + ((size_t)row * 32 + lane) * 8);
                 int z = 0;
                 for (; z + 4 <= S; z += 4) {                          // four splits in flight; summed in order 0, 1, ...
@@ -738,10 +865,45 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                     for (int u = 0; u < 4; ++u) add8(lo[u], hi[u]);
                 }
                 for (; z < S; ++z) add8(__ldcg(src + z * zstride), __ldcg(src + z * zstride + 1));
-                uint32_t bb[8];
+            };
+            if (FUSED && P.pool) {
+                // units of one pooled pixel: (warp's filter group, 8-channel piece, pooled pixel q)
+                const int Q = T / 4, U = P.wpc * K8 * Q;
+                const int *qtab = ptab + 32 * T;
+                for (int unit = zsplit + S * warp; unit < U; unit += S * nwarps) {
+                    const int q = unit % Q, k8 = (unit / Q) % K8, w = unit / (Q * K8);
+                    const int ocb = soc_s[w * P.J];
+                    const int oc0 = ocb + k8 * 8;
+                    const int qidx = qtab[q * 32 + lane];
+                    if (ocb < 0 || oc0 >= P.c_out || qidx < 0) continue;
+                    const int nv = min(8, P.c_out - oc0);
+                    uint32_t bb[8];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) bb[k] = (P.bias && k < nv) ? ((const uint32_t *)P.bias)[oc0 + k] : 0u;
-                store_piece<DT>(P, acc, bb, P.relu, P.y, (size_t)pidx * P.c_out + oc0, nv, false);
+                    for (int k = 0; k < 8; ++k) bb[k] = (P.bias && k < nv) ? ((const uint32_t *)P.bias)[oc0 + k] : 0u;
+                    uint32_t best[8], acc[8], f[8];
+                    for (int m = 0; m < 4; ++m) {
+                        const int t = pool_member<STRIDE>(q, m);
+                        sum_row((w * K8 + k8) * T + t, acc);
+                        if (m == 0) finish_piece<DT, FUSED>(P, acc, bb, oc0, nv, ptab[t * 32 + lane], best);
+                        else { finish_piece<DT, FUSED>(P, acc, bb, oc0, nv, ptab[t * 32 + lane], f); max_piece<DT>(best, f); }
+                    }
+                    emit_piece<DT, FUSED>(P, best, oc0, (size_t)qidx * P.c_out + oc0, nv);
+                }
+            } else {
+                for (int row = zsplit + S * warp; row < R; row += S * nwarps) {
+                    const int t = row % T, k8 = (row / T) % K8, w = row / (T * K8);
+                    const int ocb = soc_s[w * P.J];
+                    const int oc0 = ocb + k8 * 8;
+                    const int pidx = ptab[t * 32 + lane];
+                    if (ocb < 0 || oc0 >= P.c_out || pidx < 0) continue;
+                    const int nv = min(8, P.c_out - oc0);
+                    uint32_t acc[8], f[8], bb[8];
+                    sum_row(row, acc);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) bb[k] = (P.bias && k < nv) ? ((const uint32_t *)P.bias)[oc0 + k] : 0u;
+                    finish_piece<DT, FUSED>(P, acc, bb, oc0, nv, pidx, f);
+                    emit_piece<DT, FUSED>(P, f, oc0, (size_t)pidx * P.c_out + oc0, nv);
+                }
             }
         }
     }
@@ -1052,21 +1214,26 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-template <int DT, int STRIDE>
+template <int DT, int STRIDE, bool FUSED>
 static const void *kernel_np(int np) {
     switch (np) {
-        case 4: return (const void *)patconv_kernel<DT, STRIDE, 4>;
-        case 8: return (const void *)patconv_kernel<DT, STRIDE, 8>;
-        case 12: return (const void *)patconv_kernel<DT, STRIDE, 12>;
-        default: return (const void *)patconv_kernel<DT, STRIDE, 126>;
+        case 4: return (const void *)patconv_kernel<DT, STRIDE, 4, FUSED>;
+        case 8: return (const void *)patconv_kernel<DT, STRIDE, 8, FUSED>;
+        case 12: return (const void *)patconv_kernel<DT, STRIDE, 12, FUSED>;
+        default: return (const void *)patconv_kernel<DT, STRIDE, 126, FUSED>;
     }
 }
 
-// The kernel instance of a packed layer.
-static const void *kernel_for(const PackedHost &p) {
-    if (p.dtype == XGEN_F32) return p.stride == 1 ? kernel_np<XGEN_F32, 1>(p.np) : kernel_np<XGEN_F32, 2>(p.np);
-    if (p.dtype == XGEN_F16_F32ACC) return p.stride == 1 ? kernel_np<XGEN_F16_F32ACC, 1>(p.np) : kernel_np<XGEN_F16_F32ACC, 2>(p.np);
-    return p.stride == 1 ? kernel_np<XGEN_I8_I32, 1>(p.np) : kernel_np<XGEN_I8_I32, 2>(p.np);
+template <bool FUSED>
+static const void *kernel_of(const PackedHost &p) {
+    if (p.dtype == XGEN_F32) return p.stride == 1 ? kernel_np<XGEN_F32, 1, FUSED>(p.np) : kernel_np<XGEN_F32, 2, FUSED>(p.np);
+    if (p.dtype == XGEN_F16_F32ACC) return p.stride == 1 ? kernel_np<XGEN_F16_F32ACC, 1, FUSED>(p.np) : kernel_np<XGEN_F16_F32ACC, 2, FUSED>(p.np);
+    return p.stride == 1 ? kernel_np<XGEN_I8_I32, 1, FUSED>(p.np) : kernel_np<XGEN_I8_I32, 2, FUSED>(p.np);
+}
+
+// The kernel instance of a packed layer, without or with the fused operators.
+static const void *kernel_for(const PackedHost &p, bool fused = false) {
+    return fused ? kernel_of<true>(p) : kernel_of<false>(p);
 }
 
 // The opt-in to large dynamic shared memory is per function and per device: do it once.
@@ -1140,7 +1307,7 @@ static xgen_status layout_for(const PackedHost &p, const Geometry &g_in, int n, 
     auto smem_words = [&](int stages, int tma) {
         size_t w = (size_t)(tma ? kRawStages * ((kp.box_bytes / 4 + 31) & ~31) : 0);
         w += (size_t)stages * (kp.plane_stage_words + kp.cmd_stage_words);
-        w += 2 * (size_t)npix_box + (tma ? 0 : ((size_t)npix_box + 1) & ~(size_t)1) + 32 * (size_t)T + seg_words;
+        w += 2 * (size_t)npix_box + (tma ? 0 : ((size_t)npix_box + 1) & ~(size_t)1) + 40 * (size_t)T + seg_words;   // tables: staged pixels, output pixels (+ pooled), segments
         return w + 2 * (3 * kMaxStages + 2 * kRawStages + 2);     // + mbarriers
     };
     auto occupancy = [&](size_t words) {
@@ -1161,7 +1328,7 @@ static xgen_status layout_for(const PackedHost &p, const Geometry &g_in, int n, 
     kp.tab_off_words = kp.cmd_off_words + n_stages * kp.cmd_stage_words;
     kp.src_off_words = kp.tab_off_words + 2 * npix_box;
     kp.ptab_off_words = kp.src_off_words + (kp.use_tma ? 0 : ((npix_box + 1) & ~1));
-    kp.seg_off_words = kp.ptab_off_words + 32 * T;
+    kp.seg_off_words = kp.ptab_off_words + 40 * T;
     kp.mbar_off_words = kp.seg_off_words + (int)seg_words;
     size_t smem = smem_words(n_stages, kp.use_tma) * 4;
     // Never let more blocks share an SM than tensor memory has columns for.
@@ -1258,7 +1425,8 @@ static void forget_prepared_launches(xgen_patconv_packed *h) {
 struct SplitChoice { int splits, chunks_per_split; uint32_t *partial; };
 
 static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
-                             const void *bias, int32_t relu, void *y, void *stream, const SplitChoice *forced) {
+                             const void *bias, int32_t relu, void *y, void *stream, const SplitChoice *forced,
+                             const xgen_patconv_epilogue *ep = nullptr) {
     if (!h || !x || !y) return XGEN_ERR_INVALID_ARG;
     if (((uintptr_t)x & 15) || ((uintptr_t)y & 15) || ((uintptr_t)bias & 3)) return XGEN_ERR_INVALID_ARG;
     if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
@@ -1267,11 +1435,28 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
     if ((int64_t)n * hh * ww * p.c_in > 0x7FFFFFFFLL || (int64_t)n * ho * wo * p.c_out > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
     const int xb = p.dtype == XGEN_F32 ? 4 : (p.dtype == XGEN_F16_F32ACC ? 2 : 1);
+    // operators fused behind the convolution
+    const int pool = ep ? ep->pool : 0;
+    const void *residual = ep ? ep->residual_dev : nullptr;
+    const float *rq_scale = ep ? ep->requant_scale_dev : nullptr;
+    if (ep) {
+        if (forced) return XGEN_ERR_UNSUPPORTED;
+        if (pool != 0 && pool != 2) return XGEN_ERR_UNSUPPORTED;
+        if (pool == 2 && ((ho & 1) || (wo & 1))) return XGEN_ERR_SHAPE;
+        if (rq_scale && p.dtype != XGEN_I8_I32) return XGEN_ERR_UNSUPPORTED;
+        if (((uintptr_t)residual & 15) || ((uintptr_t)rq_scale & 3)) return XGEN_ERR_INVALID_ARG;
+        relu = ep->relu;
+    }
+    const int po = pool == 2 ? ho / 2 : ho, pw = pool == 2 ? wo / 2 : wo;
     {
-        const char *xa = (const char *)x, *ya = (const char *)y;
-        const int yb = p.dtype == XGEN_F16_F32ACC ? 2 : 4;
-        const char *xe = xa + (size_t)n * hh * ww * p.c_in * xb, *ye = ya + (size_t)n * ho * wo * p.c_out * yb;
+        const char *xa = (const char *)x, *ya = (const char *)y, *ra = (const char *)residual;
+        const int yb = rq_scale ? 1 : (p.dtype == XGEN_F16_F32ACC ? 2 : 4), rb = p.dtype == XGEN_F16_F32ACC ? 2 : 4;
+        const char *xe = xa + (size_t)n * hh * ww * p.c_in * xb, *ye = ya + (size_t)n * po * pw * p.c_out * yb;
         if (xa < ye && ya < xe) return XGEN_ERR_INVALID_ARG;   // overlap
+        if (ra) {
+            const char *re = ra + (size_t)n * ho * wo * p.c_out * rb;
+            if (ra < ye && ya < re) return XGEN_ERR_INVALID_ARG;
+        }
     }
     Layout L;
     CUtensorMap tm;
@@ -1282,6 +1467,8 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     kp.x = x; kp.y = y; kp.bias = bias;
     kp.slots = h->d_slots; kp.seg_off = h->d_seg_off; kp.slot_oc = h->d_slot_oc;
     kp.relu = relu ? 1 : 0;
+    kp.residual = residual; kp.rq_scale = rq_scale; kp.rq_zero = ep ? ep->requant_zero_point : 0;
+    kp.pool = pool; kp.po = po; kp.pw = pw;
     kp.status = h->d_status;
     kp.wait_us = h->wait_us;
     // Split runs: a caller-chosen split keeps [split][output] sums for a second kernel; the
@@ -1313,7 +1500,7 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
                 grid.x, whole, L.items - whole, n_splits, L.g.tiles, p.n_blocks, block.x, smem, kp.n_stages, L.g.rows ? "row tiling," : "grid tiling,",
                 L.g.rows ? L.g.bxn : 1 << L.g.lx_log, L.g.rows ? 1 : 1 << L.g.ly_log, L.g.rows ? 1 : 1 << L.g.ln_log,
                 L.g.tin_w, L.g.tin_h, L.g.n_slots, kp.use_tma, p.cc, planned ? 1 : 0);
-    const void *kern = kernel_for(p);
+    const void *kern = kernel_for(p, ep != nullptr);
     cudaError_t e = allow_large_smem(kern);
     if (e == cudaSuccess) {
         cudaLaunchConfig_t cfg = {};
@@ -1670,6 +1857,12 @@ xgen_status xgen_patconv_test_expect_arrivals(xgen_patconv_packed *h, int32_t ex
 xgen_status xgen_patconv_run(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
                              const void *bias, int32_t relu, void *y, void *stream) {
     return run_layer(h, x, n, hh, ww, bias, relu, y, stream, nullptr);
+}
+
+xgen_status xgen_patconv_run_fused(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh, int32_t ww,
+                                   const void *bias, const xgen_patconv_epilogue *ep, void *y, void *stream) {
+    if (!ep) return XGEN_ERR_INVALID_ARG;
+    return run_layer(h, x, n, hh, ww, bias, ep->relu, y, stream, nullptr, ep);
 }
 
 xgen_status xgen_patconv_run_static_scratch(const xgen_patconv_packed *h, const void *x, int32_t n, int32_t hh,

@@ -31,14 +31,20 @@ def guarded_output(shape, dtype):
     Returns (whole flat buffer, view of the result)."""
     import torch
     n = int(np.prod(shape))
-    buf = torch.full((n + 2 * GUARD,), SENTINEL, dtype=dtype, device="cuda")
+    buf = torch.full((n + 2 * GUARD,), _sentinel(dtype), dtype=dtype, device="cuda")
     return buf, buf[GUARD:GUARD + n].view(*shape)
+
+
+def _sentinel(dtype):
+    import torch
+    return SENTINEL % 251 if dtype == torch.uint8 else SENTINEL
 
 
 def check_guards(buf):
     g = buf.cpu().numpy()
-    assert (g[:GUARD] == SENTINEL).all(), "the kernel wrote before the start of y"
-    assert (g[-GUARD:] == SENTINEL).all(), "the kernel wrote past the end of y"
+    sentinel = _sentinel(buf.dtype)
+    assert (g[:GUARD] == sentinel).all(), "the kernel wrote before the start of y"
+    assert (g[-GUARD:] == sentinel).all(), "the kernel wrote past the end of y"
 
 
 def run_gpu(pk, x, bias, relu, plan=False):
