@@ -461,6 +461,55 @@ def run_gpu(args):
             del stk
             torch.cuda.empty_cache()
 
+    # --- operators fused behind the convolution: what they save on the layers that feed a pooling
+    # (VGG-16's stage ends) and on the integer stack (uint8 codes instead of int32 sums)
+    fused = {}
+    if rank == 0 and world == 1 and not args.no_configs and args.workload == "vgg16" and not args.only:
+        def time_layers(stk, runner, reps=7):
+            out = []
+            for item in stk.layers:
+                ts = []
+                for r in range(reps):
+                    flush.fill_(r)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    runner(item)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    ts.append(e0.elapsed_time(e1))
+                out.append(float(np.median(ts)) * 1e3)
+            return out
+
+        ends = [s for s in wl.config_vgg16() if s.name in ("conv2", "conv4", "conv7", "conv10", "conv13")]
+        stk = Stack(ends, wl.BASE_SEED, local, keep_host=False)
+        plain_us = time_layers(stk, lambda it: it[2].run(it[3].data_ptr(), it[0].n, it[0].h, it[0].w, it[4].data_ptr(),
+                                                         True, it[5].data_ptr(), stream))
+        pooled = [torch.empty((s.n, s.ho // 2, s.wo // 2, s.c_out), dtype=torch.float32, device=dev) for s in ends]
+        pool_us = time_layers(stk, lambda it: it[2].run_fused(it[3].data_ptr(), it[0].n, it[0].h, it[0].w, it[4].data_ptr(),
+                                                              pooled[ends.index(it[0])].data_ptr(), stream, relu=True, pool=2))
+        fused["vgg16_stage_ends_maxpool"] = {
+            "layers": [s.name for s in ends], "plain_us": [round(t, 2) for t in plain_us],
+            "fused_pool_us": [round(t, 2) for t in pool_us],
+            "result_bytes_plain": int(sum(s.n * s.ho * s.wo * s.c_out * 4 for s in ends)),
+            "result_bytes_fused": int(sum(s.n * s.ho * s.wo * s.c_out for s in ends)),
+            "note": "the unfused network also reads the full result back and writes the pooled one"}
+        del stk, pooled
+        sp = wl.config_resnet18()
+        stk = Stack(sp, wl.BASE_SEED, local, keep_host=False)
+        plain_us = time_layers(stk, lambda it: it[2].run(it[3].data_ptr(), it[0].n, it[0].h, it[0].w, it[4].data_ptr(),
+                                                         True, it[5].data_ptr(), stream), reps=5)
+        codes = [torch.empty((s.n, s.ho, s.wo, s.c_out), dtype=torch.uint8, device=dev) for s in sp]
+        scales = [torch.full((s.c_out,), 1e-3, dtype=torch.float32, device=dev) for s in sp]
+        rq_us = time_layers(stk, lambda it: it[2].run_fused(it[3].data_ptr(), it[0].n, it[0].h, it[0].w, it[4].data_ptr(),
+                                                            codes[sp.index(it[0])].data_ptr(), stream, relu=True,
+                                                            requant_scale_ptr=scales[sp.index(it[0])].data_ptr()), reps=5)
+        fused["resnet18_requantised"] = {
+            "plain_int32_ms": round(sum(plain_us) * 1e-3, 4), "fused_uint8_ms": round(sum(rq_us) * 1e-3, 4),
+            "result_bytes_plain": int(sum(s.n * s.ho * s.wo * s.c_out * 4 for s in sp)),
+            "result_bytes_fused": int(sum(s.n * s.ho * s.wo * s.c_out for s in sp))}
+        del stk, codes, scales
+        torch.cuda.empty_cache()
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu = oracle_sample(specs, budget_s=args.cpu_seconds)
@@ -480,7 +529,7 @@ def run_gpu(args):
                 "net_ms_per_batch": ms,
                 "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e,
                 "roofline": roofline, "measured_peaks": probe, "host_us_per_run_call": round(host_us, 2),
-                "parity_checked": parity_checked, "cpu_baseline": cpu, "per_layer": per_layer, "configs": configs}
+                "parity_checked": parity_checked, "cpu_baseline": cpu, "per_layer": per_layer, "configs": configs, "fused": fused}
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

@@ -282,17 +282,18 @@ __device__ __forceinline__ void max_piece(uint32_t (&a)[8], const uint32_t (&b)[
 // Convert a finished piece to the result's element type and store it at element offset o of y:
 // fp32 and int32 as they are, fp16 by one round-to-nearest-even, and the re-quantised integer
 // result as uint8 codes clamp(rne(float(v) * scale) + zero point, 0, 255), decided in fp32.
-// The re-quantised piece (kept out of line: it is rare, and inlined it costs the kernel registers).
-__device__ __noinline__ void emit_requantised(const float *scale, int zero, unsigned char *dst, bool vec, int nv,
-                                              uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3,
-                                              uint32_t r4, uint32_t r5, uint32_t r6, uint32_t r7) {
-    const uint32_t r[8] = {r0, r1, r2, r3, r4, r5, r6, r7};
+// The re-quantised piece: codes clamp(rne(float(v) * scale) + zero point, 0, 255).  The rounding
+// to the nearest integer (ties to even) and the clamps are the conversion instructions' own:
+// float to int32 saturates, the zero point is added with saturation, int32 to uint8 saturates.
+__device__ __forceinline__ void emit_requantised(const float (&sc)[8], int zero, unsigned char *dst, bool vec, int nv,
+                                                 const uint32_t (&r)[8]) {
     uint32_t code[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-        const float sc = k < nv ? __ldg(scale + k) : 0.f;
-        const float t = rintf(__fmul_rn((float)(int)r[k], sc)) + (float)zero;
-        code[k] = (uint32_t)fminf(fmaxf(t, 0.f), 255.f);
+        const int q = __float2int_rn(__fmul_rn((float)(int)r[k], sc[k]));
+        int qz;
+        asm("add.sat.s32 %0, %1, %2;" : "=r"(qz) : "r"(q), "r"(zero));
+        asm("cvt.sat.u8.s32 %0, %1;" : "=r"(code[k]) : "r"(qz));
     }
     if (vec) {
         uint2 pk;
@@ -306,10 +307,9 @@ __device__ __noinline__ void emit_requantised(const float *scale, int zero, unsi
 }
 
 template <int DT, bool FUSED>
-__device__ __forceinline__ void emit_piece(const KParams &P, const uint32_t (&r)[8], int oc0, size_t o, int nv) {
+__device__ __forceinline__ void emit_piece(const KParams &P, const uint32_t (&r)[8], const float (&sc)[8], size_t o, int nv) {
     if (FUSED && DT == XGEN_I8_I32 && P.rq_scale) {
-        emit_requantised(P.rq_scale + oc0, P.rq_zero, (unsigned char *)P.y + o, nv == 8 && P.vec_out >= 4 && (P.c_out & 7) == 0, nv,
-                         r[0], r[1], r[2], r[3], r[4], r[5], r[6], r[7]);
+        emit_requantised(sc, P.rq_zero, (unsigned char *)P.y + o, nv == 8 && P.vec_out >= 4 && (P.c_out & 7) == 0, nv, r);
     } else if (DT != XGEN_F16_F32ACC) {
         store_raw_piece(P, r, (uint32_t *)P.y, o, nv);
     } else {
@@ -748,11 +748,12 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         const uint32_t tmem_res = (DT == XGEN_I8_I32 && P.fold) ? tmem_int : tmem_warp;
         const int oc_base = soc[0];
         if (oc_base >= 0) {
-            const int *pt = ptab + lane;
             uint32_t *const part = part_sums ? part_sums + (size_t)zsplit * P.out_elems : nullptr;
             const int K8 = (P.J + 7) >> 3;
             uint32_t *const wrow = ws_rows ? ws_rows + ((((size_t)sitem * P.n_splits + zsplit) * (size_t)(P.wpc * K8 * T)
                                                    + (size_t)warp * K8 * T) * 32 + lane) * 8 : nullptr;
+            const int *pt = ptab + lane;
+            const int *qtab = ptab + 32 * T;
             for (int j0 = 0; j0 < P.J; j0 += 8) {
                 const int oc0 = oc_base + j0;
                 if (oc0 >= P.c_out) break;
@@ -760,6 +761,9 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                 uint32_t bb[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k) bb[k] = (P.bias && !part && !wrow && k < nv) ? ((const uint32_t *)P.bias)[oc0 + k] : 0u;
+                float sc[8];                                          // re-quantisation scales of these channels
+#pragma unroll
+                for (int k = 0; k < 8; ++k) sc[k] = (FUSED && DT == XGEN_I8_I32 && P.rq_scale && k < nv) ? __ldg(P.rq_scale + oc0 + k) : 0.f;
                 if (FUSED && P.pool && !part && !wrow) {
                     // fused 2x2 max-pool: the four sums of a pooled pixel are columns of this thread
                     for (int q = 0; q < T / 4; ++q) {
@@ -779,7 +783,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                             else { finish_piece<DT, FUSED>(P, u, bb, oc0, nv, pt[pool_member<STRIDE>(q, m) * 32], f); max_piece<DT>(best, f); }
                         }
                         if (qidx < 0) continue;
-                        emit_piece<DT, FUSED>(P, best, oc0, (size_t)qidx * P.c_out + oc0, nv);
+                        emit_piece<DT, FUSED>(P, best, sc, (size_t)qidx * P.c_out + oc0, nv);
                     }
                     continue;
                 }
@@ -807,7 +811,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                         if (part) { store_raw_piece(P, r, part, (size_t)pidx * P.c_out + oc0, nv); continue; }
                         uint32_t f[8];
                         finish_piece<DT, FUSED>(P, r, bb, oc0, nv, pidx, f);
-                        emit_piece<DT, FUSED>(P, f, oc0, (size_t)pidx * P.c_out + oc0, nv);
+                        emit_piece<DT, FUSED>(P, f, sc, (size_t)pidx * P.c_out + oc0, nv);
                     }
                 }
             }
@@ -867,27 +871,49 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                 for (; z < S; ++z) add8(__ldcg(src + z * zstride), __ldcg(src + z * zstride + 1));
             };
             if (FUSED && P.pool) {
-                // units of one pooled pixel: (warp's filter group, 8-channel piece, pooled pixel q)
+                // Units of one pooled pixel: (warp's filter group, 8-channel piece, pooled pixel q).  The
+                // four running sums a unit covers are reduced by four warps side by side; they meet in
+                // shared memory (the staging area is free by now), where the first of them takes the maximum.
                 const int Q = T / 4, U = P.wpc * K8 * Q;
                 const int *qtab = ptab + 32 * T;
-                for (int unit = zsplit + S * warp; unit < U; unit += S * nwarps) {
+                uint32_t *pool_s = smem + P.plane_off_words + (size_t)(warp * 32 + lane) * 8;
+                const int per_pass = nwarps >> 2;
+                for (int u0 = zsplit; u0 < U; u0 += S * per_pass) {
+                    const int unit = u0 + S * (warp >> 2), m = warp & 3;
+                    const bool mine = (warp >> 2) < per_pass && unit < U;
                     const int q = unit % Q, k8 = (unit / Q) % K8, w = unit / (Q * K8);
-                    const int ocb = soc_s[w * P.J];
+                    const int ocb = mine ? soc_s[w * P.J] : -1;
                     const int oc0 = ocb + k8 * 8;
-                    const int qidx = qtab[q * 32 + lane];
-                    if (ocb < 0 || oc0 >= P.c_out || qidx < 0) continue;
+                    const int qidx = mine ? qtab[q * 32 + lane] : -1;
+                    const bool live = mine && ocb >= 0 && oc0 < P.c_out && qidx >= 0;
                     const int nv = min(8, P.c_out - oc0);
-                    uint32_t bb[8];
+                    uint32_t bb[8], f[8];
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) bb[k] = (P.bias && k < nv) ? ((const uint32_t *)P.bias)[oc0 + k] : 0u;
-                    uint32_t best[8], acc[8], f[8];
-                    for (int m = 0; m < 4; ++m) {
+                    for (int k = 0; k < 8; ++k) bb[k] = (live && P.bias && k < nv) ? ((const uint32_t *)P.bias)[oc0 + k] : 0u;
+                    if (live) {
+                        uint32_t acc[8];
                         const int t = pool_member<STRIDE>(q, m);
                         sum_row((w * K8 + k8) * T + t, acc);
-                        if (m == 0) finish_piece<DT, FUSED>(P, acc, bb, oc0, nv, ptab[t * 32 + lane], best);
-                        else { finish_piece<DT, FUSED>(P, acc, bb, oc0, nv, ptab[t * 32 + lane], f); max_piece<DT>(best, f); }
+                        finish_piece<DT, FUSED>(P, acc, bb, oc0, nv, ptab[t * 32 + lane], f);
+                        if (m != 0) {
+                            *reinterpret_cast<uint4 *>(pool_s) = make_uint4(f[0], f[1], f[2], f[3]);
+                            *reinterpret_cast<uint4 *>(pool_s + 4) = make_uint4(f[4], f[5], f[6], f[7]);
+                        }
                     }
-                    emit_piece<DT, FUSED>(P, best, oc0, (size_t)qidx * P.c_out + oc0, nv);
+                    __syncthreads();
+                    if (live && m == 0) {
+                        for (int mm = 1; mm < 4; ++mm) {
+                            const uint4 a = *reinterpret_cast<const uint4 *>(pool_s + (size_t)mm * 256);
+                            const uint4 c = *reinterpret_cast<const uint4 *>(pool_s + (size_t)mm * 256 + 4);
+                            const uint32_t g[8] = {a.x, a.y, a.z, a.w, c.x, c.y, c.z, c.w};
+                            max_piece<DT>(f, g);
+                        }
+                        float sc[8];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) sc[k] = (DT == XGEN_I8_I32 && P.rq_scale && k < nv) ? __ldg(P.rq_scale + oc0 + k) : 0.f;
+                        emit_piece<DT, FUSED>(P, f, sc, (size_t)qidx * P.c_out + oc0, nv);
+                    }
+                    __syncthreads();
                 }
             } else {
                 for (int row = zsplit + S * warp; row < R; row += S * nwarps) {
@@ -901,8 +927,11 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                     sum_row(row, acc);
 #pragma unroll
                     for (int k = 0; k < 8; ++k) bb[k] = (P.bias && k < nv) ? ((const uint32_t *)P.bias)[oc0 + k] : 0u;
+                    float sc[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) sc[k] = (FUSED && DT == XGEN_I8_I32 && P.rq_scale && k < nv) ? __ldg(P.rq_scale + oc0 + k) : 0.f;
                     finish_piece<DT, FUSED>(P, acc, bb, oc0, nv, pidx, f);
-                    emit_piece<DT, FUSED>(P, f, oc0, (size_t)pidx * P.c_out + oc0, nv);
+                    emit_piece<DT, FUSED>(P, f, sc, (size_t)pidx * P.c_out + oc0, nv);
                 }
             }
         }
