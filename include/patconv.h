@@ -191,7 +191,8 @@ typedef struct {
  * are honoured as in xgen_patconv_run.
  * Errors as xgen_patconv_run, plus INVALID_ARG (NULL epilogue, misaligned residual or scale),
  * SHAPE (pooling an odd extent), UNSUPPORTED (pool other than 0 or 2; re-quantisation of a
- * floating-point layer).
+ * floating-point layer; a handle whose last xgen_patconv_plan chose 4x2-pixel blocks -- plan
+ * it again with xgen_patconv_tuning.no_small_blocks).
  */
 xgen_status xgen_patconv_run_fused(const xgen_patconv_packed *packed, const void *x_dev, int32_t n,
                                    int32_t h, int32_t w, const void *bias_dev,
@@ -311,12 +312,16 @@ xgen_status xgen_patconv_plan(xgen_patconv_packed *packed, int32_t n, int32_t h,
  *                      ended (every later run of the handle)
  *   wait_limit_ms      bound of the device-side waits, milliseconds (default
  *                      2000, at most 60000)
+ *   no_small_blocks    keep 4x4 output pixels per thread even for shapes that the
+ *                      planner would run with 4x2 pixels per thread (a single small
+ *                      image); xgen_patconv_run_fused needs the 4x4 blocks
  */
 typedef struct {
     int32_t splits;
     int32_t no_copy_engine;
     int32_t no_launch_overlap;
     int32_t wait_limit_ms;
+    int32_t no_small_blocks;
 } xgen_patconv_tuning;
 
 /* xgen_patconv_plan with the caller's tuning (NULL = xgen_patconv_plan).  Errors as
@@ -339,7 +344,8 @@ typedef struct {
                                    1: a tile is 32 consecutive blocks of the row-by-row numbering
                                    of all images' blocks (lanes_x = blocks per image row)         */
     int32_t lanes_x, lanes_y, lanes_n;  /* how a warp's 32 lanes tile x, y and images             */
-    int32_t pixels_per_lane;    /* output pixels one lane owns (16 at stride 1, 8 at stride 2)     */
+    int32_t pixels_per_lane;    /* output pixels one lane owns: 16 (4x4) at stride 1, or 8 (4x2)
+                                   where the planner chose the small block; 8 (2x4) at stride 2    */
     int32_t stages;             /* pipeline stages of staged channel chunks                        */
     int32_t uses_copy_engine;   /* input tiles arrive through the tensor copy engine               */
     int64_t shared_bytes;       /* dynamic shared memory per block                                 */

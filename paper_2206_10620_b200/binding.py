@@ -50,7 +50,8 @@ class Stats(ctypes.Structure):
 
 class Tuning(ctypes.Structure):
     _fields_ = [("splits", ctypes.c_int32), ("no_copy_engine", ctypes.c_int32),
-                ("no_launch_overlap", ctypes.c_int32), ("wait_limit_ms", ctypes.c_int32)]
+                ("no_launch_overlap", ctypes.c_int32), ("wait_limit_ms", ctypes.c_int32),
+                ("no_small_blocks", ctypes.c_int32)]
 
 
 class PlanStats(ctypes.Structure):
@@ -190,10 +191,12 @@ class Packed:
             "masks": arr(v.compiled_masks, npc, ctypes.c_uint16, np.uint16),
         }
 
-    def plan(self, n, h, w, splits=0, no_copy_engine=False, no_launch_overlap=False, wait_limit_ms=0):
+    def plan(self, n, h, w, splits=0, no_copy_engine=False, no_launch_overlap=False, wait_limit_ms=0,
+             no_small_blocks=False):
         """xgen_patconv_plan, or xgen_patconv_plan_tuned when any tuning field is given."""
-        if splits or no_copy_engine or no_launch_overlap or wait_limit_ms:
-            t = Tuning(int(splits), int(bool(no_copy_engine)), int(bool(no_launch_overlap)), int(wait_limit_ms))
+        if splits or no_copy_engine or no_launch_overlap or wait_limit_ms or no_small_blocks:
+            t = Tuning(int(splits), int(bool(no_copy_engine)), int(bool(no_launch_overlap)), int(wait_limit_ms),
+                       int(bool(no_small_blocks)))
             _check(lib().xgen_patconv_plan_tuned(self._h, n, h, w, ctypes.byref(t)), "xgen_patconv_plan_tuned")
         else:
             _check(lib().xgen_patconv_plan(self._h, n, h, w), "xgen_patconv_plan")

@@ -65,12 +65,13 @@ def table(np_):
     return LIBRARY[:np_] if np_ <= 12 else ALL_MASKS
 
 
-def gen_block(np_, stride):
+def gen_block(np_, stride, bh=4):
     """One interpreter block.  Stride 1: a thread owns 4x4 output pixels (16 running
-    sums per filter, patch 6 rows x 4 pairs); stride 2: 2x4 pixels (8 sums, patch
-    9 rows x 3 pairs)."""
+    sums per filter, patch 6 rows x 4 pairs) or, in the small-block form for images
+    that would leave most lanes of a 4x4 tiling idle, 4x2 pixels (8 sums, patch 4 rows
+    x 4 pairs); stride 2: 2x4 pixels (8 sums, patch 9 rows x 3 pairs)."""
     masks = table(np_)
-    bw, bh = (4, 4) if stride == 1 else (2, 4)
+    bw = 4 if stride == 1 else 2
     T = bw * bh
     rows = (bh - 1) * stride + 3
     ppr = 4 if stride == 1 else 3            # operand pairs per patch row
@@ -147,11 +148,11 @@ def gen_block(np_, stride):
 
 def main(out_path):
     parts = ["// Generated by gen_core.py -- do not edit.\n"]
-    for stride in (1, 2):
+    for stride, bh, tag in ((1, 4, "S1"), (2, 4, "S2"), (1, 2, "S1H2")):
         for np_ in (4, 8, 12, 126):
-            lines = gen_block(np_, stride)
-            parts.append("#define PATCONV_CORE_S%d_NP%d(sp, baseA, plane_bytes, pitch_bytes, tmem_base, baseB) \\\n"
-                         % (stride, np_))
+            lines = gen_block(np_, stride, bh)
+            parts.append("#define PATCONV_CORE_%s_NP%d(sp, baseA, plane_bytes, pitch_bytes, tmem_base, baseB) \\\n"
+                         % (tag, np_))
             parts.append("  asm volatile( \\\n")
             for s in lines:
                 parts.append('    "%s\\n" \\\n' % s)

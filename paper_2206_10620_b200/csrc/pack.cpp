@@ -187,7 +187,10 @@ xgen_status build_layout(PackedHost &out, const PackConfig &cfg) {
     const int n_groups = n_blocks * wpc;
     const int n_chunks = (cin + cc - 1) / cc;
 
+    if (cfg.block_rows != 4 && !(cfg.block_rows == 2 && out.stride == 1)) return XGEN_ERR_INVALID_ARG;
     out.J = J; out.wpc = wpc; out.cc = cc;
+    out.bh = cfg.block_rows;
+    out.tpix = (out.stride == 1 ? 4 : 2) * cfg.block_rows;
     out.slots.clear(); out.max_seg_slots = 0;
     out.n_blocks = n_blocks; out.n_chunks = n_chunks;
     out.slot_oc.assign((size_t)n_groups * J, -1);
@@ -260,7 +263,7 @@ xgen_status build_layout(PackedHost &out, const PackConfig &cfg) {
                     ++n_loads;
                     for (const Ent &e : ents) {
                         const uint32_t *w4 = &out.kw4[((size_t)soc[e.j] * cin + ic) * 4];
-                        push_slot((uint32_t)e.p, (uint32_t)(e.j * pix_per_thread(out.stride)), w4);
+                        push_slot((uint32_t)e.p, (uint32_t)(e.j * out.tpix), w4);
                     }
                 }
                 push_slot((uint32_t)np + 1, 0, nullptr);

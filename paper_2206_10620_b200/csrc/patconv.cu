@@ -176,10 +176,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, volati
     return false;
 }
 
-template <int STRIDE, int NP>
+template <int STRIDE, int NP, int BH>
 __device__ __forceinline__ void run_commands(uint32_t sp, uint32_t base_a, uint32_t plane_bytes,
                                              uint32_t pitch_bytes, uint32_t tmem_base, uint32_t base_b) {
-    if (STRIDE == 1) {
+    if (STRIDE == 1 && BH == 2) {
+        if (NP == 4) PATCONV_CORE_S1H2_NP4(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
+        else if (NP == 8) PATCONV_CORE_S1H2_NP8(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
+        else if (NP == 12) PATCONV_CORE_S1H2_NP12(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
+        else PATCONV_CORE_S1H2_NP126(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
+    } else if (STRIDE == 1) {
         if (NP == 4) PATCONV_CORE_S1_NP4(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
         else if (NP == 8) PATCONV_CORE_S1_NP8(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
         else if (NP == 12) PATCONV_CORE_S1_NP12(sp, base_a, plane_bytes, pitch_bytes, tmem_base, base_b);
@@ -353,7 +358,8 @@ struct SlotOrigin { int gn, gy0, gx0; bool used; };
 // ---- the kernel -----------------------------------------------------------------
 // FUSED: with the operators fused behind the convolution (residual addition, max-pool,
 // re-quantisation); the plain instances carry none of that code.
-template <int DT, int STRIDE, int NP, bool FUSED>
+// BH: rows of the pixel block a thread owns (4; 2 = the small 4x2 block of stride 1).
+template <int DT, int STRIDE, int NP, bool FUSED, int BH = 4>
 __global__ void __launch_bounds__((kMaxWarps + kProducerWarps) * 32)
 patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     extern __shared__ __align__(128) uint32_t smem[];
@@ -361,7 +367,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     __shared__ int abort_s;
     __shared__ int soc_s[kMaxWarps * 16];           // original output channel of every filter slot of this block
     constexpr int XB = DTraits<DT>::xbytes;
-    constexpr int BW = STRIDE == 1 ? 4 : 2, BH = 4;   // output pixels per thread: BW x BH
+    constexpr int BW = STRIDE == 1 ? 4 : 2;           // output pixels per thread: BW x BH
     constexpr int T = BW * BH;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -732,7 +738,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
             const uint32_t sp = smem_base + (uint32_t)(P.cmd_off_words + s * P.cmd_stage_words) * 4u +
                                 (uint32_t)(sg - s0) * (kDevSlotWords * 4u);
             const uint32_t base_a = smem_base + (uint32_t)(P.plane_off_words + s * P.plane_stage_words) * 4u + thr_off;
-            run_commands<STRIDE, NP>(sp, base_a, plane_bytes, pitch_bytes, tmem_warp, base_a + half_bytes);
+            run_commands<STRIDE, NP, BH>(sp, base_a, plane_bytes, pitch_bytes, tmem_warp, base_a + half_bytes);
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty(s));
             if (DT == XGEN_I8_I32 && P.fold && ((k + 1) % P.flush_chunks == 0)) fold_partial_sums();
@@ -1006,7 +1012,6 @@ static bool log_enabled() {
 }
 
 static inline int pixels_per_thread_x(int stride) { return stride == 1 ? 4 : 2; }
-static inline int pixels_per_thread(int stride) { return 4 * pixels_per_thread_x(stride); }
 
 struct Geometry {
     int lx_log, ly_log, ln_log, tiles_x, tiles_y, tiles_n;
@@ -1033,10 +1038,10 @@ static int row_load_conflicts(F addr) {
 
 // Grid tiling: the 32 lanes of a warp tile LX x LY x LN (powers of two) blocks of 4x4 (2x4)
 // pixels; chosen to cover the most output pixels per tile.
-static Geometry grid_geometry(int n, int ho, int wo, int stride) {
+static Geometry grid_geometry(int n, int ho, int wo, int stride, int bh) {
     Geometry best{};
     double best_eff = -1.0;
-    const int bw = pixels_per_thread_x(stride), bh = 4;
+    const int bw = pixels_per_thread_x(stride);
     for (int lx_log = 5; lx_log >= 0; --lx_log)
         for (int ly_log = 5 - lx_log; ly_log >= 0; --ly_log) {
             const int ln_log = 5 - lx_log - ly_log;
@@ -1067,7 +1072,7 @@ static Geometry grid_geometry(int n, int ho, int wo, int stride) {
             const int LX = 1 << best.lx_log, LY = 1 << best.ly_log;
             const int c = row_load_conflicts([&](int lane) {
                 int x = lane & (LX - 1), y = (lane >> best.lx_log) & (LY - 1), nn = lane >> (best.lx_log + best.ly_log);
-                return nn * istr + y * 4 * stride * p + x * 4;
+                return nn * istr + y * bh * stride * p + x * 4;
             });
             if (c < best_c) { best_c = c; best_p = p; best_i = istr; }
         }
@@ -1082,8 +1087,8 @@ static Geometry grid_geometry(int n, int ho, int wo, int stride) {
 // tile takes 32 consecutive ones, so only the last tile of the launch has idle lanes; what is
 // lost is the part of edge blocks that hangs over the image.  Every block row a tile touches is
 // staged as a slot of its own: the full image width plus halo, with its own halo rows.
-static bool row_geometry(int n, int ho, int wo, int stride, Geometry &g) {
-    const int bw = pixels_per_thread_x(stride), bh = 4;
+static bool row_geometry(int n, int ho, int wo, int stride, int bh, Geometry &g) {
+    const int bw = pixels_per_thread_x(stride);
     const int bxn = (wo + bw - 1) / bw, byn = (ho + bh - 1) / bh;
     if (bxn > 32) return false;
     const int64_t total = (int64_t)n * byn * bxn;
@@ -1243,26 +1248,28 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-template <int DT, int STRIDE, bool FUSED>
+template <int DT, int STRIDE, bool FUSED, int BH>
 static const void *kernel_np(int np) {
     switch (np) {
-        case 4: return (const void *)patconv_kernel<DT, STRIDE, 4, FUSED>;
-        case 8: return (const void *)patconv_kernel<DT, STRIDE, 8, FUSED>;
-        case 12: return (const void *)patconv_kernel<DT, STRIDE, 12, FUSED>;
-        default: return (const void *)patconv_kernel<DT, STRIDE, 126, FUSED>;
+        case 4: return (const void *)patconv_kernel<DT, STRIDE, 4, FUSED, BH>;
+        case 8: return (const void *)patconv_kernel<DT, STRIDE, 8, FUSED, BH>;
+        case 12: return (const void *)patconv_kernel<DT, STRIDE, 12, FUSED, BH>;
+        default: return (const void *)patconv_kernel<DT, STRIDE, 126, FUSED, BH>;
     }
 }
 
-template <bool FUSED>
-static const void *kernel_of(const PackedHost &p) {
-    if (p.dtype == XGEN_F32) return p.stride == 1 ? kernel_np<XGEN_F32, 1, FUSED>(p.np) : kernel_np<XGEN_F32, 2, FUSED>(p.np);
-    if (p.dtype == XGEN_F16_F32ACC) return p.stride == 1 ? kernel_np<XGEN_F16_F32ACC, 1, FUSED>(p.np) : kernel_np<XGEN_F16_F32ACC, 2, FUSED>(p.np);
-    return p.stride == 1 ? kernel_np<XGEN_I8_I32, 1, FUSED>(p.np) : kernel_np<XGEN_I8_I32, 2, FUSED>(p.np);
+template <int DT>
+static const void *kernel_of(const PackedHost &p, bool fused) {
+    if (p.stride == 2) return fused ? kernel_np<DT, 2, true, 4>(p.np) : kernel_np<DT, 2, false, 4>(p.np);
+    if (p.bh == 2) return kernel_np<DT, 1, false, 2>(p.np);          // the small block has no fused instances
+    return fused ? kernel_np<DT, 1, true, 4>(p.np) : kernel_np<DT, 1, false, 4>(p.np);
 }
 
 // The kernel instance of a packed layer, without or with the fused operators.
 static const void *kernel_for(const PackedHost &p, bool fused = false) {
-    return fused ? kernel_of<true>(p) : kernel_of<false>(p);
+    if (p.dtype == XGEN_F32) return kernel_of<XGEN_F32>(p, fused);
+    if (p.dtype == XGEN_F16_F32ACC) return kernel_of<XGEN_F16_F32ACC>(p, fused);
+    return kernel_of<XGEN_I8_I32>(p, fused);
 }
 
 // The opt-in to large dynamic shared memory is per function and per device: do it once.
@@ -1321,7 +1328,7 @@ static xgen_status layout_for(const PackedHost &p, const Geometry &g_in, int n, 
     // widest aligned store per 8-channel piece: 8 words (32-byte aligned rows), 4, or scalar
     kp.vec_out = ((p.c_out % 8) == 0 && y_aligned32) ? 8 : ((p.c_out % 4) == 0 ? 4 : 0);
     const bool is_i8 = p.dtype == XGEN_I8_I32;
-    const int T = pixels_per_thread(p.stride);
+    const int T = p.tpix;
     kp.flush_chunks = 16777216 / (p.cc * 4 * 32640);
     if (kp.flush_chunks < 1) return XGEN_ERR_UNSUPPORTED;
     kp.fold = (is_i8 && p.int_totals) ? 1 : 0;
@@ -1379,9 +1386,9 @@ static xgen_status layout_for(const PackedHost &p, const Geometry &g_in, int n, 
 static xgen_status make_layout(const PackedHost &p, int n, int hh, int ww, bool y_aligned32, bool tma_ok, Layout &L,
                                bool *rows_wanted = nullptr) {
     const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
-    const Geometry grid = grid_geometry(n, ho, wo, p.stride);
+    const Geometry grid = grid_geometry(n, ho, wo, p.stride, p.bh);
     Geometry rows;
-    const bool want = row_geometry(n, ho, wo, p.stride, rows) && rows.covered > 1.08 * grid.covered;
+    const bool want = row_geometry(n, ho, wo, p.stride, p.bh, rows) && rows.covered > 1.08 * grid.covered;
     if (rows_wanted) *rows_wanted = want;
     const xgen_status gs = layout_for(p, grid, n, hh, ww, y_aligned32, tma_ok, L);
     if (want) {
@@ -1397,7 +1404,7 @@ static xgen_status make_layout(const PackedHost &p, int n, int hh, int ww, bool 
 
 // 1 KB rows of partial sums one (item, split) writes in a split run reduced inside the kernel.
 static size_t rows_per_item(const PackedHost &p) {
-    return (size_t)p.wpc * ((p.J + 7) / 8) * pixels_per_thread(p.stride);
+    return (size_t)p.wpc * ((p.J + 7) / 8) * p.tpix;
 }
 
 // The prepared launch of (shape, input address, alignment class of y): from the handle's
@@ -1469,7 +1476,7 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
     const void *residual = ep ? ep->residual_dev : nullptr;
     const float *rq_scale = ep ? ep->requant_scale_dev : nullptr;
     if (ep) {
-        if (forced) return XGEN_ERR_UNSUPPORTED;
+        if (forced || p.bh != 4) return XGEN_ERR_UNSUPPORTED;
         if (pool != 0 && pool != 2) return XGEN_ERR_UNSUPPORTED;
         if (pool == 2 && ((ho & 1) || (wo & 1))) return XGEN_ERR_SHAPE;
         if (rq_scale && p.dtype != XGEN_I8_I32) return XGEN_ERR_UNSUPPORTED;
@@ -1738,7 +1745,7 @@ xgen_status xgen_patconv_plan_info(const xgen_patconv_packed *h, int32_t n, int3
     out->lanes_x = L.g.rows ? L.g.bxn : 1 << L.g.lx_log; out->lanes_y = L.g.rows ? 1 : 1 << L.g.ly_log;
     out->lanes_n = L.g.rows ? 1 : 1 << L.g.ln_log;
     out->covered = L.g.covered;
-    out->pixels_per_lane = pixels_per_thread(p.stride);
+    out->pixels_per_lane = p.tpix;
     out->stages = L.kp.n_stages;
     out->uses_copy_engine = L.kp.use_tma;
     out->shared_bytes = (int64_t)L.smem;
@@ -1757,29 +1764,63 @@ xgen_status xgen_patconv_plan_tuned(xgen_patconv_packed *h, int32_t n, int32_t h
     if ((int64_t)n * ho * wo * p.c_out > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
     const xgen_patconv_tuning tn = tuning ? *tuning : xgen_patconv_tuning{};
     const bool tma_ok = !tn.no_copy_engine && encode_tiled_fn() != nullptr;
-    Layout L;
-    bool rows_wanted = false;
-    xgen_status ls = make_layout(p, n, hh, ww, true, tma_ok, L, &rows_wanted);
-    if (ls != XGEN_OK) return ls;
     int prev = 0;
     if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(h->device) != cudaSuccess) return XGEN_ERR_CUDA;
     xgen_status rs = XGEN_OK;
+    // Rebuild the command stream for another grouping (the kept weights are still in the handle)
+    // and upload it again; every later run of the handle uses the new layout.
+    auto relayout = [&](PackConfig cfg) {
+        xgen_status st = cudaDeviceSynchronize() == cudaSuccess ? XGEN_OK : XGEN_ERR_CUDA;
+        try {
+            if (st == XGEN_OK) st = build_layout(h->host, cfg);
+            while (st == XGEN_OK && cfg.channels_per_chunk > 4 &&
+                   (size_t)h->host.max_seg_slots * kDevSlotBytes > kCmdStageBudget) {
+                cfg.channels_per_chunk /= 2;
+                st = build_layout(h->host, cfg);
+            }
+        } catch (const std::bad_alloc &) {
+            st = XGEN_ERR_ALLOC;
+        }
+        if (st == XGEN_OK) st = upload_layout(h);
+        forget_prepared_launches(h);
+        return st;
+    };
+    // Block shape.  A stride-1 thread owns 4x4 output pixels; a shape that leaves most lanes of
+    // every such tiling idle (a single 14x14 image fills 38 % of a warp's 512 pixel slots) runs
+    // with 4x2 pixels per thread and 16 filters per warp instead, if that at least covers 1.4
+    // times as much.  Integer layers with int32 totals keep the large block (their second
+    // tensor-memory row leaves no room for 16 filters).
+    {
+        auto covered = [&](int bh) {
+            const Geometry g = grid_geometry(n, ho, wo, p.stride, bh);
+            Geometry r;
+            return row_geometry(n, ho, wo, p.stride, bh, r) ? std::max(g.covered, r.covered) : g.covered;
+        };
+        const bool small = p.stride == 1 && !p.int_totals && !tn.no_small_blocks && covered(4) < 0.55 && covered(2) >= 1.4 * covered(4);
+        if (small != (p.bh == 2)) {
+            PackConfig cfg = choose_pack_config(p.c_in, p.c_out, p.dtype, p.stride, p.int_totals);
+            if (p.dtype == XGEN_I8_I32 && cfg.channels_per_chunk < 4) cfg.channels_per_chunk = 4;
+            if (small) {
+                cfg.block_rows = 2;
+                cfg.filters_per_group = 16;
+                cfg.groups_per_block = std::min((p.c_out + 15) / 16, (int)kMaxWarps);
+            }
+            rs = relayout(cfg);
+            if (rs != XGEN_OK) { cudaSetDevice(prev); h->plan_splits = 1; h->plan_n = 0; return rs; }
+        }
+    }
+    Layout L;
+    bool rows_wanted = false;
+    xgen_status ls = make_layout(p, n, hh, ww, true, tma_ok, L, &rows_wanted);
+    if (ls != XGEN_OK) { cudaSetDevice(prev); return ls; }
     if (rows_wanted && !L.g.rows && p.cc > 4) {
         // Row tiling covers more of this shape but its staged tile (one slot per block row)
-        // does not fit with the chunk size chosen at pack time: rebuild the command stream
-        // with half the channels per chunk (the kept weights are still in the handle) and
-        // upload it again.  Every later run of the handle uses the new layout.
-        if (cudaDeviceSynchronize() != cudaSuccess) rs = XGEN_ERR_CUDA;
-        if (rs == XGEN_OK) {
-            try {
-                rs = build_layout(h->host, PackConfig{p.J, p.wpc, p.cc / 2});
-            } catch (const std::bad_alloc &) {
-                rs = XGEN_ERR_ALLOC;
-            }
-        }
-        if (rs == XGEN_OK) rs = upload_layout(h);
+        // does not fit with the chunk size chosen at pack time: half the channels per chunk.
+        PackConfig cfg{p.J, p.wpc, p.cc / 2};
+        cfg.block_rows = p.bh;
+        rs = relayout(cfg);
         if (rs == XGEN_OK) rs = make_layout(p, n, hh, ww, true, tma_ok, L);
-        if (rs != XGEN_OK) { cudaSetDevice(prev); h->plan_splits = 1; h->plan_n = 0; forget_prepared_launches(h); return rs; }
+        if (rs != XGEN_OK) { cudaSetDevice(prev); h->plan_splits = 1; h->plan_n = 0; return rs; }
     }
     int sms = 148, bps = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
@@ -1800,7 +1841,7 @@ xgen_status xgen_patconv_plan_tuned(xgen_patconv_packed *h, int32_t n, int32_t h
     // are split (they are numbered last, so their blocks start as the wave before them drains),
     // all earlier items run whole.
     const int64_t capacity = std::max<int64_t>(1, (int64_t)sms * bps);
-    const double slot_macs_item = 4.0 * (double)p.stats.kernels_surviving / (double)p.n_blocks * 32.0 * pixels_per_thread(p.stride);
+    const double slot_macs_item = 4.0 * (double)p.stats.kernels_surviving / (double)p.n_blocks * 32.0 * p.tpix;
     auto sm_rate = [&](int warps) { return 50.0 * std::pow((double)std::min(warps, 16) / 16.0, 0.65); };   // multiply-adds per cycle
     int64_t splits = 1, whole = L.items;
     if (L.items <= capacity) {

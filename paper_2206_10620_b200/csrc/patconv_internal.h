@@ -29,6 +29,7 @@ struct PackConfig {
     int filters_per_group;   // J
     int groups_per_block;    // warps per thread block
     int channels_per_chunk;  // input channels staged per pipeline step (power of two)
+    int block_rows = 4;      // rows of the pixel block a thread owns: 4, or 2 (stride 1 only: 4x2 pixels)
 };
 
 // Host image of a packed layer.
@@ -36,6 +37,7 @@ struct PackedHost {
     int c_in = 0, c_out = 0, stride = 1;
     xgen_dtype dtype = XGEN_F32;
     int J = 0, wpc = 0, cc = 0, np = 0;          // np: compiled pattern-table size
+    int bh = 4, tpix = 16;                        // block rows and output pixels of a thread (tensor-memory columns per filter)
     int n_blocks = 0, n_chunks = 0;
     int max_seg_slots = 0;
     std::vector<uint32_t> slots;                  // kSlotWords words per command

@@ -142,6 +142,58 @@ def test_row_tiling(dtype, case):
     compare(d, run_gpu(pk, d.x, None, False), bias=None, relu=False)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "f16", "i8"])
+@pytest.mark.parametrize("shape", [(1, 14, 14), (1, 7, 7), (1, 13, 10), (2, 6, 5)])
+def test_small_blocks_for_small_images(dtype, shape):
+    """A single small image leaves most lanes of every 4x4-pixel tiling idle: planning such a shape
+    switches the handle to 4x2 pixels per thread and 16 filters per warp (the command stream is
+    rebuilt); planning a large shape switches it back."""
+    import torch
+    n, h, w = shape
+    d = _layer(dtype, n, 96, 200, h, w, 1, prune=0.6, lib=12, seed=121)
+    pk = pack(d)
+    assert pk.plan_info(n, h, w)["pixels_per_lane"] == 16
+    y0 = run_gpu(pk, d.x, d.bias, True)
+    compare(d, y0)
+    pk.plan(n, h, w)
+    info = pk.plan_info(n, h, w)
+    assert info["pixels_per_lane"] == 8 and pk.stats()["filters_per_group"] == 16
+    compare(d, run_gpu(pk, d.x, d.bias, True))
+    compare(d, run_gpu(pk, d.x, None, False), bias=None, relu=False)
+    pk.plan(n, h, w, splits=3)
+    assert pk.plan_info(n, h, w)["splits"] == 3
+    y1 = run_gpu(pk, d.x, d.bias, True)
+    compare(d, y1)
+    # the fused operators need the large block
+    x = torch.from_numpy(d.x).cuda()
+    y = torch.empty((n, h, w, 200), dtype={"f32": torch.float32, "f16": torch.float16, "i8": torch.int32}[dtype], device="cuda")
+    with pytest.raises(binding.PatconvError) as e:
+        pk.run_fused(x.data_ptr(), n, h, w, 0, y.data_ptr(), relu=True)
+    assert e.value.status == 4
+    pk.plan(n, h, w, no_small_blocks=True)
+    assert pk.plan_info(n, h, w)["pixels_per_lane"] == 16
+    pk.run_fused(x.data_ptr(), n, h, w, 0, y.data_ptr(), relu=True)
+    pk.sync()
+    compare(d, y.cpu().numpy(), bias=None)
+    # another, large shape on the same handle: back to 4x4 blocks
+    pk.plan(n, h, w)
+    assert pk.plan_info(n, h, w)["pixels_per_lane"] == 8
+    d2 = _layer(dtype, 2, 96, 200, 40, 40, 1, prune=0.6, lib=12, seed=121)
+    pk.plan(2, 40, 40)
+    assert pk.plan_info(2, 40, 40)["pixels_per_lane"] == 16
+    d2.w, d2.pid, d2.masks = d.w, d.pid, d.masks
+    compare(d2, run_gpu(pk, d2.x, d.bias, True), bias=d.bias)
+
+
+def test_small_blocks_universal_table():
+    d = _layer("f32", 1, 32, 48, 12, 12, 1, prune=0.4, lib=4, seed=131)
+    d.masks = np.array([0x00F, 0x1E0, 0x145, 0x0AA], dtype=np.uint16)
+    pk = pack(d)
+    pk.plan(1, 12, 12)
+    assert pk.plan_info(1, 12, 12)["pixels_per_lane"] == 8 and pk.stats()["patterns_compiled"] == 126
+    compare(d, run_gpu(pk, d.x, d.bias, True))
+
+
 @pytest.mark.parametrize("dtype,stride", [("f32", 2), ("f16", 1), ("f16", 2), ("i8", 1), ("i8", 2)])
 def test_universal_table_other_variants(dtype, stride):
     d = _layer(dtype, 2, 24, 40, 13, 15, stride, prune=0.4, lib=4, seed=71)
