@@ -205,7 +205,7 @@ def run_reference(args):
 class Stack:
     """The layers of one workload on the device: packed, planned, with inputs and outputs."""
 
-    def __init__(self, specs, seed, device_index, plan=True, keep_host=True):
+    def __init__(self, specs, seed, device_index, plan=True, keep_host=True, no_small_blocks=False):
         import torch
         from paper_2206_10620_b200 import binding
         self.torch = torch
@@ -217,7 +217,7 @@ class Stack:
             d = wl.make_layer(s, seed=seed)
             pk = binding.Packed(s.c_in, s.c_out, s.stride, s.dtype, d.masks, d.w, d.pid, device=device_index)
             if plan:
-                pk.plan(s.n, s.h, s.w)
+                pk.plan(s.n, s.h, s.w, no_small_blocks=no_small_blocks)
             x = torch.from_numpy(d.x).to(dev)
             b = torch.from_numpy(d.bias).to(dev)
             y = torch.empty((s.n, s.ho, s.wo, s.c_out), dtype=tdt[s.dtype], device=dev)
@@ -481,7 +481,7 @@ def run_gpu(args):
             return out
 
         ends = [s for s in wl.config_vgg16() if s.name in ("conv2", "conv4", "conv7", "conv10", "conv13")]
-        stk = Stack(ends, wl.BASE_SEED, local, keep_host=False)
+        stk = Stack(ends, wl.BASE_SEED, local, keep_host=False, no_small_blocks=True)   # the fused operators need 4x4 blocks
         plain_us = time_layers(stk, lambda it: it[2].run(it[3].data_ptr(), it[0].n, it[0].h, it[0].w, it[4].data_ptr(),
                                                          True, it[5].data_ptr(), stream))
         pooled = [torch.empty((s.n, s.ho // 2, s.wo // 2, s.c_out), dtype=torch.float32, device=dev) for s in ends]

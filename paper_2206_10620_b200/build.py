@@ -32,8 +32,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-shared", "-Xcompiler", "-fPIC", "-I", _INC, "-I", _CSRC, "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    if os.environ.get("PATCONV_F2") is not None:
-        cmd += ["-DPATCONV_F2=%d" % int(os.environ["PATCONV_F2"])]
     cmd += [os.path.join(_CSRC, s) for s in _SOURCES]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB_PATH)
