@@ -277,19 +277,29 @@ xgen_status xgen_patconv_enqueue_host(const xgen_patconv_packed *packed, const v
  * cross-channel reduction of this implementation).  Shapes with more items
  * than the GPU holds blocks run in waves; there the items of the last, partly
  * filled wave are split the same way, so that the wave ends sooner.  The blocks of a split write
- * their partial sums to a workspace, count themselves in, wait (with a bound in
- * time) for the others and each reduce a share, all inside the one kernel.
- * Because they wait for each other, the split count is chosen so that every
- * block of the launch is resident at once on an otherwise idle GPU.  Hence the
- * rule: a planned split launch must not share the GPU with another planned
- * split launch -- of this handle (they also share the workspace) or of any
- * other handle -- nor with any other kernel that may keep its blocks from
- * becoming resident; put such launches on one stream or order them with
- * events.  If the rule is broken the blocks may hold each other's places; the
- * waits then run out (default 2 s), the kernel ends, its results are invalid,
- * and xgen_patconv_last_status returns XGEN_ERR_TIMEOUT (xgen_patconv_run has
- * returned XGEN_OK long before: it only enqueues).  Work that merely delays the
- * blocks (a kernel running before them on the same stream) is harmless.
+ * their partial sums to a workspace and count themselves in, all inside the one
+ * kernel; the planner then picks one of two ways to add the sums up (see
+ * xgen_patconv_plan_stats.last_arriver).
+ *   Waiting splits: the blocks wait (with a bound in time) for the others and each
+ * reduce a share.  Because they wait for each other, the split count is chosen so
+ * that every block of the launch is resident at once on an otherwise idle GPU.
+ * Hence the rule: such a launch must not share the GPU with another waiting split
+ * launch -- of this handle or of any other handle -- nor with any other kernel
+ * that may keep its blocks from becoming resident; put such launches on one
+ * stream or order them with events.  If the rule is broken the blocks may hold
+ * each other's places; the waits then run out (default 2 s), the kernel ends,
+ * its results are invalid, and xgen_patconv_last_status returns
+ * XGEN_ERR_TIMEOUT (xgen_patconv_run has returned XGEN_OK long before: it only
+ * enqueues).  Work that merely delays the blocks (a kernel running before them
+ * on the same stream) is harmless.
+ *   Last arriver: nobody waits; the block of an item that counts itself in last adds
+ * up all of the item's sums.  Any number of splits and of blocks is allowed (the
+ * blocks run in waves), and other kernels, waiting splits of other handles among
+ * them, may share the GPU.  It measured slower than waiting splits on every shape
+ * tried, so the planner takes it only on request (xgen_patconv_tuning.reduce_mode
+ * = 2): the mode for callers that run planned layers on several streams at once.
+ *   Either way two planned split launches of ONE handle must not run at the same
+ * time (they share the workspace and the counters): one stream, or events.
  * The call allocates the workspace and the counters, owned by the handle, so it
  * synchronises the device and must not be called while the handle is in use.
  * Without this call every shape runs unsplit.
@@ -315,6 +325,9 @@ xgen_status xgen_patconv_plan(xgen_patconv_packed *packed, int32_t n, int32_t h,
  *   no_small_blocks    keep 4x4 output pixels per thread even for shapes that the
  *                      planner would run with 4x2 pixels per thread (a single small
  *                      image); xgen_patconv_run_fused needs the 4x4 blocks
+ *   reduce_mode        how split items are added up: 0 or 1 by waiting splits, 2 by the
+ *                      last arriver (then `splits` is clamped to the number of channel
+ *                      chunks only, not to what is resident at once)
  */
 typedef struct {
     int32_t splits;
@@ -322,6 +335,7 @@ typedef struct {
     int32_t no_launch_overlap;
     int32_t wait_limit_ms;
     int32_t no_small_blocks;
+    int32_t reduce_mode;
 } xgen_patconv_tuning;
 
 /* xgen_patconv_plan with the caller's tuning (NULL = xgen_patconv_plan).  Errors as
@@ -351,6 +365,9 @@ typedef struct {
     int64_t shared_bytes;       /* dynamic shared memory per block                                 */
     int64_t workspace_bytes;    /* partial-sum workspace of the planned split, 0 if unsplit        */
     double  covered;            /* output pixels / pixel slots of all tiles (lanes x pixels each)  */
+    int32_t last_arriver;       /* split items are added up by the block that arrives last (nobody
+                                   waits) rather than by all of their blocks after a wait         */
+    int32_t reserved;
 } xgen_patconv_plan_stats;
 
 /* Fill *stats for the shape.  No CUDA work is enqueued.  Errors: INVALID_ARG, SHAPE, UNSUPPORTED. */
@@ -359,7 +376,7 @@ xgen_status xgen_patconv_plan_info(const xgen_patconv_packed *packed, int32_t n,
 
 /*
  * Testing aid, not for production use (the paper has no counterpart): make every later
- * planned split launch of the handle wait for `extra` arrivals more than its own blocks
+ * planned launch of waiting splits of the handle wait for `extra` arrivals more than its own blocks
  * will ever deliver.  With extra > 0 the wait of every block runs out after the handle's
  * wait limit (xgen_patconv_tuning.wait_limit_ms), the kernel ends normally, and
  * xgen_patconv_last_status returns XGEN_ERR_TIMEOUT once; extra = 0 restores normal

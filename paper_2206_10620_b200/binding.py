@@ -51,7 +51,7 @@ class Stats(ctypes.Structure):
 class Tuning(ctypes.Structure):
     _fields_ = [("splits", ctypes.c_int32), ("no_copy_engine", ctypes.c_int32),
                 ("no_launch_overlap", ctypes.c_int32), ("wait_limit_ms", ctypes.c_int32),
-                ("no_small_blocks", ctypes.c_int32)]
+                ("no_small_blocks", ctypes.c_int32), ("reduce_mode", ctypes.c_int32)]
 
 
 class PlanStats(ctypes.Structure):
@@ -62,7 +62,8 @@ class PlanStats(ctypes.Structure):
                 ("lanes_x", ctypes.c_int32), ("lanes_y", ctypes.c_int32),
                 ("lanes_n", ctypes.c_int32), ("pixels_per_lane", ctypes.c_int32), ("stages", ctypes.c_int32),
                 ("uses_copy_engine", ctypes.c_int32), ("shared_bytes", ctypes.c_int64),
-                ("workspace_bytes", ctypes.c_int64), ("covered", ctypes.c_double)]
+                ("workspace_bytes", ctypes.c_int64), ("covered", ctypes.c_double),
+                ("last_arriver", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 class ProbeResult(ctypes.Structure):
@@ -192,11 +193,11 @@ class Packed:
         }
 
     def plan(self, n, h, w, splits=0, no_copy_engine=False, no_launch_overlap=False, wait_limit_ms=0,
-             no_small_blocks=False):
+             no_small_blocks=False, reduce_mode=0):
         """xgen_patconv_plan, or xgen_patconv_plan_tuned when any tuning field is given."""
-        if splits or no_copy_engine or no_launch_overlap or wait_limit_ms or no_small_blocks:
+        if splits or no_copy_engine or no_launch_overlap or wait_limit_ms or no_small_blocks or reduce_mode:
             t = Tuning(int(splits), int(bool(no_copy_engine)), int(bool(no_launch_overlap)), int(wait_limit_ms),
-                       int(bool(no_small_blocks)))
+                       int(bool(no_small_blocks)), int(reduce_mode))
             _check(lib().xgen_patconv_plan_tuned(self._h, n, h, w, ctypes.byref(t)), "xgen_patconv_plan_tuned")
         else:
             _check(lib().xgen_patconv_plan(self._h, n, h, w), "xgen_patconv_plan")
@@ -204,7 +205,7 @@ class Packed:
     def plan_info(self, n, h, w) -> dict:
         s = PlanStats()
         _check(lib().xgen_patconv_plan_info(self._h, n, h, w, ctypes.byref(s)), "xgen_patconv_plan_info")
-        return {k: getattr(s, k) for k, _ in PlanStats._fields_}
+        return {k: getattr(s, k) for k, _ in PlanStats._fields_ if k != "reserved"}
 
     def test_expect_arrivals(self, extra):
         _check(lib().xgen_patconv_test_expect_arrivals(self._h, int(extra)), "xgen_patconv_test_expect_arrivals")

@@ -112,6 +112,7 @@ struct KParams {
     uint32_t *counters;
     uint32_t target;                     // counter value at which every split of an item has arrived
     int n_splits;
+    int last_reduces;                    // nobody waits: the block that arrives last adds up the whole item
     uint32_t wait_us;                    // bound of every device-side wait, microseconds
 };
 
@@ -825,11 +826,18 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
     }
 
     if (ws_rows) {
-        // ===== split item: wait for the other splits of this item, then reduce a share =====
+        // ===== split item: the partial sums of all splits of this item are added up either by
+        // all of its blocks, each taking a share once every split has arrived (they wait for each
+        // other: the planner keeps them within what the GPU holds at once), or, with any number
+        // of splits, by whichever block arrives last (nobody waits) =====
         asm volatile("griddepcontrol.wait;" ::: "memory");       // the producer warps join in here
         __threadfence();
         __syncthreads();
-        if (tid == 0) {
+        if (tid == 0 && P.last_reduces) {
+            uint32_t old;
+            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(P.counters + sitem) : "memory");
+            if (old + 1u != P.target) abort_s = 2;                // not the last one: nothing left to do
+        } else if (tid == 0) {
             uint32_t *cnt = P.counters + sitem;
             asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(cnt) : "memory");
             bool ok = false;
@@ -851,6 +859,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
         if (!abort_s) {
             const int K8 = (P.J + 7) >> 3;
             const int R = P.wpc * K8 * T, S = P.n_splits, nwarps = nthreads >> 5;
+            const int row0 = P.last_reduces ? 0 : zsplit, rstep = P.last_reduces ? 1 : S;   // this block's share of the rows
             const uint32_t *base = ws_rows + (size_t)sitem * S * R * 256;
             const size_t zstride = (size_t)R * 64;                // uint4 per split
             // the sums of row `row` (one running sum of every lane, 8 channels) over all splits, in split order
@@ -866,15 +875,15 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                     }
                 };
                 const uint4 *src = reinterpret_cast<const uint4 *>(base + ((size_t)row * 32 + lane) * 8);
-                int z = 0;
-                for (; z + 4 <= S; z += 4) {                          // four splits in flight; summed in order 0, 1, ...
+                for (int z = 0; z < S; z += 4) {                      // four splits in flight; summed in order 0, 1, ...
                     uint4 lo[4], hi[4];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) { lo[u] = __ldcg(src + (z + u) * zstride); hi[u] = __ldcg(src + (z + u) * zstride + 1); }
+                    for (int u = 0; u < 4; ++u)
+                        if (z + u < S) { lo[u] = __ldcg(src + (z + u) * zstride); hi[u] = __ldcg(src + (z + u) * zstride + 1); }
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) add8(lo[u], hi[u]);
+                    for (int u = 0; u < 4; ++u)
+                        if (z + u < S) add8(lo[u], hi[u]);
                 }
-                for (; z < S; ++z) add8(__ldcg(src + z * zstride), __ldcg(src + z * zstride + 1));
             };
             if (FUSED && P.pool) {
                 // Units of one pooled pixel: (warp's filter group, 8-channel piece, pooled pixel q).  The
@@ -884,8 +893,8 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                 const int *qtab = ptab + 32 * T;
                 uint32_t *pool_s = smem + P.plane_off_words + (size_t)(warp * 32 + lane) * 8;
                 const int per_pass = nwarps >> 2;
-                for (int u0 = zsplit; u0 < U; u0 += S * per_pass) {
-                    const int unit = u0 + S * (warp >> 2), m = warp & 3;
+                for (int u0 = row0; u0 < U; u0 += rstep * per_pass) {
+                    const int unit = u0 + rstep * (warp >> 2), m = warp & 3;
                     const bool mine = (warp >> 2) < per_pass && unit < U;
                     const int q = unit % Q, k8 = (unit / Q) % K8, w = unit / (Q * K8);
                     const int ocb = mine ? soc_s[w * P.J] : -1;
@@ -922,7 +931,7 @@ patconv_kernel(const KParams P, const __grid_constant__ CUtensorMap tmap) {
                     __syncthreads();
                 }
             } else {
-                for (int row = zsplit + S * warp; row < R; row += S * nwarps) {
+                for (int row = row0 + rstep * warp; row < R; row += rstep * nwarps) {
                     const int t = row % T, k8 = (row / T) % K8, w = row / (T * K8);
                     const int ocb = soc_s[w * P.J];
                     const int oc0 = ocb + k8 * 8;
@@ -1158,6 +1167,7 @@ struct xgen_patconv_packed {
     // set by xgen_patconv_plan: split the channel chunks of this shape across blocks
     int plan_n = 0, plan_h = 0, plan_w = 0, plan_splits = 1, plan_cps = 0;
     int plan_whole = 0;                 // items of the planned shape that run whole (the others are split)
+    bool plan_last = false;             // split items are added up by their last block to arrive (nobody waits)
     uint32_t *d_partial = nullptr;      // partial sums of the planned split, reduced inside the kernel
     size_t partial_bytes = 0;
     uint32_t *d_counters = nullptr;     // one arrival counter per (tile, filter block) of the planned shape
@@ -1557,7 +1567,8 @@ static xgen_status run_layer(const xgen_patconv_packed *h, const void *x, int32_
             std::lock_guard<std::mutex> lock(h->split_mu);
             kp.ws = h->d_partial;
             kp.counters = h->d_counters;
-            kp.target = (h->split_seq + 1u) * (uint32_t)n_splits + (uint32_t)h->hook_extra_arrivals;
+            kp.last_reduces = h->plan_last ? 1 : 0;
+            kp.target = (h->split_seq + 1u) * (uint32_t)n_splits + (h->plan_last ? 0u : (uint32_t)h->hook_extra_arrivals);
             e = cudaLaunchKernelExC(&cfg, kern, args);
             if (e == cudaSuccess) e = cudaGetLastError();
             if (e == cudaSuccess) ++h->split_seq;
@@ -1749,6 +1760,8 @@ xgen_status xgen_patconv_plan_info(const xgen_patconv_packed *h, int32_t n, int3
     out->stages = L.kp.n_stages;
     out->uses_copy_engine = L.kp.use_tma;
     out->shared_bytes = (int64_t)L.smem;
+    out->last_arriver = planned && h->plan_last ? 1 : 0;
+    out->reserved = 0;
     out->workspace_bytes = planned ? (int64_t)((size_t)(L.items - h->plan_whole) * (size_t)h->plan_splits * rows_per_item(p) * 1024) : 0;
     return XGEN_OK;
 }
@@ -1758,7 +1771,8 @@ xgen_status xgen_patconv_plan_tuned(xgen_patconv_packed *h, int32_t n, int32_t h
     if (!h) return XGEN_ERR_INVALID_ARG;
     if (n < 1 || hh < 1 || ww < 1) return XGEN_ERR_SHAPE;
     if (h->device < 0) return XGEN_ERR_CUDA;
-    if (tuning && (tuning->splits < 0 || tuning->wait_limit_ms < 0)) return XGEN_ERR_INVALID_ARG;
+    if (tuning && (tuning->splits < 0 || tuning->wait_limit_ms < 0 || tuning->reduce_mode < 0 || tuning->reduce_mode > 2))
+        return XGEN_ERR_INVALID_ARG;
     const PackedHost &p = h->host;
     const int ho = (hh + 2 - 3) / p.stride + 1, wo = (ww + 2 - 3) / p.stride + 1;
     if ((int64_t)n * ho * wo * p.c_out > 0x7FFFFFFFLL) return XGEN_ERR_SHAPE;
@@ -1843,44 +1857,59 @@ xgen_status xgen_patconv_plan_tuned(xgen_patconv_packed *h, int32_t n, int32_t h
     const int64_t capacity = std::max<int64_t>(1, (int64_t)sms * bps);
     const double slot_macs_item = 4.0 * (double)p.stats.kernels_surviving / (double)p.n_blocks * 32.0 * p.tpix;
     auto sm_rate = [&](int warps) { return 50.0 * std::pow((double)std::min(warps, 16) / 16.0, 0.65); };   // multiply-adds per cycle
+    // Cost model, cycles.  A block costs a fixed prologue and epilogue plus its multiply-adds at the
+    // rate an SM sustains with the warps it then hosts.  Waiting splits add the exchange of the
+    // partial sums (every block writes its sums, waits, and reduces a share).
+    auto parts_of = [&](int64_t k) { const int c = (int)((p.n_chunks + k - 1) / k); return (int64_t)((p.n_chunks + c - 1) / c); };
+    auto work_of = [&](int64_t k) { return slot_macs_item * (double)((p.n_chunks + k - 1) / k) / (double)p.n_chunks; };
+    const size_t ws_limit = (size_t)1 << 30;                    // no plan takes more than 1 GiB of workspace
+    auto ws_bytes = [&](int64_t n_items, int64_t k) { return (size_t)n_items * (size_t)parts_of(k) * rows_per_item(p) * 1024; };
     int64_t splits = 1, whole = L.items;
-    if (L.items <= capacity) {
-        const int64_t max_splits = std::max<int64_t>(1, std::min<int64_t>(p.n_chunks, capacity / std::max(1, L.items)));
-        auto estimate = [&](int64_t k) {
-            const int cps_k = (int)((p.n_chunks + k - 1) / k);
-            const int64_t parts = (p.n_chunks + cps_k - 1) / cps_k;
-            const int64_t blocks = L.items * parts;
-            const int per_sm = (int)((blocks + sms - 1) / sms);
-            const double work = slot_macs_item * (double)cps_k / (double)p.n_chunks;
-            double t = 9000.0 + work * per_sm / sm_rate(per_sm * p.wpc);
+    bool last = false;
+    // The splits of an item that wait for each other inside the kernel must all be resident at
+    // once: (split items) x splits <= SMs x blocks per SM.  Two cases.  Few items (not more than
+    // the GPU holds blocks): every item is split.  Many items: the GPU works through them in waves
+    // of `capacity` blocks, and the last wave is only partly filled; the items of that last wave
+    // are split (they are numbered last, so their blocks start as the wave before them drains),
+    // all earlier items run whole.
+    const bool few = L.items <= capacity;
+    const int64_t rest = few ? L.items : L.items % capacity;     // the items that may be split
+    if (rest > 0) {
+        const int64_t max_wait = std::max<int64_t>(1, std::min<int64_t>(p.n_chunks, capacity / rest));
+        auto t_wait = [&](int64_t k) {
+            const int64_t parts = parts_of(k), blocks = rest * parts;
+            const int per_sm = few ? (int)((blocks + sms - 1) / sms) : bps;
+            double t = 9000.0 + work_of(k) * (few ? per_sm : 1) / sm_rate(per_sm * p.wpc);
             if (parts > 1) t += 5000.0 + 150.0 * (double)parts;
             return t;
         };
-        double best_t = estimate(1);
-        for (int64_t k = 2; k <= max_splits; ++k) {
-            const double t = estimate(k);
-            if (t < 0.97 * best_t) { best_t = t; splits = k; }
+        const double margin = few ? 0.97 : 0.9;                  // a split has to pay for itself
+        double best_t = t_wait(1);
+        // Splits added up by the last arriver are never the planner's own choice: with more blocks
+        // than the GPU holds at once they run in waves, and on the shapes tried (items between a
+        // half and three times the SM count, 2 to 8 splits) every such plan measured slower than
+        // the best plan of whole items and waiting splits.  They are there for callers that must
+        // run planned launches of several handles at the same time (reduce_mode = 2).
+        for (int64_t k = 2; k <= max_wait; ++k) {
+            const double t = t_wait(k);
+            if (t < margin * best_t) { best_t = t; splits = k; }
         }
-        if (tn.splits >= 1) splits = std::min<int64_t>(tn.splits, max_splits);
-        whole = 0;
-    } else {
-        const int64_t rest = L.items % capacity;               // items of the last, partly filled wave
-        const int64_t max_splits = rest > 0 ? std::min<int64_t>(p.n_chunks, capacity / rest) : 1;
-        const double t_item = 9000.0 + slot_macs_item / sm_rate(bps * p.wpc);
-        double best_t = t_item;                                  // the last wave with whole items
-        for (int64_t k = 2; k <= max_splits; ++k) {
-            const int cps_k = (int)((p.n_chunks + k - 1) / k);
-            const int64_t parts = (p.n_chunks + cps_k - 1) / cps_k;
-            const double t = 9000.0 + slot_macs_item * (double)cps_k / (double)p.n_chunks / sm_rate(bps * p.wpc) +
-                             5000.0 + 150.0 * (double)parts;
-            if (t < 0.9 * best_t) { best_t = t; splits = k; }
+        last = tn.reduce_mode == 2 && splits > 1;                // the same count, nobody waiting
+        if (tn.splits >= 1) {
+            if (tn.reduce_mode == 2) {
+                last = tn.splits > 1;
+                splits = std::min<int64_t>(tn.splits, p.n_chunks);
+                while (splits > 1 && ws_bytes(rest, splits) > ws_limit) --splits;
+            } else {
+                last = false;
+                splits = std::max<int64_t>(1, std::min<int64_t>(tn.splits, max_wait));
+            }
         }
-        if (tn.splits >= 1) splits = std::max<int64_t>(1, std::min<int64_t>(tn.splits, max_splits));
         whole = splits > 1 ? L.items - rest : L.items;
     }
     const int cps = (int)((p.n_chunks + splits - 1) / splits);
     splits = (p.n_chunks + cps - 1) / cps;
-    if (splits <= 1) whole = L.items;
+    if (splits <= 1) { whole = L.items; last = false; }
     const int64_t split_items = L.items - whole;
     if (rs == XGEN_OK && cudaDeviceSynchronize() != cudaSuccess) rs = XGEN_ERR_CUDA;
     if (rs == XGEN_OK && splits > 1) {
@@ -1910,7 +1939,7 @@ xgen_status xgen_patconv_plan_tuned(xgen_patconv_packed *h, int32_t n, int32_t h
     h->tuning = tn;
     h->wait_us = tn.wait_limit_ms > 0 ? (uint32_t)std::min<int64_t>((int64_t)tn.wait_limit_ms * 1000, 60000000) : 2000000u;
     h->plan_n = n; h->plan_h = hh; h->plan_w = ww;
-    h->plan_splits = (int)splits; h->plan_cps = cps; h->plan_whole = (int)whole;
+    h->plan_splits = (int)splits; h->plan_cps = cps; h->plan_whole = (int)whole; h->plan_last = last;
     return XGEN_OK;
 }
 

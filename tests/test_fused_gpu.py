@@ -26,7 +26,7 @@ def _residual(d, ho, wo, seed):
     return r.astype(np.float32 if s.dtype == "f32" else np.float16)
 
 
-def run_fused(pk, d, relu, pool, residual=None, scale=None, zp=0, plan_splits=None):
+def run_fused(pk, d, relu, pool, residual=None, scale=None, zp=0, plan_splits=None, reduce_mode=0):
     import torch
     s = d.spec
     x = torch.from_numpy(d.x).cuda()
@@ -35,7 +35,7 @@ def run_fused(pk, d, relu, pool, residual=None, scale=None, zp=0, plan_splits=No
     step = 2 if pool == 2 else 1
     ydt = torch.uint8 if scale is not None else {"f32": torch.float32, "f16": torch.float16, "i8": torch.int32}[s.dtype]
     if plan_splits is not None:
-        pk.plan(s.n, s.h, s.w, splits=plan_splits)
+        pk.plan(s.n, s.h, s.w, splits=plan_splits, reduce_mode=reduce_mode)
     buf, y = guarded_output((s.n, ho // step, wo // step, s.c_out), ydt)
     rt = None if residual is None else torch.from_numpy(residual).cuda()
     st_ = None if scale is None else torch.from_numpy(scale).cuda()
@@ -130,6 +130,21 @@ def test_fused_behind_a_planned_split(dtype, stride):
     compare_fused(d, run_fused(pk, d, False, 0, res), False, 0, res)
     if dtype == "i8":
         scale = (wl.uniform01(4, "AUX", 10, 144) * 2e-3 + 1e-4).astype(np.float32)
+        compare_fused(d, run_fused(pk, d, True, 2, res, scale, 7), True, 2, res, scale, 7)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "i8"])
+def test_fused_behind_a_split_added_up_by_the_last_block(dtype):
+    d = _layer(dtype, 2, 128, 144, 16, 16, 1, prune=0.6, seed=43)
+    pk = pack(d)
+    res = _residual(d, 16, 16, seed=9)
+    got = run_fused(pk, d, True, 2, res, plan_splits=4, reduce_mode=2)
+    info = pk.plan_info(2, 16, 16)
+    assert info["splits"] == 4 and info["last_arriver"] == 1
+    compare_fused(d, got, True, 2, res)
+    compare_fused(d, run_fused(pk, d, False, 0, res), False, 0, res)
+    if dtype == "i8":
+        scale = (wl.uniform01(4, "AUX", 11, 144) * 2e-3 + 1e-4).astype(np.float32)
         compare_fused(d, run_fused(pk, d, True, 2, res, scale, 7), True, 2, res, scale, 7)
 
 

@@ -52,12 +52,64 @@ def test_planned_split_over_several_tiles_and_filter_blocks(dtype, stride):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "f16", "i8"])
+@pytest.mark.parametrize("stride", [1, 2])
+def test_split_added_up_by_the_last_block_to_arrive(dtype, stride):
+    """Splits that do not wait for each other: more blocks than any GPU holds at once, running in
+    waves; the block of an item that counts itself in last adds up all of its partial sums."""
+    n = 24 if stride == 1 else 40
+    d = _layer(dtype, n, 64, 72, 40, 40, stride, prune=0.6, lib=8, seed=71)
+    pk = pack(d)
+    pk.plan(n, 40, 40, splits=4, reduce_mode=2)
+    info = pk.plan_info(n, 40, 40)
+    assert info["last_arriver"] == 1 and info["splits"] == 4 and info["whole_items"] == 0
+    assert info["blocks"] == 4 * info["items"] and info["blocks"] > 160
+    before = binding.launch_count()
+    y = run_gpu(pk, d.x, d.bias, True)
+    assert binding.launch_count() - before == 1
+    compare(d, y)
+    compare(d, run_gpu(pk, d.x, None, False), bias=None, relu=False)
+    assert np.array_equal(run_gpu(pk, d.x, d.bias, True), y)        # fixed order of the additions
+    # the same sums in the same order as splits that wait (2 x 4 blocks are resident anywhere)
+    small = _layer(dtype, 1, 64, 72, 16, 16, stride, prune=0.6, lib=8, seed=72)
+    pk2 = pack(small)
+    pk2.plan(1, 16, 16, splits=4, reduce_mode=1)
+    assert pk2.plan_info(1, 16, 16)["last_arriver"] == 0
+    y_wait = run_gpu(pk2, small.x, small.bias, True)
+    pk2.plan(1, 16, 16, splits=4, reduce_mode=2)
+    assert pk2.plan_info(1, 16, 16)["last_arriver"] == 1
+    assert np.array_equal(run_gpu(pk2, small.x, small.bias, True), y_wait)
+
+
+def test_two_handles_at_once_with_splits_that_do_not_wait():
+    """Planned layers of two handles on two streams at the same time: with reduce_mode=2 no block
+    waits for another, so the launches may share the GPU in any interleaving."""
+    import torch
+    ds = [_layer("f32", 8, 64, 72, 24, 24, 1, prune=0.6, lib=8, seed=s) for s in (73, 74)]
+    pks = [pack(d) for d in ds]
+    streams = [torch.cuda.Stream() for _ in ds]
+    xs, bs, ys = [], [], []
+    for d, pk in zip(ds, pks):
+        pk.plan(8, 24, 24, splits=4, reduce_mode=2)
+        assert pk.plan_info(8, 24, 24)["last_arriver"] == 1
+        xs.append(torch.from_numpy(d.x).cuda()); bs.append(torch.from_numpy(d.bias).cuda())
+        ys.append(guarded_output((8, 24, 24, 72), torch.float32))
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for d, pk, st, x, b, (buf, y) in zip(ds, pks, streams, xs, bs, ys):
+            pk.run(x.data_ptr(), 8, 24, 24, b.data_ptr(), True, y.data_ptr(), st.cuda_stream)
+    for d, pk, st, (buf, y) in zip(ds, pks, streams, ys):
+        pk.sync(st.cuda_stream)
+        check_guards(buf)
+        compare(d, y.cpu().numpy())
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "i8"])
 def test_last_wave_is_split(dtype):
     """More items than the GPU holds blocks: the items of the last, partly filled wave are split
     (and reduced inside the kernel), all earlier items run whole -- in one launch."""
     d = _layer(dtype, 60, 32, 16, 40, 40, 1, prune=0.5, lib=8, seed=111)
     pk = pack(d)
-    pk.plan(60, 40, 40, splits=2)
+    pk.plan(60, 40, 40, splits=2, reduce_mode=1)
     info = pk.plan_info(60, 40, 40)
     assert 150 < info["items"] < 220             # 188 tiles of 32 blocks (row tiling) x 1 filter block
     if info["splits"] == 2:                      # a GPU with 148 block slots: 148 whole + 40 x 2
@@ -228,8 +280,9 @@ def test_bounded_wait_runs_out_and_the_handle_recovers():
     import torch
     d = _layer("f32", 1, 128, 32, 12, 12, 1, prune=0.5, lib=8, seed=91)
     pk = pack(d)
-    pk.plan(1, 12, 12, splits=4, wait_limit_ms=20)
-    assert pk.plan_info(1, 12, 12)["splits"] == 4
+    pk.plan(1, 12, 12, splits=4, wait_limit_ms=20, reduce_mode=1)
+    info = pk.plan_info(1, 12, 12)
+    assert info["splits"] == 4 and info["last_arriver"] == 0
     compare(d, run_gpu(pk, d.x, d.bias, True))
     pk.test_expect_arrivals(1)
     x = torch.from_numpy(d.x).cuda()
