@@ -325,6 +325,12 @@ xgen_status xgen_patconv_plan(xgen_patconv_packed *packed, int32_t n, int32_t h,
  *   no_small_blocks    keep 4x4 output pixels per thread even for shapes that the
  *                      planner would run with 4x2 pixels per thread (a single small
  *                      image); xgen_patconv_run_fused needs the 4x4 blocks
+ *   channels_per_chunk input channels staged per pipeline step: 4, 8 or 16 (the command
+ *                      stream is rebuilt and uploaded again; halved automatically while a
+ *                      block's commands of one chunk exceed their 24 KB stage)
+ *   groups_per_block   filter groups (consumer warps) per thread block, 1..16, at most the
+ *                      library's own choice: fewer groups make more, smaller blocks of
+ *                      output channels, hence more work items and fewer channel splits
  *   reduce_mode        how split items are added up: 0 or 1 by waiting splits, 2 by the
  *                      last arriver (then `splits` is clamped to the number of channel
  *                      chunks only, not to what is resident at once)
@@ -336,6 +342,8 @@ typedef struct {
     int32_t wait_limit_ms;
     int32_t no_small_blocks;
     int32_t reduce_mode;
+    int32_t channels_per_chunk;
+    int32_t groups_per_block;
 } xgen_patconv_tuning;
 
 /* xgen_patconv_plan with the caller's tuning (NULL = xgen_patconv_plan).  Errors as

@@ -51,7 +51,8 @@ class Stats(ctypes.Structure):
 class Tuning(ctypes.Structure):
     _fields_ = [("splits", ctypes.c_int32), ("no_copy_engine", ctypes.c_int32),
                 ("no_launch_overlap", ctypes.c_int32), ("wait_limit_ms", ctypes.c_int32),
-                ("no_small_blocks", ctypes.c_int32), ("reduce_mode", ctypes.c_int32)]
+                ("no_small_blocks", ctypes.c_int32), ("reduce_mode", ctypes.c_int32),
+                ("channels_per_chunk", ctypes.c_int32), ("groups_per_block", ctypes.c_int32)]
 
 
 class PlanStats(ctypes.Structure):
@@ -193,11 +194,12 @@ class Packed:
         }
 
     def plan(self, n, h, w, splits=0, no_copy_engine=False, no_launch_overlap=False, wait_limit_ms=0,
-             no_small_blocks=False, reduce_mode=0):
+             no_small_blocks=False, reduce_mode=0, channels_per_chunk=0, groups_per_block=0):
         """xgen_patconv_plan, or xgen_patconv_plan_tuned when any tuning field is given."""
-        if splits or no_copy_engine or no_launch_overlap or wait_limit_ms or no_small_blocks or reduce_mode:
+        if (splits or no_copy_engine or no_launch_overlap or wait_limit_ms or no_small_blocks or reduce_mode
+                or channels_per_chunk or groups_per_block):
             t = Tuning(int(splits), int(bool(no_copy_engine)), int(bool(no_launch_overlap)), int(wait_limit_ms),
-                       int(bool(no_small_blocks)), int(reduce_mode))
+                       int(bool(no_small_blocks)), int(reduce_mode), int(channels_per_chunk), int(groups_per_block))
             _check(lib().xgen_patconv_plan_tuned(self._h, n, h, w, ctypes.byref(t)), "xgen_patconv_plan_tuned")
         else:
             _check(lib().xgen_patconv_plan(self._h, n, h, w), "xgen_patconv_plan")

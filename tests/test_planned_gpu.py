@@ -273,6 +273,35 @@ def test_tuning_switches_keep_the_result(knob, dtype):
     assert np.array_equal(y0, y1)        # same sums in the same order, whatever stages the tiles
 
 
+@pytest.mark.parametrize("dtype,stride", [("f32", 1), ("f16", 2), ("i8", 1)])
+def test_tuned_grouping_keeps_the_result(dtype, stride):
+    """The tuning-decided parameters of a layer (channels per chunk, filter groups per block) rebuild
+    the command stream at plan time; every grouping computes the same layer."""
+    d = _layer(dtype, 2, 64, 200, 24, 24, stride, prune=0.5, lib=8, seed=83)
+    pk = pack(d)
+    pk.plan(2, 24, 24)
+    base = pk.plan_info(2, 24, 24)
+    compare(d, run_gpu(pk, d.x, d.bias, True))
+    seen = set()
+    for cc, g in ((4, 0), (16, 0), (0, 4), (8, 8), (4, 1)):
+        pk.plan(2, 24, 24, channels_per_chunk=cc, groups_per_block=g)
+        info, st = pk.plan_info(2, 24, 24), pk.stats()
+        if cc:
+            assert st["channels_per_chunk"] in (cc, cc // 2, cc // 4)    # halved while a chunk's commands overflow their stage
+        if g:
+            assert st["groups_per_block"] == min(g, base["threads_per_block"] // 32 - 4)
+            assert info["threads_per_block"] == 32 * (st["groups_per_block"] + 4)
+        seen.add((st["channels_per_chunk"], st["groups_per_block"]))
+        compare(d, run_gpu(pk, d.x, d.bias, True))
+    assert len(seen) >= 4
+    pk.plan(2, 24, 24)                               # back to the library's own grouping
+    assert pk.plan_info(2, 24, 24)["filter_blocks"] == base["filter_blocks"]
+    compare(d, run_gpu(pk, d.x, d.bias, True))
+    with pytest.raises(binding.PatconvError) as e:
+        pk.plan(2, 24, 24, channels_per_chunk=5)
+    assert e.value.status == 1
+
+
 def test_bounded_wait_runs_out_and_the_handle_recovers():
     """A planned split told to expect one arrival that never comes: every block's wait runs out
     after the (shortened) limit, the kernel ends by itself, xgen_patconv_last_status reports
