@@ -4,8 +4,9 @@ Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
 this package; the CUDA library never does, and this package never imports the
 CUDA library or its binding.
 
-`build()` compiles `patconv_ref.c` with gcc into `libpatconv_ref.so` next to
-it; `conv()` runs one layer.  Floating-point inputs (fp32 or fp16 arrays) are
+`build()` compiles `patconv_ref.c` and `blockgemm_ref.c` with gcc into
+`libpatconv_ref.so` next to them; `conv()` runs one pattern-pruned layer,
+`block_gemm()` one block-pruned matrix product.  Floating-point inputs (fp32 or fp16 arrays) are
 widened to double exactly before the call, so the oracle's result is the
 double-precision value of the layer on the stored inputs.  Parity status:
 pinned (see the header of patconv_ref.c).
@@ -20,16 +21,18 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "patconv_ref.c")
+_SRC_GEMM = os.path.join(_HERE, "blockgemm_ref.c")
 _LIB = os.path.join(_HERE, "libpatconv_ref.so")
 _lib = None
 
 
 def build(force: bool = False) -> str:
     """Compile the C oracle if the shared object is missing or stale."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    newest = max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_GEMM))
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest:
         tmp = _LIB + ".tmp%d" % os.getpid()
         subprocess.check_call(["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared",
-                               "-o", tmp, _SRC, "-lm"])
+                               "-o", tmp, _SRC, _SRC_GEMM, "-lm"])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -49,6 +52,8 @@ def _load():
         lib.patconv_ref_fused_f64.restype = I
         lib.patconv_ref_fused_i64.argtypes = [P, P, I, I, I, I, I, I, P, I, P, P]
         lib.patconv_ref_fused_i64.restype = I
+        lib.blockgemm_ref_f64.argtypes = [P, P, P, P, P, I, ctypes.c_long, I, I, I, I, P, P]
+        lib.blockgemm_ref_f64.restype = I
         _lib = lib
     return _lib
 
@@ -151,3 +156,37 @@ def conv_fused(x, w, pid, masks, bias=None, relu=False, stride=1, residual=None,
     if rc:
         raise ValueError("oracle error %d" % rc)
     return out
+
+
+def block_gemm(x, w, row_keep, col_keep, br, bc, bias=None, relu=False, with_scale=False):
+    """One block-pruned matrix product (paper Sec. 2.1, "Block-Based Pruning").
+
+    x        [M,K]    float16/32/64: one row per pixel (NHWC) or token
+    w        [Cout,K] dense; values at pruned positions are ignored
+    row_keep [ceil(Cout/br), ceil(K/bc), br] uint8, 0 = this row of the block is pruned
+    col_keep [ceil(Cout/br), ceil(K/bc), bc] uint8, 0 = this column of the block is pruned
+    bias     [Cout] or None
+    Returns y [M,Cout] float64; with `with_scale` also S = |bias| + sum |w*x| per output.
+    """
+    lib = _load()
+    x = np.asarray(x)
+    w = np.asarray(w)
+    m, k = x.shape
+    c_out = w.shape[0]
+    if w.shape != (c_out, k):
+        raise ValueError("w must be [Cout,K]")
+    nbr, nbc = (c_out + br - 1) // br, (k + bc - 1) // bc
+    rk = np.ascontiguousarray(row_keep, dtype=np.uint8)
+    ck = np.ascontiguousarray(col_keep, dtype=np.uint8)
+    if rk.shape != (nbr, nbc, br) or ck.shape != (nbr, nbc, bc):
+        raise ValueError("row_keep / col_keep must be [blocks of rows, blocks of columns, br | bc]")
+    xc = np.ascontiguousarray(x, dtype=np.float64)
+    wc = np.ascontiguousarray(w, dtype=np.float64)
+    bcst = None if bias is None else np.ascontiguousarray(bias, dtype=np.float64)
+    y = np.empty((m, c_out), dtype=np.float64)
+    s = np.empty_like(y) if with_scale else None
+    rc = lib.blockgemm_ref_f64(_ptr(xc), _ptr(wc), _ptr(rk), _ptr(ck), _ptr(bcst), int(bool(relu)),
+                               m, k, c_out, br, bc, _ptr(y), _ptr(s))
+    if rc:
+        raise ValueError("oracle error %d" % rc)
+    return (y, s) if with_scale else y

@@ -276,3 +276,117 @@ CONFIGS = {
     "resnet18": config_resnet18,
     "sweep": config_sweep,
 }
+
+
+# --- block-pruned matrix products (fully connected layers, 1x1 convolutions) ---
+@dataclasses.dataclass
+class GemmSpec:
+    """Shape and pruning recipe of one block-pruned matrix product
+    y[m, c_out] = x[m, k] . W[c_out, k]^T: W is cut into blocks of br rows x bc
+    columns, and every block keeps round(row_keep * rows) of its rows and
+    round(col_keep * columns) of its columns."""
+    name: str
+    m: int                        # rows of x: pixels of an NHWC tensor (n*h*w) or tokens
+    k: int                        # input features
+    c_out: int
+    br: int = 32
+    bc: int = 32
+    row_keep: float = 0.5
+    col_keep: float = 0.5
+    dtype: str = "f32"            # "f32" | "f16"
+    x_dist: str = "relu_normal"
+    bias_sigma: float = 0.01
+    relu: bool = True
+    index: int = 0
+
+    @property
+    def nbr(self) -> int:
+        return (self.c_out + self.br - 1) // self.br
+
+    @property
+    def nbc(self) -> int:
+        return (self.k + self.bc - 1) // self.bc
+
+    def elem_bytes(self):
+        return {"f32": (4, 4, 4), "f16": (2, 2, 2)}[self.dtype]
+
+
+@dataclasses.dataclass
+class GemmData:
+    spec: GemmSpec
+    w: np.ndarray          # [c_out, k] float32 | float16 (dense, unmasked)
+    row_keep: np.ndarray   # uint8 [nbr, nbc, br]
+    col_keep: np.ndarray   # uint8 [nbr, nbc, bc]
+    bias: np.ndarray       # [c_out] float32
+    x: np.ndarray          # [m, k] float32 | float16
+
+    def kept_weights(self) -> int:
+        """Weights that survive (edge blocks count only the rows and columns that exist)."""
+        s = self.spec
+        total = 0
+        for i in range(s.nbr):
+            rows = min(s.br, s.c_out - i * s.br)
+            for j in range(s.nbc):
+                cols = min(s.bc, s.k - j * s.bc)
+                total += int(self.row_keep[i, j, :rows].sum()) * int(self.col_keep[i, j, :cols].sum())
+        return total
+
+    def useful_macs(self) -> int:
+        return self.kept_weights() * self.spec.m
+
+    def dense_macs(self) -> int:
+        return self.spec.m * self.spec.k * self.spec.c_out
+
+    def compulsory_bytes(self) -> int:
+        bx, bw, by = self.spec.elem_bytes()
+        s = self.spec
+        return s.m * s.k * bx + s.m * s.c_out * by + self.kept_weights() * bw + 4 * s.c_out
+
+
+def _keep_exact(keys: np.ndarray, count: int) -> np.ndarray:
+    """uint8 flags keeping the `count` entries with the smallest keys."""
+    flags = np.zeros(len(keys), dtype=np.uint8)
+    flags[np.argsort(keys, kind="stable")[:count]] = 1
+    return flags
+
+
+def make_block_gemm(spec: GemmSpec, seed: int = BASE_SEED, m_override: int | None = None) -> GemmData:
+    """Draw every tensor of one block-pruned matrix product.  `m_override` draws
+    only the first rows of x (same values as the full tensor's leading rows)."""
+    L = 1000 + spec.index                         # streams apart from the convolution layers'
+    m = spec.m if m_override is None else m_override
+    ft = np.float32 if spec.dtype == "f32" else np.float16
+    sigma = math.sqrt(2.0 / max(1.0, spec.k * spec.col_keep))
+    w = (normal(seed, "W", L, spec.c_out * spec.k) * sigma).astype(ft).reshape(spec.c_out, spec.k)
+    if spec.x_dist == "relu_normal":
+        x64 = np.maximum(normal(seed, "X", L, m * spec.k), 0.0)
+    elif spec.x_dist == "upm1":
+        x64 = 2.0 * uniform01(seed, "X", L, m * spec.k) - 1.0
+    else:
+        x64 = uniform01(seed, "X", L, m * spec.k)
+    x = x64.astype(ft).reshape(m, spec.k)
+    bias = (normal(seed, "B", L, spec.c_out) * spec.bias_sigma).astype(np.float32)
+    nbr, nbc = spec.nbr, spec.nbc
+    rkeys = raw_u64(seed, "CONN", L, nbr * nbc * spec.br, sub=1).reshape(nbr, nbc, spec.br)
+    ckeys = raw_u64(seed, "CONN", L, nbr * nbc * spec.bc, sub=2).reshape(nbr, nbc, spec.bc)
+    row_keep = np.zeros((nbr, nbc, spec.br), dtype=np.uint8)
+    col_keep = np.zeros((nbr, nbc, spec.bc), dtype=np.uint8)
+    for i in range(nbr):
+        rows = min(spec.br, spec.c_out - i * spec.br)
+        for j in range(nbc):
+            cols = min(spec.bc, spec.k - j * spec.bc)
+            row_keep[i, j, :rows] = _keep_exact(rkeys[i, j, :rows], int(round(spec.row_keep * rows)))
+            col_keep[i, j, :cols] = _keep_exact(ckeys[i, j, :cols], int(round(spec.col_keep * cols)))
+    return GemmData(spec=spec, w=w, row_keep=row_keep, col_keep=col_keep, bias=bias, x=x)
+
+
+def config_resnet50_1x1(batch: int = 32, dtype: str = "f16", row_keep: float = 0.4,
+                        col_keep: float = 0.4, br: int = 32, bc: int = 32) -> list[GemmSpec]:
+    """The distinct 1x1 convolutions of ResNet-50's bottleneck blocks in matrix form
+    (rows of x = batch * pixels), block-pruned to about one sixth of the weights."""
+    shapes = [(64, 64, 56), (64, 256, 56), (256, 64, 56), (256, 128, 56), (128, 512, 28),
+              (512, 128, 28), (512, 256, 28), (256, 1024, 14), (1024, 256, 14),
+              (1024, 512, 14), (512, 2048, 7), (2048, 512, 7)]
+    return [GemmSpec(f"pw{i + 1}_{k}to{co}_{hw}", batch * hw * hw, k, co, br, bc, row_keep, col_keep,
+                     dtype, "relu_normal", 0.01, True, i)
+            for i, (k, co, hw) in enumerate(shapes)]
