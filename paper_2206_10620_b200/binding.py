@@ -26,7 +26,9 @@ EXPORTS = ["xgen_patconv_pack", "xgen_patconv_run", "xgen_patconv_run_static_scr
            "xgen_patconv_plan_tuned", "xgen_patconv_plan_info", "xgen_patconv_test_expect_arrivals",
            "xgen_patconv_out_shape", "xgen_patconv_query", "xgen_patconv_view",
            "xgen_patconv_last_status", "xgen_patconv_free", "xgen_strerror",
-           "xgen_patconv_launch_count", "xgen_patconv_probe", "xgen_patconv_run_fused"]
+           "xgen_patconv_launch_count", "xgen_patconv_probe", "xgen_patconv_run_fused",
+           "xgen_blockgemm_pack", "xgen_blockgemm_run", "xgen_blockgemm_query", "xgen_blockgemm_view",
+           "xgen_blockgemm_free"]
 
 
 class Desc(ctypes.Structure):
@@ -78,6 +80,25 @@ class Epilogue(ctypes.Structure):
                 ("requant_scale_dev", ctypes.c_void_p), ("requant_zero_point", ctypes.c_int32)]
 
 
+class GemmDesc(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_int32), ("c_out", ctypes.c_int32), ("block_rows", ctypes.c_int32),
+                ("block_cols", ctypes.c_int32), ("dtype", ctypes.c_int)]
+
+
+class GemmStats(ctypes.Structure):
+    _fields_ = [("weights_total", ctypes.c_int64), ("weights_kept", ctypes.c_int64),
+                ("weight_bytes", ctypes.c_int64), ("stream_bytes", ctypes.c_int64),
+                ("padded_slots", ctypes.c_int64), ("column_groups", ctypes.c_int64),
+                ("row_commands", ctypes.c_int64), ("rows_per_warp", ctypes.c_int32),
+                ("warps_per_block", ctypes.c_int32), ("row_blocks", ctypes.c_int32),
+                ("stage_cols", ctypes.c_int32), ("n_stages", ctypes.c_int32),
+                ("max_stage_bytes", ctypes.c_int32)]
+
+
+class GemmHostView(ctypes.Structure):
+    _fields_ = [("units", ctypes.c_void_p), ("n_units", ctypes.c_int64), ("seg_off", ctypes.c_void_p)]
+
+
 class HostView(ctypes.Structure):
     _fields_ = [("slots", ctypes.c_void_p), ("n_slots", ctypes.c_int64),
                 ("seg_off", ctypes.c_void_p), ("slot_oc", ctypes.c_void_p),
@@ -122,8 +143,14 @@ def lib():
         L.xgen_strerror.restype = ctypes.c_char_p
         L.xgen_patconv_launch_count.restype = ctypes.c_int64
         L.xgen_patconv_probe.argtypes = [ctypes.c_int, ctypes.POINTER(ProbeResult)]
+        L.xgen_blockgemm_pack.argtypes = [ctypes.POINTER(GemmDesc), P, P, P, ctypes.c_int, ctypes.POINTER(P)]
+        L.xgen_blockgemm_run.argtypes = [P, P, ctypes.c_int64, P, I, P, P]
+        L.xgen_blockgemm_query.argtypes = [P, ctypes.POINTER(GemmStats)]
+        L.xgen_blockgemm_view.argtypes = [P, ctypes.POINTER(GemmHostView)]
+        L.xgen_blockgemm_free.argtypes = [P]
+        L.xgen_blockgemm_free.restype = None
         for name in EXPORTS:
-            if name not in ("xgen_patconv_free", "xgen_strerror", "xgen_patconv_launch_count"):
+            if name not in ("xgen_patconv_free", "xgen_strerror", "xgen_patconv_launch_count", "xgen_blockgemm_free"):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -276,3 +303,55 @@ def probe(device=0) -> dict:
 
 def strerror(status: int) -> str:
     return lib().xgen_strerror(int(status)).decode()
+
+
+class BlockGemm:
+    """Owner of one xgen_blockgemm_packed handle (block-pruned matrix product)."""
+
+    def __init__(self, k, c_out, block_rows, block_cols, dtype, dense_w, row_keep, col_keep, device=0):
+        self._h = ctypes.c_void_p()
+        self.dtype = DTYPES[dtype] if isinstance(dtype, str) else int(dtype)
+        self.k, self.c_out = int(k), int(c_out)
+        want = {F32: np.float32, F16_F32ACC: np.float16}.get(self.dtype, np.float32)
+        w = np.ascontiguousarray(dense_w, dtype=want)
+        nbr, nbc = -(-c_out // block_rows), -(-k // block_cols)
+        rk = np.ascontiguousarray(row_keep, dtype=np.uint8)
+        ck = np.ascontiguousarray(col_keep, dtype=np.uint8)
+        if w.size != c_out * k or rk.size != nbr * nbc * block_rows or ck.size != nbr * nbc * block_cols:
+            raise ValueError("dense_w must be [c_out,k], row_keep [nbr,nbc,block_rows], col_keep [nbr,nbc,block_cols]")
+        d = GemmDesc(k, c_out, block_rows, block_cols, self.dtype)
+        _check(lib().xgen_blockgemm_pack(ctypes.byref(d), w.ctypes.data, rk.ctypes.data, ck.ctypes.data, int(device),
+                                         ctypes.byref(self._h)), "xgen_blockgemm_pack")
+
+    def close(self):
+        if self._h:
+            lib().xgen_blockgemm_free(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def stats(self) -> dict:
+        s = GemmStats()
+        _check(lib().xgen_blockgemm_query(self._h, ctypes.byref(s)), "xgen_blockgemm_query")
+        return {k: getattr(s, k) for k, _ in GemmStats._fields_}
+
+    def view(self):
+        """(units [n,4] uint32, seg_off int32): copies of the host image of the packed stream."""
+        v = GemmHostView()
+        _check(lib().xgen_blockgemm_view(self._h, ctypes.byref(v)), "xgen_blockgemm_view")
+        st = self.stats()
+        n_seg = st["row_blocks"] * st["n_stages"] * (st["warps_per_block"] + 1)
+        units = np.ctypeslib.as_array(ctypes.cast(v.units, ctypes.POINTER(ctypes.c_uint32)), shape=(max(v.n_units, 0) * 4,)).copy() \
+            if v.n_units > 0 else np.zeros(0, np.uint32)
+        seg = np.ctypeslib.as_array(ctypes.cast(v.seg_off, ctypes.POINTER(ctypes.c_int32)), shape=(n_seg,)).copy()
+        return units.reshape(-1, 4), seg
+
+    def run(self, x_ptr, m, bias_ptr, relu, y_ptr, stream=0):
+        """Enqueue the layer on a CUDA stream; pointers are device addresses (ints)."""
+        _check(lib().xgen_blockgemm_run(self._h, ctypes.c_void_p(x_ptr), int(m), ctypes.c_void_p(bias_ptr or None),
+                                        int(bool(relu)), ctypes.c_void_p(y_ptr), ctypes.c_void_p(stream or None)),
+               "xgen_blockgemm_run")

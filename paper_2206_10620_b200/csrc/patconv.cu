@@ -1013,6 +1013,7 @@ patconv_reduce_kernel(const uint32_t *__restrict__ partial, int splits, size_t o
 
 // ---- host side ----------------------------------------------------------------------
 static std::atomic<int64_t> g_launches{0};
+void count_launch() { g_launches.fetch_add(1); }
 
 // The one environment switch, read once when the library is first used.
 static bool log_enabled() {

@@ -63,4 +63,7 @@ xgen_status pack_host(const xgen_patconv_desc &desc, const void *dense_w, const 
 // Rebuild slots / seg_off / slot_oc / stats of an already parsed layer for a grouping.
 xgen_status build_layout(PackedHost &p, const PackConfig &cfg);
 
+// Every kernel launch of the library counts itself here (xgen_patconv_launch_count).
+void count_launch();
+
 }  // namespace patconv
