@@ -260,6 +260,60 @@ def layer_bounds(s, fp32_tflops, dp4a_tmacs, hbm_gbs):
     return t_fp32, t_dp4a, t_hbm
 
 
+def time_block_gemm(torch, binding, dev, stream, flush, fp32_tflops, hbm_gbs, oracle_check=True, only="", reps=5):
+    """Times xgen_blockgemm_run on the 1x1 layers of ResNet-50 in matrix form.  Per layer: median
+    microseconds, useful TFLOP/s (kept weights only), the fraction of the fp32 FMA pipe and of the
+    binding roofline (the slower of kept multiply-adds on that pipe and compulsory bytes at HBM rate)."""
+    out = {"layers": [], "recipe": "ResNet-50 1x1 convolutions as [batch*pixels, c_in] x [c_out, c_in]^T, batch 32, fp16 storage, "
+                                   "32x32 pruning blocks, 40 % of rows and 40 % of columns kept per block"}
+    t_all = ideal_all = flops_all = 0.0
+    for spec in wl.config_resnet50_1x1():
+        if only and not spec.name.startswith(only):
+            continue
+        d = wl.make_block_gemm(spec)
+        pk = binding.BlockGemm(spec.k, spec.c_out, spec.br, spec.bc, spec.dtype, d.w, d.row_keep, d.col_keep, device=dev.index)
+        x = torch.from_numpy(d.x).to(dev)
+        b = torch.from_numpy(d.bias).to(dev)
+        y = torch.empty((spec.m, spec.c_out), dtype=x.dtype, device=dev)
+        for _ in range(3):
+            pk.run(x.data_ptr(), spec.m, b.data_ptr(), True, y.data_ptr(), stream)
+        torch.cuda.synchronize()
+        ts = []
+        for r in range(reps):
+            flush.fill_(r)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            pk.run(x.data_ptr(), spec.m, b.data_ptr(), True, y.data_ptr(), stream)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        us = float(np.median(ts)) * 1e3
+        macs = d.useful_macs()
+        t_alu = 2.0 * macs / (fp32_tflops * 1e12)
+        t_hbm = d.compulsory_bytes() / (hbm_gbs * 1e9)
+        rec = {"layer": spec.name, "rows": spec.m, "us": round(us, 2), "useful_tflops": round(2.0 * macs / us * 1e-6, 2),
+               "dense_equiv_tflops": round(2.0 * d.dense_macs() / us * 1e-6, 2),
+               "frac_of_fp32_pipe": round(t_alu * 1e6 / us, 4), "bound": "alu" if t_alu >= t_hbm else "hbm",
+               "ideal_us": round(max(t_alu, t_hbm) * 1e6, 2), "frac_of_binding_roofline": round(max(t_alu, t_hbm) * 1e6 / us, 4)}
+        if oracle_check and spec.m <= 8192:
+            import oracle
+            got = y[:256].cpu().numpy().astype(np.float64)
+            ref, S = oracle.block_gemm(d.x[:256], d.w, d.row_keep, d.col_keep, spec.br, spec.bc, bias=d.bias, relu=True, with_scale=True)
+            rec["parity_ok"] = bool((np.abs(got - ref) <= 2e-3 * np.maximum(np.abs(ref), 0.01 * S) + 1e-30).all())
+        out["layers"].append(rec)
+        t_all += us
+        ideal_all += max(t_alu, t_hbm) * 1e6
+        flops_all += 2.0 * macs
+        del pk, x, b, y
+    torch.cuda.empty_cache()
+    if t_all > 0:
+        out["total_us"] = round(t_all, 1)
+        out["useful_tflops"] = round(flops_all / t_all * 1e-6, 2)
+        out["frac_of_fp32_pipe"] = round(flops_all / t_all * 1e-6 / fp32_tflops, 4)
+        out["frac_of_binding_roofline"] = round(ideal_all / t_all, 4)
+    return out
+
+
 def run_gpu(args):
     import torch
     from paper_2206_10620_b200 import binding
@@ -285,6 +339,13 @@ def run_gpu(args):
     fp32_peak = max(probe["ffma_tflops"], probe["ffma2_tflops"])
     dp4a_peak = probe["dp4a_tmacs"]
     hbm, hbm_src = measured_hbm_gbs()
+
+    if args.block_gemm_only:                        # profiling aid: one layer of the matrix products, nothing else
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        rec = time_block_gemm(torch, binding, dev, torch.cuda.current_stream().cuda_stream, flush, fp32_peak, hbm,
+                              oracle_check=False, only=args.block_gemm_only, reps=3)
+        print(json.dumps({"block_gemm": rec, "measured_peaks": probe}), flush=True)
+        return
 
     specs = workload(args.workload)
     if args.only:
@@ -510,6 +571,13 @@ def run_gpu(args):
         del stk, codes, scales
         torch.cuda.empty_cache()
 
+    # --- the block-pruned matrix product on ResNet-50's 1x1 convolutions (batch 32, fp16 storage,
+    # 32 x 32 blocks keeping 40 % of their rows and 40 % of their columns: about one sixth of the
+    # weights), each layer alone after an L2 flush
+    block_gemm = {}
+    if rank == 0 and world == 1 and not args.no_configs and args.workload == "vgg16" and not args.only:
+        block_gemm = time_block_gemm(torch, binding, dev, stream, flush, fp32_peak, hbm, oracle_check=not args.no_parity)
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu = oracle_sample(specs, budget_s=args.cpu_seconds)
@@ -529,7 +597,8 @@ def run_gpu(args):
                 "net_ms_per_batch": ms,
                 "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e,
                 "roofline": roofline, "measured_peaks": probe, "host_us_per_run_call": round(host_us, 2),
-                "parity_checked": parity_checked, "cpu_baseline": cpu, "per_layer": per_layer, "configs": configs, "fused": fused}
+                "parity_checked": parity_checked, "cpu_baseline": cpu, "per_layer": per_layer, "configs": configs, "fused": fused,
+                "block_gemm": block_gemm}
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -549,6 +618,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--no-configs", action="store_true", help="skip the other named workloads")
     ap.add_argument("--no-parity", action="store_true", help="skip the oracle comparison of the timed layers")
+    ap.add_argument("--block-gemm-only", default="", help="time only this layer of the block-pruned matrix products "
+                    "(a prefix of its name, e.g. pw5) and print its record: profiling aid")
     ap.add_argument("--only", default="", help="comma-separated layer names: restrict the stack (profiling aid)")
     args = ap.parse_args()
     if args.impl == "reference":

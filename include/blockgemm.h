@@ -35,6 +35,10 @@ typedef struct {
     int32_t block_cols;     /* columns of a pruning block, >= 1 (likewise at the right edge) */
     xgen_dtype dtype;       /* XGEN_F32 (x, W, y fp32) or XGEN_F16_F32ACC (x, W, y IEEE fp16, bias
                                fp32, sums in fp32, one round-to-nearest-even at the store)  */
+    int32_t warps_per_block; /* tuning-decided (paper Sec. 2.3: the layerwise representation carries
+                               such parameters): warps of a thread block, 16 output channels each;
+                               0 = the library's choice, else 1..16.  Fewer warps make smaller
+                               thread blocks, of which an SM holds several at a time            */
 } xgen_blockgemm_desc;
 
 /* What xgen_blockgemm_query reports. */

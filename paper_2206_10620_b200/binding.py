@@ -82,7 +82,7 @@ class Epilogue(ctypes.Structure):
 
 class GemmDesc(ctypes.Structure):
     _fields_ = [("k", ctypes.c_int32), ("c_out", ctypes.c_int32), ("block_rows", ctypes.c_int32),
-                ("block_cols", ctypes.c_int32), ("dtype", ctypes.c_int)]
+                ("block_cols", ctypes.c_int32), ("dtype", ctypes.c_int), ("warps_per_block", ctypes.c_int32)]
 
 
 class GemmStats(ctypes.Structure):
@@ -308,7 +308,8 @@ def strerror(status: int) -> str:
 class BlockGemm:
     """Owner of one xgen_blockgemm_packed handle (block-pruned matrix product)."""
 
-    def __init__(self, k, c_out, block_rows, block_cols, dtype, dense_w, row_keep, col_keep, device=0):
+    def __init__(self, k, c_out, block_rows, block_cols, dtype, dense_w, row_keep, col_keep, device=0,
+                 warps_per_block=0):
         self._h = ctypes.c_void_p()
         self.dtype = DTYPES[dtype] if isinstance(dtype, str) else int(dtype)
         self.k, self.c_out = int(k), int(c_out)
@@ -319,7 +320,7 @@ class BlockGemm:
         ck = np.ascontiguousarray(col_keep, dtype=np.uint8)
         if w.size != c_out * k or rk.size != nbr * nbc * block_rows or ck.size != nbr * nbc * block_cols:
             raise ValueError("dense_w must be [c_out,k], row_keep [nbr,nbc,block_rows], col_keep [nbr,nbc,block_cols]")
-        d = GemmDesc(k, c_out, block_rows, block_cols, self.dtype)
+        d = GemmDesc(k, c_out, block_rows, block_cols, self.dtype, int(warps_per_block))
         _check(lib().xgen_blockgemm_pack(ctypes.byref(d), w.ctypes.data, rk.ctypes.data, ck.ctypes.data, int(device),
                                          ctypes.byref(self._h)), "xgen_blockgemm_pack")
 

@@ -60,7 +60,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
             raise subprocess.CalledProcessError(job.returncode, "nvcc -c (%s)" % obj)
         os.replace(obj + ".tmp", obj)
     tmp = LIB_PATH + ".tmp%d" % os.getpid()
-    subprocess.check_call([nvcc, "-shared", "-o", tmp] + objs)
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp] + objs)
     os.replace(tmp, LIB_PATH)
     return LIB_PATH
 

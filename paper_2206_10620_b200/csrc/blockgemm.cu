@@ -41,6 +41,7 @@ constexpr int kRowsPerWarp = 16;       // output channels a warp accumulates
 constexpr int kPixPerLane = 8;         // rows of x a lane owns: lane, lane + 32, ...
 constexpr int kTileM = 32 * kPixPerLane;
 constexpr int kMaxWarps = 16;
+constexpr int kDefaultWarps = 8;       // two such thread blocks share an SM and overlap their phases
 constexpr int kGroupCols = 8;          // columns of one activation load
 constexpr int kRowUnits = 3;           // 16-byte units of a row command: header, weights 0..3, weights 4..7
 constexpr int kSmemLimit = 220 * 1024;
@@ -169,7 +170,7 @@ static size_t raw_pitch_words(xgen_dtype dt, int ks) {
 }
 
 static size_t smem_bytes(const Host &h) {
-    return 2 * (size_t)kTileM * raw_pitch_words(h.dtype, h.ks) * 4 + 2 * (size_t)std::max(h.max_stage_units, 1) * 16;
+    return 2 * (size_t)kTileM * raw_pitch_words(h.dtype, h.ks) * 4 + 2 * (size_t)(h.max_stage_units + 1) * 16;   // + 1: the look-ahead of the last command
 }
 
 struct GParams {
@@ -264,11 +265,16 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) blockgemm_kernel(const GPar
     const int32_t *seg_g = P.seg_off + (size_t)rb * P.ns * (P.warps + 1);
 
     // Stage s: copy the tile's rows of x for columns [s*ks, s*ks + ks) and the block's commands.
-    auto issue = [&](int s, int buf, int &my_b, int &my_e) {
-        const int32_t *sg = seg_g + (size_t)s * (P.warps + 1);
-        const int seg_b = sg[0], seg_e = sg[P.warps];
-        my_b = sg[warp] - seg_b;
-        my_e = sg[warp + 1] - seg_b;
+    // Where a stage's commands lie: the whole block's piece and this warp's part of it.
+    auto load_seg = [&](int s, int &seg_b, int &seg_e, int &my_b, int &my_e) {
+        if (s < P.ns) {
+            const int32_t *sg = seg_g + (size_t)s * (P.warps + 1);
+            seg_b = sg[0]; seg_e = sg[P.warps];
+            my_b = sg[warp] - seg_b;
+            my_e = sg[warp + 1] - seg_b;
+        }
+    };
+    auto issue = [&](int s, int buf, int seg_b, int seg_e) {
         uint4 *cdst = cmd + (size_t)buf * P.cmd_units;
         for (int u = tid; u < seg_e - seg_b; u += nthreads) cp_async16(smem_u32(cdst + u), P.stream + seg_b + u);
         uint32_t *rdst = raw + (size_t)buf * kTileM * pitch;
@@ -311,14 +317,22 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) blockgemm_kernel(const GPar
         cp_async_commit();
     };
 
-    int nb = 0, ne = 0;
-    issue(0, 0, nb, ne);
+    // The offsets of a stage are fetched one iteration before its copies are issued, so that
+    // their latency is not waited for.
+    int sb = 0, se = 0, nb = 0, ne = 0, sb2 = 0, se2 = 0, nb2 = 0, ne2 = 0;
+    load_seg(0, sb, se, nb, ne);
+    load_seg(1, sb2, se2, nb2, ne2);
+    issue(0, 0, sb, se);
     for (int s = 0; s < P.ns; ++s) {
         const int buf = s & 1;
         const int my_b = nb, my_e = ne;
         cp_async_wait_all();
         __syncthreads();                 // stage s has landed; everybody has left stage s - 1
-        if (s + 1 < P.ns) issue(s + 1, buf ^ 1, nb, ne);
+        if (s + 1 < P.ns) {
+            issue(s + 1, buf ^ 1, sb2, se2);
+            nb = nb2; ne = ne2;
+            load_seg(s + 2, sb2, se2, nb2, ne2);
+        }
 
         const uint4 *cp = cmd + (size_t)buf * P.cmd_units + my_b;
         const uint4 *ce = cmd + (size_t)buf * P.cmd_units + my_e;
@@ -346,25 +360,27 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) blockgemm_kernel(const GPar
                 }
             }
             const uint4 *rp = cp + 1;
+            uint32_t tcol = rp[0].x;
             for (uint32_t r = 0; r < hd.x; ++r, rp += kRowUnits) {
-                const uint32_t tcol = rp[0].x;
-                const uint4 wa = rp[1], wb = rp[2];
                 uint32_t a[8];
                 tmem_ld8(tw + tcol, a);
+                const uint4 wa = rp[1], wb = rp[2];
                 const uint32_t wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+                const uint32_t tcol_here = tcol;
+                tcol = rp[kRowUnits].x;          // the next command's row (a spare unit lies behind the last one)
                 tmem_wait_ld();
                 unsigned long long acc[4];
 #pragma unroll
                 for (int t = 0; t < 4; ++t) acc[t] = pack2(a[2 * t], a[2 * t + 1]);
 #pragma unroll
                 for (int i = 0; i < kGroupCols; ++i) {
-                    const unsigned long long ww = pack2(wv[i], wv[i]);
+                    const unsigned long long ww = pack2(wv[i], wv[i]);   // the same weight for both rows of x
 #pragma unroll
                     for (int t = 0; t < 4; ++t) acc[t] = fma2(xr[i][t], ww, acc[t]);
                 }
 #pragma unroll
                 for (int t = 0; t < 4; ++t) unpack2(acc[t], a[2 * t], a[2 * t + 1]);
-                tmem_st8(tw + tcol, a);
+                tmem_st8(tw + tcol_here, a);
             }
             cp = rp;
         }
@@ -453,6 +469,7 @@ xgen_status xgen_blockgemm_pack(const xgen_blockgemm_desc *d, const void *dense_
     *out = nullptr;
     if (d->k < 1 || d->c_out < 1 || d->block_rows < 1 || d->block_cols < 1) return XGEN_ERR_INVALID_ARG;
     if (d->dtype != XGEN_F32 && d->dtype != XGEN_F16_F32ACC) return XGEN_ERR_UNSUPPORTED;
+    if (d->warps_per_block < 0 || d->warps_per_block > kMaxWarps) return XGEN_ERR_INVALID_ARG;
     if ((int64_t)d->k * d->c_out > (int64_t)1 << 28) return XGEN_ERR_SHAPE;
     xgen_blockgemm_packed *h = new (std::nothrow) xgen_blockgemm_packed();
     if (!h) return XGEN_ERR_ALLOC;
@@ -460,7 +477,7 @@ xgen_status xgen_blockgemm_pack(const xgen_blockgemm_desc *d, const void *dense_
     try {
         H.k = d->k; H.c_out = d->c_out; H.br = d->block_rows; H.bc = d->block_cols; H.dtype = d->dtype;
         const int groups = (d->c_out + kRowsPerWarp - 1) / kRowsPerWarp;
-        H.warps = std::min(groups, kMaxWarps);
+        H.warps = std::min(groups, d->warps_per_block > 0 ? d->warps_per_block : kDefaultWarps);
         H.rows_per_block = H.warps * kRowsPerWarp;
         H.n_rb = (d->c_out + H.rows_per_block - 1) / H.rows_per_block;
         std::vector<float> w((size_t)d->k * d->c_out);
@@ -540,7 +557,7 @@ xgen_status xgen_blockgemm_run(const xgen_blockgemm_packed *hc, const void *x, i
     P.relu = relu ? 1 : 0;
     P.async_x = (((uintptr_t)x % 4) == 0 && (H.dtype == XGEN_F32 || H.k % 2 == 0)) ? 1 : 0;
     P.vec_y = (((uintptr_t)y % 16) == 0 && (H.c_out * eb) % 16 == 0) ? 1 : 0;
-    P.cmd_units = std::max(H.max_stage_units, 1);
+    P.cmd_units = H.max_stage_units + 1;
     const int cols = ((H.warps + 3) / 4) * kRowsPerWarp * kPixPerLane;
     P.tmem_cols = cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
     const size_t smem = smem_bytes(H);
