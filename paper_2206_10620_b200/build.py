@@ -10,7 +10,7 @@ _CSRC = os.path.join(_HERE, "csrc")
 _INC = os.path.join(os.path.dirname(_HERE), "include")
 LIB_PATH = os.path.join(_HERE, "libpatconv.so")
 _SOURCES = ["patconv.cu", "blockgemm.cu", "probe.cu", "pack.cpp"]
-_DEPS = _SOURCES + ["patconv_internal.h", "gen_core.py", os.path.join(_INC, "patconv.h"),
+_DEPS = _SOURCES + ["patconv_internal.h", "gen_core.py", "gen_blockgemm.py", os.path.join(_INC, "patconv.h"),
                     os.path.join(_INC, "blockgemm.h")]
 
 
@@ -18,7 +18,8 @@ _OBJ_DIR = os.path.join(_HERE, "_build")
 # what each source includes besides itself
 _INCLUDES = {
     "patconv.cu": ["patconv_internal.h", "gen_core.py", os.path.join(_INC, "patconv.h")],
-    "blockgemm.cu": ["patconv_internal.h", os.path.join(_INC, "patconv.h"), os.path.join(_INC, "blockgemm.h")],
+    "blockgemm.cu": ["patconv_internal.h", "gen_blockgemm.py", os.path.join(_INC, "patconv.h"),
+                     os.path.join(_INC, "blockgemm.h")],
     "probe.cu": [os.path.join(_INC, "patconv.h")],
     "pack.cpp": ["patconv_internal.h", os.path.join(_INC, "patconv.h")],
 }
@@ -42,6 +43,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB_PATH
     gen = os.path.join(_CSRC, "core_gen.inc")
     subprocess.check_call([sys.executable, os.path.join(_CSRC, "gen_core.py"), gen])
+    subprocess.check_call([sys.executable, os.path.join(_CSRC, "gen_blockgemm.py"),
+                           os.path.join(_CSRC, "blockgemm_core.inc")])
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     os.makedirs(_OBJ_DIR, exist_ok=True)
     flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",

@@ -15,6 +15,9 @@
 //    fetches the row it addresses, adds 8 columns x 8 rows of x to it with two-wide fp32
 //    FMAs, and puts it back.
 //
+// A row command is three 16-byte units (header, weights 0..3, weights 4..7); gen_blockgemm.py
+// holds the code that interprets them.
+//
 // The packer turns every (warp, stage) into a list of column groups (up to eight kept columns
 // of one pruning block, padded with a column that reads zeros) each followed by one command
 // per kept row with the eight weights.  Pruned rows and columns cost nothing at run time.
@@ -33,6 +36,7 @@
 #include <vector>
 
 #include "blockgemm.h"
+#include "blockgemm_core.inc"
 #include "patconv_internal.h"
 
 namespace blockgemm {
@@ -43,7 +47,6 @@ constexpr int kTileM = 32 * kPixPerLane;
 constexpr int kMaxWarps = 16;
 constexpr int kDefaultWarps = 8;       // two such thread blocks share an SM and overlap their phases
 constexpr int kGroupCols = 8;          // columns of one activation load
-constexpr int kRowUnits = 3;           // 16-byte units of a row command: header, weights 0..3, weights 4..7
 constexpr int kSmemLimit = 220 * 1024;
 
 struct Host {
@@ -274,44 +277,54 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) blockgemm_kernel(const GPar
             my_e = sg[warp + 1] - seg_b;
         }
     };
+    // Asynchronous staging, 4 bytes per copy: a thread always copies the same 4-byte unit of a row,
+    // for rows rows_step apart, so its addresses advance by constants.
+    constexpr int kUnits = DT == XGEN_F32 ? KS : KS / 2;          // 4-byte units of a staged row
+    constexpr int kUnitElems = DT == XGEN_F32 ? 1 : 2;
+    const int esz = DT == XGEN_F32 ? 4 : 2;
+    const int a_row0 = tid / kUnits, a_unit = tid % kUnits;
+    const int rows_step = nthreads / kUnits;
+    const int a_iters = (kTileM + rows_step - 1) / rows_step;
+    const long long a_left = min(P.m - m0, (long long)kTileM) - a_row0;   // rows of the tile from this thread's first row on
+    const int a_lim = a_left <= 0 ? 0 : (int)min((long long)a_iters, (a_left + rows_step - 1) / rows_step);
+    const char *a_src0 = static_cast<const char *>(P.x) + ((size_t)(m0 + a_row0) * P.k + (size_t)a_unit * kUnitElems) * esz;
+    const size_t a_src_step = (size_t)rows_step * P.k * esz;
+    const uint32_t a_dst0 = smem_u32(raw) + (uint32_t)(a_row0 * pitch + a_unit) * 4u;
+    const uint32_t a_dst_step = (uint32_t)(rows_step * pitch) * 4u;
+
     auto issue = [&](int s, int buf, int seg_b, int seg_e) {
         uint4 *cdst = cmd + (size_t)buf * P.cmd_units;
         for (int u = tid; u < seg_e - seg_b; u += nthreads) cp_async16(smem_u32(cdst + u), P.stream + seg_b + u);
         uint32_t *rdst = raw + (size_t)buf * kTileM * pitch;
         const int c0 = s * KS;
-        if (DT == XGEN_F32) {
+        if (P.async_x) {
+            const bool col_ok = c0 + a_unit * kUnitElems < P.k;
+            const char *src = a_src0 + (size_t)c0 * esz;
+            uint32_t dst = a_dst0 + (uint32_t)buf * (uint32_t)(kTileM * pitch * 4);
+#pragma unroll 4
+            for (int i = 0; i < a_iters; ++i) {
+                const bool ok = col_ok && i < a_lim;
+                if (a_row0 + i * rows_step < kTileM)     // (a tile's rows need not divide among the threads)
+                    cp_async4(dst, ok ? (const void *)src : P.x, ok ? 4 : 0);
+                src += a_src_step;
+                dst += a_dst_step;
+            }
+        } else if (DT == XGEN_F32) {
             const float *x = static_cast<const float *>(P.x);
             constexpr int total = kTileM * KS;
-            if (P.async_x) {
-                for (int e = tid; e < total; e += nthreads) {
-                    const int p = e >> ks_log, c = e & (KS - 1);
-                    const bool ok = (m0 + p < P.m) && (c0 + c < P.k);
-                    cp_async4(smem_u32(rdst + (size_t)p * pitch + c), ok ? (const void *)(x + (size_t)(m0 + p) * P.k + c0 + c) : P.x, ok ? 4 : 0);
-                }
-            } else {
-                for (int e = tid; e < total; e += nthreads) {
-                    const int p = e >> ks_log, c = e & (KS - 1);
-                    const bool ok = (m0 + p < P.m) && (c0 + c < P.k);
-                    rdst[(size_t)p * pitch + c] = ok ? __float_as_uint(x[(size_t)(m0 + p) * P.k + c0 + c]) : 0u;
-                }
+            for (int e = tid; e < total; e += nthreads) {
+                const int p = e >> ks_log, c = e & (KS - 1);
+                const bool ok = (m0 + p < P.m) && (c0 + c < P.k);
+                rdst[(size_t)p * pitch + c] = ok ? __float_as_uint(x[(size_t)(m0 + p) * P.k + c0 + c]) : 0u;
             }
         } else {
             const __half *x = static_cast<const __half *>(P.x);
-            if (P.async_x) {                 // two halves per copy: k and the row starts are even
-                constexpr int total = kTileM * (KS / 2);
-                for (int e = tid; e < total; e += nthreads) {
-                    const int p = e >> (ks_log - 1), c = 2 * (e & (KS / 2 - 1));
-                    const bool ok = (m0 + p < P.m) && (c0 + c < P.k);
-                    cp_async4(smem_u32(rdst + (size_t)p * pitch + c / 2), ok ? (const void *)(x + (size_t)(m0 + p) * P.k + c0 + c) : P.x, ok ? 4 : 0);
-                }
-            } else {
-                unsigned short *rh = reinterpret_cast<unsigned short *>(rdst);
-                constexpr int total = kTileM * KS;
-                for (int e = tid; e < total; e += nthreads) {
-                    const int p = e >> ks_log, c = e & (KS - 1);
-                    const bool ok = (m0 + p < P.m) && (c0 + c < P.k);
-                    rh[(size_t)p * pitch * 2 + c] = ok ? __half_as_ushort(x[(size_t)(m0 + p) * P.k + c0 + c]) : (unsigned short)0;
-                }
+            unsigned short *rh = reinterpret_cast<unsigned short *>(rdst);
+            constexpr int total = kTileM * KS;
+            for (int e = tid; e < total; e += nthreads) {
+                const int p = e >> ks_log, c = e & (KS - 1);
+                const bool ok = (m0 + p < P.m) && (c0 + c < P.k);
+                rh[(size_t)p * pitch * 2 + c] = ok ? __half_as_ushort(x[(size_t)(m0 + p) * P.k + c0 + c]) : (unsigned short)0;
             }
         }
         cp_async_commit();
@@ -334,55 +347,18 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) blockgemm_kernel(const GPar
             load_seg(s + 2, sb2, se2, nb2, ne2);
         }
 
-        const uint4 *cp = cmd + (size_t)buf * P.cmd_units + my_b;
-        const uint4 *ce = cmd + (size_t)buf * P.cmd_units + my_e;
-        const uint32_t *rsrc = raw + (size_t)buf * kTileM * pitch + (size_t)lane * pitch;
-        while (cp < ce) {
-            const uint4 hd = *cp;
-            tmem_wait_st();              // no write to a row is in flight when it is fetched again
-            unsigned long long xr[kGroupCols][kPixPerLane / 2];
-#pragma unroll
-            for (int i = 0; i < kGroupCols; ++i) {
-                const uint32_t ci = ((i < 4 ? hd.y : hd.z) >> (8 * (i & 3))) & 0xffu;
-                if (DT == XGEN_F32) {
-                    const uint32_t *src = rsrc + ci;
-#pragma unroll
-                    for (int t = 0; t < kPixPerLane / 2; ++t)
-                        xr[i][t] = pack2(src[(size_t)(2 * t) * 32 * pitch], src[(size_t)(2 * t + 1) * 32 * pitch]);
-                } else {
-                    const unsigned short *src = reinterpret_cast<const unsigned short *>(rsrc) + ci;
-#pragma unroll
-                    for (int t = 0; t < kPixPerLane / 2; ++t) {
-                        const float a = __half2float(__ushort_as_half(src[(size_t)(2 * t) * 64 * pitch]));
-                        const float b = __half2float(__ushort_as_half(src[(size_t)(2 * t + 1) * 64 * pitch]));
-                        xr[i][t] = pack2(__float_as_uint(a), __float_as_uint(b));
-                    }
-                }
-            }
-            const uint4 *rp = cp + 1;
-            uint32_t tcol = rp[0].x;
-            for (uint32_t r = 0; r < hd.x; ++r, rp += kRowUnits) {
-                uint32_t a[8];
-                tmem_ld8(tw + tcol, a);
-                const uint4 wa = rp[1], wb = rp[2];
-                const uint32_t wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
-                const uint32_t tcol_here = tcol;
-                tcol = rp[kRowUnits].x;          // the next command's row (a spare unit lies behind the last one)
-                tmem_wait_ld();
-                unsigned long long acc[4];
-#pragma unroll
-                for (int t = 0; t < 4; ++t) acc[t] = pack2(a[2 * t], a[2 * t + 1]);
-#pragma unroll
-                for (int i = 0; i < kGroupCols; ++i) {
-                    const unsigned long long ww = pack2(wv[i], wv[i]);   // the same weight for both rows of x
-#pragma unroll
-                    for (int t = 0; t < 4; ++t) acc[t] = fma2(xr[i][t], ww, acc[t]);
-                }
-#pragma unroll
-                for (int t = 0; t < 4; ++t) unpack2(acc[t], a[2 * t], a[2 * t + 1]);
-                tmem_st8(tw + tcol_here, a);
-            }
-            cp = rp;
+        // The warp's commands of this stage, interpreted by the generated code (gen_blockgemm.py).
+        uint32_t cp = smem_u32(cmd + (size_t)buf * P.cmd_units + my_b);
+        const uint32_t ce = smem_u32(cmd + (size_t)buf * P.cmd_units + my_e);
+        const uint32_t xbase = smem_u32(raw + (size_t)buf * kTileM * pitch + (size_t)lane * pitch);
+        if (DT == XGEN_F32) {
+            if (KS == 32) BLOCKGEMM_CORE_F32_KS32(cp, ce, xbase, tw);
+            else if (KS == 16) BLOCKGEMM_CORE_F32_KS16(cp, ce, xbase, tw);
+            else BLOCKGEMM_CORE_F32_KS8(cp, ce, xbase, tw);
+        } else {
+            if (KS == 32) BLOCKGEMM_CORE_F16_KS32(cp, ce, xbase, tw);
+            else if (KS == 16) BLOCKGEMM_CORE_F16_KS16(cp, ce, xbase, tw);
+            else BLOCKGEMM_CORE_F16_KS8(cp, ce, xbase, tw);
         }
     }
     tmem_wait_st();
