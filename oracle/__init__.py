@@ -6,7 +6,8 @@ CUDA library or its binding.
 
 `build()` compiles `patconv_ref.c` and `blockgemm_ref.c` with gcc into
 `libpatconv_ref.so` next to them; `conv()` runs one pattern-pruned layer,
-`block_gemm()` one block-pruned matrix product.  Floating-point inputs (fp32 or fp16 arrays) are
+`block_gemm()` one block-pruned matrix product, `depthwise()` one
+pattern-pruned depthwise layer.  Floating-point inputs (fp32 or fp16 arrays) are
 widened to double exactly before the call, so the oracle's result is the
 double-precision value of the layer on the stored inputs.  Parity status:
 pinned (see the header of patconv_ref.c).
@@ -54,6 +55,8 @@ def _load():
         lib.patconv_ref_fused_i64.restype = I
         lib.blockgemm_ref_f64.argtypes = [P, P, P, P, P, I, ctypes.c_long, I, I, I, I, P, P]
         lib.blockgemm_ref_f64.restype = I
+        lib.dwconv_ref_f64.argtypes = [P, P, P, P, I, P, I, I, I, I, I, I, P, P]
+        lib.dwconv_ref_f64.restype = I
         _lib = lib
     return _lib
 
@@ -187,6 +190,38 @@ def block_gemm(x, w, row_keep, col_keep, br, bc, bias=None, relu=False, with_sca
     s = np.empty_like(y) if with_scale else None
     rc = lib.blockgemm_ref_f64(_ptr(xc), _ptr(wc), _ptr(rk), _ptr(ck), _ptr(bcst), int(bool(relu)),
                                m, k, c_out, br, bc, _ptr(y), _ptr(s))
+    if rc:
+        raise ValueError("oracle error %d" % rc)
+    return (y, s) if with_scale else y
+
+
+def depthwise(x, w, pid, masks, bias=None, relu=False, stride=1, with_scale=False):
+    """One depthwise pattern-pruned 3x3 layer, padding 1: every channel has one 3x3 kernel.
+
+    x     [N,H,W,C] float16/32/64
+    w     [C,3,3]   dense; values at pruned taps are ignored
+    pid   [C] int16 pattern id per channel, -1 = the channel's kernel is removed
+    masks [P] uint16, bit 3*dy+dx = tap kept
+    Returns y [N,Ho,Wo,C] float64; with `with_scale` also S = |bias| + sum |w*x|.
+    """
+    lib = _load()
+    x = np.asarray(x)
+    n, h, wd, c = x.shape
+    w = np.asarray(w)
+    if w.shape != (c, 3, 3):
+        raise ValueError("w must be [C,3,3]")
+    pid = np.ascontiguousarray(pid, dtype=np.int16)
+    if pid.shape != (c,):
+        raise ValueError("pid must be [C]")
+    masks = np.ascontiguousarray(masks, dtype=np.uint16)
+    ho, wo = out_shape(h, wd, stride)
+    xc = np.ascontiguousarray(x, dtype=np.float64)
+    wc = np.ascontiguousarray(w, dtype=np.float64)
+    bc = None if bias is None else np.ascontiguousarray(bias, dtype=np.float64)
+    y = np.empty((n, ho, wo, c), dtype=np.float64)
+    s = np.empty_like(y) if with_scale else None
+    rc = lib.dwconv_ref_f64(_ptr(xc), _ptr(wc), _ptr(pid), _ptr(masks), len(masks), _ptr(bc),
+                            int(bool(relu)), n, h, wd, c, stride, _ptr(y), _ptr(s))
     if rc:
         raise ValueError("oracle error %d" % rc)
     return (y, s) if with_scale else y

@@ -247,3 +247,54 @@ int patconv_ref_fused_i64(const int64_t *pre, const int32_t *residual, int relu,
                 }
     return 0;
 }
+
+/*
+ * Depthwise pattern-pruned 3x3 convolution (paper Sec. 2.1: pattern pruning "can
+ * generalize" beyond the dense 3x3 layer; here every channel has ONE 3x3 kernel of
+ * its own, which keeps the 4 weights of its pattern or is removed altogether):
+ *
+ *   pre[n,oy,ox,c] = bias[c] + sum_{dy,dx} Wm[c,dy,dx] * X[n, oy*s+dy-1, ox*s+dx-1, c]
+ *   Wm[c,dy,dx] = W[c,dy,dx] if pid[c] >= 0 and bit (3*dy+dx) of masks[pid[c]] is set, else 0
+ *
+ * with zero padding 1, stride s in {1,2}, Y = relu ? max(pre, 0) : pre.  Plain loops over
+ * the dense 9-tap kernels, double accumulation in the order (dy, dx).
+ *   x [n][h][w][c], wt [c][3][3], pid [c], bias [c] or NULL, y [n][ho][wo][c],
+ *   s_abs optional, shaped like y: |bias| + sum |Wm * X|.
+ * Parity status: pinned (a hand-computed case, the full layer's oracle with a diagonal
+ * connectivity, closed forms for constant input, pruned taps and removed channels
+ * contributing nothing, linearity, the error scale) -- tests/test_oracle_dwconv_pins.py.
+ * Returns 0, 1 for a pattern id outside the library, 2 for a bad shape.
+ */
+int dwconv_ref_f64(const double *x, const double *wt, const int16_t *pid, const uint16_t *masks, int P,
+                   const double *bias, int relu, int n, int h, int w, int c, int stride,
+                   double *y, double *s_abs) {
+    if (n < 0 || h < 1 || w < 1 || c < 1 || (stride != 1 && stride != 2)) return 2;
+    for (int ch = 0; ch < c; ++ch) if (pid[ch] >= P) return 1;
+    int ho = (h + 2 - 3) / stride + 1, wo = (w + 2 - 3) / stride + 1;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int in = 0; in < n; ++in) {
+        for (int oy = 0; oy < ho; ++oy) {
+            for (int ox = 0; ox < wo; ++ox) {
+                for (int ch = 0; ch < c; ++ch) {
+                    double acc = bias ? bias[ch] : 0.0;
+                    double sab = bias ? fabs(bias[ch]) : 0.0;
+                    const int p = pid[ch];
+                    for (int dy = 0; dy < 3; ++dy) {
+                        for (int dx = 0; dx < 3; ++dx) {
+                            const int keep = (p >= 0) && ((masks[p] >> (3 * dy + dx)) & 1);
+                            const int iy = oy * stride + dy - 1, ix = ox * stride + dx - 1;
+                            if (!keep || iy < 0 || iy >= h || ix < 0 || ix >= w) continue;
+                            const double t = wt[(size_t)ch * 9 + 3 * dy + dx] * x[(((size_t)in * h + iy) * w + ix) * c + ch];
+                            acc += t;
+                            sab += fabs(t);
+                        }
+                    }
+                    const size_t o = (((size_t)in * ho + oy) * wo + ox) * c + ch;
+                    y[o] = (relu && acc < 0.0) ? 0.0 : acc;
+                    if (s_abs) s_abs[o] = sab;
+                }
+            }
+        }
+    }
+    return 0;
+}

@@ -390,3 +390,81 @@ def config_resnet50_1x1(batch: int = 32, dtype: str = "f16", row_keep: float = 0
     return [GemmSpec(f"pw{i + 1}_{k}to{co}_{hw}", batch * hw * hw, k, co, br, bc, row_keep, col_keep,
                      dtype, "relu_normal", 0.01, True, i)
             for i, (k, co, hw) in enumerate(shapes)]
+
+
+# --- depthwise pattern-pruned 3x3 layers ---------------------------------------
+@dataclasses.dataclass
+class DepthwiseSpec:
+    """One depthwise 3x3 layer: every channel has one kernel, which keeps the 4 weights
+    of a pattern; a fraction `prune` of the channels loses its kernel altogether."""
+    name: str
+    n: int
+    c: int
+    h: int
+    w: int
+    stride: int = 1
+    dtype: str = "f32"            # "f32" | "f16"
+    prune: float = 0.0
+    lib_size: int = 8
+    x_dist: str = "relu_normal"
+    bias_sigma: float = 0.01
+    relu: bool = True
+    index: int = 0
+
+    @property
+    def ho(self) -> int:
+        return (self.h + 2 - 3) // self.stride + 1
+
+    @property
+    def wo(self) -> int:
+        return (self.w + 2 - 3) // self.stride + 1
+
+    @property
+    def k_surv(self) -> int:
+        return self.c - int(round(self.prune * self.c))
+
+    def useful_macs(self) -> int:
+        return 4 * self.k_surv * self.n * self.ho * self.wo
+
+    def compulsory_bytes(self) -> int:
+        b = 4 if self.dtype == "f32" else 2
+        return (self.n * self.h * self.w * self.c + self.n * self.ho * self.wo * self.c) * b + self.k_surv * (4 * b + 2) + 4 * self.c
+
+
+@dataclasses.dataclass
+class DepthwiseData:
+    spec: DepthwiseSpec
+    masks: np.ndarray     # uint16 [P]
+    pid: np.ndarray       # int16 [c], -1 = kernel removed
+    w: np.ndarray         # [c, 3, 3] (dense, unmasked)
+    bias: np.ndarray      # [c] float32
+    x: np.ndarray         # [n, h, w, c]
+
+
+def make_depthwise(spec: DepthwiseSpec, seed: int = BASE_SEED, n_override: int | None = None) -> DepthwiseData:
+    L = 2000 + spec.index                         # streams apart from the other layer kinds
+    n = spec.n if n_override is None else n_override
+    masks = pattern_library(spec.lib_size)
+    pid = integers(seed, "PID", L, spec.c, 0, spec.lib_size - 1).astype(np.int16)
+    n_pruned = int(round(spec.prune * spec.c))
+    if n_pruned:
+        pid[np.argsort(raw_u64(seed, "CONN", L, spec.c), kind="stable")[:n_pruned]] = -1
+    ft = np.float32 if spec.dtype == "f32" else np.float16
+    w = (normal(seed, "W", L, spec.c * 9) * math.sqrt(2.0 / 9.0)).astype(ft).reshape(spec.c, 3, 3)
+    nx = n * spec.h * spec.w * spec.c
+    if spec.x_dist == "relu_normal":
+        x64 = np.maximum(normal(seed, "X", L, nx), 0.0)
+    elif spec.x_dist == "upm1":
+        x64 = 2.0 * uniform01(seed, "X", L, nx) - 1.0
+    else:
+        x64 = uniform01(seed, "X", L, nx)
+    bias = (normal(seed, "B", L, spec.c) * spec.bias_sigma).astype(np.float32)
+    return DepthwiseData(spec, masks, pid, w, bias, x64.astype(ft).reshape(n, spec.h, spec.w, spec.c))
+
+
+def config_mobilenet_depthwise(batch: int = 32, dtype: str = "f16") -> list[DepthwiseSpec]:
+    """The distinct depthwise 3x3 layers of a MobileNet-v1-shaped network (channels x extent, stride)."""
+    shapes = [(32, 112, 1), (64, 112, 2), (128, 56, 1), (128, 56, 2), (256, 28, 1), (256, 28, 2),
+              (512, 14, 1), (512, 14, 2), (1024, 7, 1)]
+    return [DepthwiseSpec(f"dw{i + 1}_{c}_{hw}s{s}", batch, c, hw, hw, s, dtype, 0.0, 8, "relu_normal", 0.01, True, i)
+            for i, (c, hw, s) in enumerate(shapes)]
