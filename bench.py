@@ -314,6 +314,54 @@ def time_block_gemm(torch, binding, dev, stream, flush, fp32_tflops, hbm_gbs, or
     return out
 
 
+def time_depthwise(torch, binding, dev, stream, flush, hbm_gbs, oracle_check=True, only="", reps=5):
+    """Times xgen_dwconv_run on the depthwise 3x3 layers of a MobileNet-v1-shaped network (batch 32,
+    fp16 storage).  The layer is bound by HBM: per layer the achieved rate of its compulsory bytes
+    (x once, y once, kept weights) and that rate's fraction of the measured copy rate."""
+    out = {"layers": [], "recipe": "depthwise 3x3 layers of a MobileNet-v1-shaped network, batch 32, fp16 storage, NHWC, "
+                                   "8-pattern library, bias+ReLU fused"}
+    t_all = b_all = 0.0
+    for spec in wl.config_mobilenet_depthwise():
+        if only and not spec.name.startswith(only):
+            continue
+        d = wl.make_depthwise(spec)
+        pk = binding.Depthwise(spec.c, spec.stride, spec.dtype, d.masks, d.w, d.pid, device=dev.index)
+        x = torch.from_numpy(d.x).to(dev)
+        b = torch.from_numpy(d.bias).to(dev)
+        y = torch.empty((spec.n, spec.ho, spec.wo, spec.c), dtype=x.dtype, device=dev)
+        for _ in range(3):
+            pk.run(x.data_ptr(), spec.n, spec.h, spec.w, b.data_ptr(), True, y.data_ptr(), stream)
+        torch.cuda.synchronize()
+        ts = []
+        for r in range(reps):
+            flush.fill_(r)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            pk.run(x.data_ptr(), spec.n, spec.h, spec.w, b.data_ptr(), True, y.data_ptr(), stream)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        us = float(np.median(ts)) * 1e3
+        nbytes = spec.compulsory_bytes()
+        rec = {"layer": spec.name, "us": round(us, 2), "mbytes": round(nbytes / 1e6, 1), "gbs": round(nbytes / us * 1e-3, 1),
+               "frac_of_hbm": round(nbytes / us * 1e-3 / hbm_gbs, 4), "useful_gflops": round(2.0 * spec.useful_macs() / us * 1e-3, 1)}
+        if oracle_check and spec.c >= 512:
+            import oracle
+            got = y[:1].cpu().numpy().astype(np.float64)
+            ref, S = oracle.depthwise(d.x[:1], d.w, d.pid, d.masks, bias=d.bias, relu=True, stride=spec.stride, with_scale=True)
+            rec["parity_ok"] = bool((np.abs(got - ref) <= 2e-3 * np.maximum(np.abs(ref), 0.01 * S) + 2.0 ** -25).all())
+        out["layers"].append(rec)
+        t_all += us
+        b_all += nbytes
+        del pk, x, b, y
+    torch.cuda.empty_cache()
+    if t_all > 0:
+        out["total_us"] = round(t_all, 1)
+        out["gbs"] = round(b_all / t_all * 1e-3, 1)
+        out["frac_of_hbm"] = round(b_all / t_all * 1e-3 / hbm_gbs, 4)
+    return out
+
+
 def run_gpu(args):
     import torch
     from paper_2206_10620_b200 import binding
@@ -345,6 +393,13 @@ def run_gpu(args):
         rec = time_block_gemm(torch, binding, dev, torch.cuda.current_stream().cuda_stream, flush, fp32_peak, hbm,
                               oracle_check=False, only=args.block_gemm_only, reps=3)
         print(json.dumps({"block_gemm": rec, "measured_peaks": probe}), flush=True)
+        return
+
+    if args.depthwise_only:                         # profiling aid: one depthwise layer, nothing else
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        rec = time_depthwise(torch, binding, dev, torch.cuda.current_stream().cuda_stream, flush, hbm,
+                             oracle_check=False, only=args.depthwise_only, reps=3)
+        print(json.dumps({"depthwise": rec}), flush=True)
         return
 
     specs = workload(args.workload)
@@ -578,6 +633,10 @@ def run_gpu(args):
     if rank == 0 and world == 1 and not args.no_configs and args.workload == "vgg16" and not args.only:
         block_gemm = time_block_gemm(torch, binding, dev, stream, flush, fp32_peak, hbm, oracle_check=not args.no_parity)
 
+    depthwise = {}
+    if rank == 0 and world == 1 and not args.no_configs and args.workload == "vgg16" and not args.only:
+        depthwise = time_depthwise(torch, binding, dev, stream, flush, hbm, oracle_check=not args.no_parity)
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu = oracle_sample(specs, budget_s=args.cpu_seconds)
@@ -598,7 +657,7 @@ def run_gpu(args):
                 "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e,
                 "roofline": roofline, "measured_peaks": probe, "host_us_per_run_call": round(host_us, 2),
                 "parity_checked": parity_checked, "cpu_baseline": cpu, "per_layer": per_layer, "configs": configs, "fused": fused,
-                "block_gemm": block_gemm}
+                "block_gemm": block_gemm, "depthwise": depthwise}
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -620,6 +679,8 @@ def main():
     ap.add_argument("--no-parity", action="store_true", help="skip the oracle comparison of the timed layers")
     ap.add_argument("--block-gemm-only", default="", help="time only this layer of the block-pruned matrix products "
                     "(a prefix of its name, e.g. pw5) and print its record: profiling aid")
+    ap.add_argument("--depthwise-only", default="", help="time only this depthwise layer (a prefix of its name, e.g. dw3): "
+                    "profiling aid")
     ap.add_argument("--only", default="", help="comma-separated layer names: restrict the stack (profiling aid)")
     args = ap.parse_args()
     if args.impl == "reference":

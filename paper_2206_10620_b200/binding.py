@@ -28,7 +28,8 @@ EXPORTS = ["xgen_patconv_pack", "xgen_patconv_run", "xgen_patconv_run_static_scr
            "xgen_patconv_last_status", "xgen_patconv_free", "xgen_strerror",
            "xgen_patconv_launch_count", "xgen_patconv_probe", "xgen_patconv_run_fused",
            "xgen_blockgemm_pack", "xgen_blockgemm_run", "xgen_blockgemm_query", "xgen_blockgemm_view",
-           "xgen_blockgemm_free"]
+           "xgen_blockgemm_free",
+           "xgen_dwconv_pack", "xgen_dwconv_run", "xgen_dwconv_query", "xgen_dwconv_free"]
 
 
 class Desc(ctypes.Structure):
@@ -95,6 +96,11 @@ class GemmStats(ctypes.Structure):
                 ("max_stage_bytes", ctypes.c_int32)]
 
 
+class DwDesc(ctypes.Structure):
+    _fields_ = [("channels", ctypes.c_int32), ("stride", ctypes.c_int32), ("pad", ctypes.c_int32),
+                ("dtype", ctypes.c_int), ("num_patterns", ctypes.c_int32), ("pattern_masks", ctypes.c_void_p)]
+
+
 class GemmHostView(ctypes.Structure):
     _fields_ = [("units", ctypes.c_void_p), ("n_units", ctypes.c_int64), ("seg_off", ctypes.c_void_p)]
 
@@ -149,8 +155,14 @@ def lib():
         L.xgen_blockgemm_view.argtypes = [P, ctypes.POINTER(GemmHostView)]
         L.xgen_blockgemm_free.argtypes = [P]
         L.xgen_blockgemm_free.restype = None
+        L.xgen_dwconv_pack.argtypes = [ctypes.POINTER(DwDesc), P, P, ctypes.c_int, ctypes.POINTER(P)]
+        L.xgen_dwconv_run.argtypes = [P, P, I, I, I, P, I, P, P]
+        L.xgen_dwconv_query.argtypes = [P, ctypes.POINTER(ctypes.c_int64)]
+        L.xgen_dwconv_free.argtypes = [P]
+        L.xgen_dwconv_free.restype = None
         for name in EXPORTS:
-            if name not in ("xgen_patconv_free", "xgen_strerror", "xgen_patconv_launch_count", "xgen_blockgemm_free"):
+            if name not in ("xgen_patconv_free", "xgen_strerror", "xgen_patconv_launch_count", "xgen_blockgemm_free",
+                            "xgen_dwconv_free"):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -356,3 +368,43 @@ class BlockGemm:
         _check(lib().xgen_blockgemm_run(self._h, ctypes.c_void_p(x_ptr), int(m), ctypes.c_void_p(bias_ptr or None),
                                         int(bool(relu)), ctypes.c_void_p(y_ptr), ctypes.c_void_p(stream or None)),
                "xgen_blockgemm_run")
+
+
+class Depthwise:
+    """Owner of one xgen_dwconv_packed handle (depthwise pattern-pruned 3x3 layer)."""
+
+    def __init__(self, channels, stride, dtype, masks, dense_w, pattern_id, device=0, pad=1):
+        self._h = ctypes.c_void_p()
+        self.dtype = DTYPES[dtype] if isinstance(dtype, str) else int(dtype)
+        self.c, self.stride = int(channels), int(stride)
+        masks = np.ascontiguousarray(masks, dtype=np.uint16)
+        want = {F32: np.float32, F16_F32ACC: np.float16}.get(self.dtype, np.float32)
+        w = np.ascontiguousarray(dense_w, dtype=want)
+        pid = np.ascontiguousarray(pattern_id, dtype=np.int16)
+        if w.size != channels * 9 or pid.size != channels:
+            raise ValueError("dense_w must be [channels,3,3] and pattern_id [channels]")
+        d = DwDesc(channels, stride, pad, self.dtype, len(masks), masks.ctypes.data)
+        _check(lib().xgen_dwconv_pack(ctypes.byref(d), w.ctypes.data, pid.ctypes.data, int(device),
+                                      ctypes.byref(self._h)), "xgen_dwconv_pack")
+
+    def close(self):
+        if self._h:
+            lib().xgen_dwconv_free(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def kernels_surviving(self) -> int:
+        v = ctypes.c_int64()
+        _check(lib().xgen_dwconv_query(self._h, ctypes.byref(v)), "xgen_dwconv_query")
+        return v.value
+
+    def run(self, x_ptr, n, h, w, bias_ptr, relu, y_ptr, stream=0):
+        """Enqueue the layer on a CUDA stream; pointers are device addresses (ints)."""
+        _check(lib().xgen_dwconv_run(self._h, ctypes.c_void_p(x_ptr), n, h, w, ctypes.c_void_p(bias_ptr or None),
+                                     int(bool(relu)), ctypes.c_void_p(y_ptr), ctypes.c_void_p(stream or None)),
+               "xgen_dwconv_run")

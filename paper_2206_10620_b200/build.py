@@ -9,9 +9,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_HERE, "csrc")
 _INC = os.path.join(os.path.dirname(_HERE), "include")
 LIB_PATH = os.path.join(_HERE, "libpatconv.so")
-_SOURCES = ["patconv.cu", "blockgemm.cu", "probe.cu", "pack.cpp"]
+_SOURCES = ["patconv.cu", "blockgemm.cu", "dwconv.cu", "probe.cu", "pack.cpp"]
 _DEPS = _SOURCES + ["patconv_internal.h", "gen_core.py", "gen_blockgemm.py", os.path.join(_INC, "patconv.h"),
-                    os.path.join(_INC, "blockgemm.h")]
+                    os.path.join(_INC, "blockgemm.h"), os.path.join(_INC, "dwconv.h")]
 
 
 _OBJ_DIR = os.path.join(_HERE, "_build")
@@ -20,6 +20,7 @@ _INCLUDES = {
     "patconv.cu": ["patconv_internal.h", "gen_core.py", os.path.join(_INC, "patconv.h")],
     "blockgemm.cu": ["patconv_internal.h", "gen_blockgemm.py", os.path.join(_INC, "patconv.h"),
                      os.path.join(_INC, "blockgemm.h")],
+    "dwconv.cu": ["patconv_internal.h", os.path.join(_INC, "patconv.h"), os.path.join(_INC, "dwconv.h")],
     "probe.cu": [os.path.join(_INC, "patconv.h")],
     "pack.cpp": ["patconv_internal.h", os.path.join(_INC, "patconv.h")],
 }
