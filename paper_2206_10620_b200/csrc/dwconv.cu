@@ -43,7 +43,7 @@ struct DParams {
 };
 
 template <int DT, int V>
-__device__ __forceinline__ void load_vec(const void *x, size_t elem, float (&v)[V]) {
+__device__ __forceinline__ void load_vec(const void *x, unsigned elem, float (&v)[V]) {
     if constexpr (DT == XGEN_F32) {
         if constexpr (V == 4) {
             const float4 t = __ldg(reinterpret_cast<const float4 *>(static_cast<const float *>(x) + elem));
@@ -60,7 +60,7 @@ __device__ __forceinline__ void load_vec(const void *x, size_t elem, float (&v)[
 }
 
 template <int DT, int V>
-__device__ __forceinline__ void store_vec(void *y, size_t elem, const float (&v)[V]) {
+__device__ __forceinline__ void store_vec(void *y, unsigned elem, const float (&v)[V]) {
     if constexpr (DT == XGEN_F32) {
         if constexpr (V == 4) *reinterpret_cast<float4 *>(static_cast<float *>(y) + elem) = make_float4(v[0], v[1], v[2], v[3]);
         else static_cast<float *>(y)[elem] = v[0];
@@ -100,6 +100,16 @@ __global__ void __launch_bounds__(256) dwconv_kernel(const DParams P) {
         for (int t = 0; t < TX; ++t)
 #pragma unroll
             for (int v = 0; v < V; ++v) acc[t][v] = 0.0f;
+        // Tensors hold fewer than 2^31 elements, so element offsets are 32-bit.  Which of the strip's
+        // input columns lie inside the image is the same for the three rows: decided once.
+        unsigned col_off[NC];
+        bool col_ok[NC];
+#pragma unroll
+        for (int j = 0; j < NC; ++j) {
+            const int ix = ox0 * S + j - 1;
+            col_ok[j] = ix >= 0 && ix < P.w;
+            col_off[j] = (unsigned)(col_ok[j] ? ix : 0) * (unsigned)P.c + (unsigned)ch;
+        }
         // one input row at a time (holding all three rows in registers at once measured slower:
         // fewer threads fit an SM)
 #pragma unroll
@@ -108,13 +118,12 @@ __global__ void __launch_bounds__(256) dwconv_kernel(const DParams P) {
             if (iy < 0 || iy >= P.h) continue;
             float wt[3][V];
 #pragma unroll
-            for (int dx = 0; dx < 3; ++dx) load_vec<XGEN_F32, V>(P.w9, (size_t)(3 * dy + dx) * P.c + ch, wt[dx]);
+            for (int dx = 0; dx < 3; ++dx) load_vec<XGEN_F32, V>(P.w9, (unsigned)(3 * dy + dx) * (unsigned)P.c + (unsigned)ch, wt[dx]);
             float col[NC][V];
-            const size_t row = ((size_t)n * P.h + iy) * P.w;
+            const unsigned row = ((unsigned)n * (unsigned)P.h + (unsigned)iy) * (unsigned)P.w * (unsigned)P.c;
 #pragma unroll
             for (int j = 0; j < NC; ++j) {
-                const int ix = ox0 * S + j - 1;
-                if (ix >= 0 && ix < P.w) load_vec<DT, V>(P.x, (row + ix) * P.c + ch, col[j]);
+                if (col_ok[j]) load_vec<DT, V>(P.x, row + col_off[j], col[j]);
                 else {
 #pragma unroll
                     for (int v = 0; v < V; ++v) col[j][v] = 0.0f;
@@ -128,7 +137,7 @@ __global__ void __launch_bounds__(256) dwconv_kernel(const DParams P) {
                     for (int v = 0; v < V; ++v) acc[t][v] = fmaf(wt[dx][v], col[t * S + dx][v], acc[t][v]);
         }
         float b[V];
-        if (P.bias) load_vec<XGEN_F32, V>(P.bias, ch, b);
+        if (P.bias) load_vec<XGEN_F32, V>(P.bias, (unsigned)ch, b);
         else {
 #pragma unroll
             for (int v = 0; v < V; ++v) b[v] = 0.0f;
@@ -143,7 +152,7 @@ __global__ void __launch_bounds__(256) dwconv_kernel(const DParams P) {
                 o[v] = acc[t][v] + b[v];
                 if (P.relu) o[v] = fmaxf(o[v], 0.0f);
             }
-            store_vec<DT, V>(P.y, (((size_t)n * P.ho + oy) * P.wo + ox) * P.c + ch, o);
+            store_vec<DT, V>(P.y, (((unsigned)n * (unsigned)P.ho + (unsigned)oy) * (unsigned)P.wo + (unsigned)ox) * (unsigned)P.c + (unsigned)ch, o);
         }
     }
 }
